@@ -1,0 +1,383 @@
+// CPU oracle for the BF16 + stochastic-rounding AdamW update.
+//
+// THIS FILE IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It is a plain, slow, one-element-at-a-time
+// restatement of what the update computes, written from the paper's definitions so that a reader
+// can check it by eye.  It shares no code, header, table or helper with the CUDA library and the
+// CUDA library never calls it.  Only the test-suite, the smoke check and the benchmark's
+// CPU-baseline leg load it.
+//
+// What is defined here, and the passage each item follows:
+//   oracle_philox4x32_10      Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw, SC'11).  The
+//                             paper only asks for "a random state for the optimizer" that is equal
+//                             on every replica (Algorithm 1, REQUIRE list and the r <- r^(opt)
+//                             step); a counter-based generator gives that by construction.
+//   oracle_sr_bf16_bits       stochastic rounding Q_SR of Eq. 2, realised the way Section 3
+//                             describes it: take the FP32 value, add uniform noise below the bits
+//                             that BF16 keeps, shift the fraction out.
+//   oracle_rne_bf16_bits      nearest rounding Q of Eq. 1 in its IEEE round-half-to-even form.
+//   oracle_adamw_scalars      the per-iteration scalars of Algorithm 1 (bias corrections of the
+//                             m-hat and v-hat steps, alpha_t * lambda).
+//   oracle_adamw_element      one element of Algorithm 1 (moment updates, bias-corrected
+//                             direction, decoupled decay), in FP32, before any rounding.
+//   oracle_adamw_step         Algorithm 1 over an array: element function + Q_SR on x, m and v.
+//   oracle_sr_downcast        Q_SR applied to an FP32 array.
+//   oracle_sqnorm             sum of squares of the gradient with a fixed summation tree
+//   oracle_clip_scale         global-norm clipping coefficient.  (Neither is in the paper; they
+//                             are the usual companions of the update and are defined below.)
+//
+// Floating point: FP32 round-to-nearest-even for the element function (Section 3: the update
+// "temporarily upcasts to FP32"), no flush-to-zero, no contraction except where fmaf is written.
+// Build with -ffp-contract=off and without -ffast-math.
+//
+// Pins (tests/, run without a GPU): Philox known-answer vectors of its authors; Eq. 2's two-neighbour
+// property, exact P(up), exact mean (unbiasedness) and exact variance by enumerating all 65536
+// noise values; the stagnation and random-walk examples of Section 2; every FP32 intermediate of
+// the element function against correctly rounded exact rational arithmetic; the step-1 closed
+// form; a library AdamW as a loose bound; the summation tree against exact integer arithmetic.
+// Not pinned by the paper (its Algorithm 1 is ambiguous there; "parity unpinned" for that choice
+// alone): where epsilon sits relative to the square root.  This file uses the AdamW convention of
+// the optimizer the paper cites, sqrt(v/(1-beta2^t)) + epsilon.
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+namespace {
+
+inline uint32_t bits_of(float x) {
+    uint32_t b;
+    std::memcpy(&b, &x, sizeof b);
+    return b;
+}
+
+inline float float_of(uint32_t b) {
+    float x;
+    std::memcpy(&x, &b, sizeof x);
+    return x;
+}
+
+inline float bf16_to_float(uint16_t h) { return float_of(static_cast<uint32_t>(h) << 16); }
+
+inline bool is_nan_bits(uint32_t b) { return (b & 0x7FFFFFFFu) > 0x7F800000u; }
+
+constexpr uint16_t kCanonicalNaN = 0x7FC0;
+
+// ---- Philox4x32-10 -------------------------------------------------------------------------
+// One round maps the counter (c0,c1,c2,c3) under the round key (k0,k1) to
+//   ( hi(M1*c2) ^ c1 ^ k0,  lo(M1*c2),  hi(M0*c0) ^ c3 ^ k1,  lo(M0*c0) )
+// with 32x32->64 bit products; between rounds the key advances by the Weyl constants.
+void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+    const uint64_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+    const uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        if (round > 0) {
+            k0 += W0;
+            k1 += W1;
+        }
+        const uint64_t p0 = M0 * c0;
+        const uint64_t p1 = M1 * c2;
+        const uint32_t n0 = static_cast<uint32_t>(p1 >> 32) ^ c1 ^ k0;
+        const uint32_t n1 = static_cast<uint32_t>(p1);
+        const uint32_t n2 = static_cast<uint32_t>(p0 >> 32) ^ c3 ^ k1;
+        const uint32_t n3 = static_cast<uint32_t>(p0);
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// ---- the optimizer's random state r^(opt)_t ------------------------------------------------
+// Algorithm 1 needs a random state that is the same on every replica at iteration t.  Here the
+// state is a pure function of (seed, step, tensor_id, global element index):
+//   key     = (seed[31:0], step)
+//   counter = (index[31:0], index[63:32], tensor_id, seed[63:32])
+// and the four output words serve, in order, the roundings of x, m and v (the fourth is unused).
+// Each rounding consumes the top 16 bits of its word.
+struct Noise3 { uint32_t rp, rm, rv; };
+
+Noise3 noise_for(uint64_t seed, uint32_t step, uint32_t tensor_id, uint64_t index) {
+    const uint32_t ctr[4] = {static_cast<uint32_t>(index), static_cast<uint32_t>(index >> 32),
+                             tensor_id, static_cast<uint32_t>(seed >> 32)};
+    const uint32_t key[2] = {static_cast<uint32_t>(seed), step};
+    uint32_t w[4];
+    philox4x32_10(ctr, key, w);
+    return Noise3{w[0] >> 16, w[1] >> 16, w[2] >> 16};
+}
+
+// ---- Eq. 2 by dithering --------------------------------------------------------------------
+// BF16 keeps the top 16 bits of the FP32 pattern; the low 16 bits are the position of x between
+// its two BF16 neighbours, in units of 2^-16 of their distance.  Adding a uniform integer
+// r in [0, 65536) to the pattern carries into the kept bits exactly when low16 + r >= 65536,
+// i.e. for low16 of the 65536 values of r: probability (x - floor)/Delta of moving to the
+// neighbour away from zero, as Eq. 2 asks.  The pattern is sign-magnitude, so one unsigned add
+// serves both signs, crosses binades and the subnormal boundary, and leaves values that are
+// already BF16 (low16 == 0), zeros and infinities untouched.  A finite value beyond the largest
+// finite BF16 moves to infinity with the same rule.  Any NaN becomes the one quiet NaN 0x7FC0, so
+// that the result does not depend on which NaN payload a platform produces.
+uint16_t sr_bf16_bits(uint32_t fbits, uint32_t r16) {
+    if (is_nan_bits(fbits)) return kCanonicalNaN;
+    return static_cast<uint16_t>((fbits + (r16 & 0xFFFFu)) >> 16);
+}
+
+// ---- Eq. 1, IEEE form ----------------------------------------------------------------------
+// Round to the nearer neighbour; a value exactly half-way goes to the neighbour whose last kept
+// bit is zero.
+uint16_t rne_bf16_bits(uint32_t fbits) {
+    if (is_nan_bits(fbits)) return kCanonicalNaN;
+    const uint32_t last_kept = (fbits >> 16) & 1u;
+    return static_cast<uint16_t>((fbits + 0x7FFFu + last_kept) >> 16);
+}
+
+// beta^t by repeated squaring in double; no libm call, so every platform gets the same bits.
+double int_power(double base, uint32_t exponent) {
+    double result = 1.0;
+    while (exponent != 0) {
+        if (exponent & 1u) result *= base;
+        base *= base;
+        exponent >>= 1;
+    }
+    return result;
+}
+
+}  // namespace
+
+extern "C" {
+
+// Hyper-parameters as the caller states them (Algorithm 1, REQUIRE list; epsilon of the update).
+struct oracle_hparams {
+    float lr;            // alpha_t
+    float beta1;
+    float beta2;
+    float eps;
+    float weight_decay;  // lambda
+    uint32_t flags;      // bit0/1/2: stochastic rounding on x / m / v (else nearest-even)
+};
+
+// Scalars that are the same for every element of one iteration.
+struct oracle_scalars {
+    float beta1;
+    float beta2;
+    float one_minus_beta1;  // FP32 subtraction
+    float one_minus_beta2;
+    float step_size;        // alpha_t / (1 - beta1^t)          (the m-hat step folded into alpha_t)
+    float rsqrt_bc2;        // 1 / sqrt(1 - beta2^t)            (the v-hat step)
+    float eps;
+    float lr_wd;            // alpha_t * lambda
+};
+
+// The FP32 intermediates of one element, in the order they are produced.
+struct oracle_trace {
+    float g;      // gscale * g_in
+    float a;      // (1-beta1) * g
+    float m_new;  // beta1*m + a                     (moment update for m)
+    float b1;     // (1-beta2) * g
+    float b2;     // b1 * g
+    float v_new;  // beta2*v + b2                    (moment update for v)
+    float s;      // sqrt(v_new)
+    float den;    // s * rsqrt_bc2 + eps
+    float u;      // m_new / den
+    float w;      // lr_wd * x
+    float q;      // step_size*u + w
+    float x_new;  // x - q                           (argument of Q_SR in the update step)
+};
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+    philox4x32_10(ctr, key, out);
+}
+
+// The three 16-bit noise values (x, m, v) for one element.
+void oracle_noise(uint64_t seed, uint32_t step, uint32_t tensor_id, uint64_t index, uint32_t out[3]) {
+    const Noise3 r = noise_for(seed, step, tensor_id, index);
+    out[0] = r.rp; out[1] = r.rm; out[2] = r.rv;
+}
+
+uint16_t oracle_sr_bf16_bits(uint32_t fbits, uint32_t r16) { return sr_bf16_bits(fbits, r16); }
+
+uint16_t oracle_rne_bf16_bits(uint32_t fbits) { return rne_bf16_bits(fbits); }
+
+// Returns 0 on success, 1 for arguments the update is not defined for.
+int oracle_adamw_scalars(const oracle_hparams* hp, uint32_t step, oracle_scalars* out) {
+    if (step == 0) return 1;  // 1 - beta^0 = 0: the bias correction divides by zero
+    const double b1 = hp->beta1, b2 = hp->beta2, lr = hp->lr, wd = hp->weight_decay;
+    const double bc1 = 1.0 - int_power(b1, step);
+    const double bc2 = 1.0 - int_power(b2, step);
+    out->beta1 = hp->beta1;
+    out->beta2 = hp->beta2;
+    out->one_minus_beta1 = 1.0f - hp->beta1;
+    out->one_minus_beta2 = 1.0f - hp->beta2;
+    out->step_size = static_cast<float>(lr / bc1);
+    out->rsqrt_bc2 = static_cast<float>(1.0 / std::sqrt(bc2));
+    out->eps = hp->eps;
+    out->lr_wd = static_cast<float>(lr * wd);
+    return 0;
+}
+
+// One element of Algorithm 1 in FP32.  Each line is one correctly rounded operation; fmaf is a
+// single rounding of a*b+c.
+void oracle_adamw_element(float x, float g_in, float m, float v, float gscale,
+                          const oracle_scalars* sc, oracle_trace* t) {
+    t->g = gscale * g_in;
+    t->a = sc->one_minus_beta1 * t->g;
+    t->m_new = fmaf(sc->beta1, m, t->a);
+    t->b1 = sc->one_minus_beta2 * t->g;
+    t->b2 = t->b1 * t->g;
+    t->v_new = fmaf(sc->beta2, v, t->b2);
+    t->s = sqrtf(t->v_new);
+    t->den = fmaf(t->s, sc->rsqrt_bc2, sc->eps);
+    t->u = t->m_new / t->den;
+    t->w = sc->lr_wd * x;
+    t->q = fmaf(sc->step_size, t->u, t->w);
+    t->x_new = x - t->q;
+}
+
+// Algorithm 1 on n elements, in place.  p, m, v hold BF16 bit patterns; g is BF16 (g_is_f32 == 0)
+// or FP32 (g_is_f32 == 1).  elem_offset is the global index of element 0, so that a shard of a
+// larger buffer draws the same noise as the whole would.
+int oracle_adamw_step(uint16_t* p, const void* g, int g_is_f32, uint16_t* m, uint16_t* v, uint64_t n,
+                      const oracle_hparams* hp, float gscale, uint64_t seed, uint32_t step,
+                      uint32_t tensor_id, uint64_t elem_offset) {
+    oracle_scalars sc;
+    if (oracle_adamw_scalars(hp, step, &sc) != 0) return 1;
+    const uint16_t* g16 = static_cast<const uint16_t*>(g);
+    const float* g32 = static_cast<const float*>(g);
+    const bool sr_p = hp->flags & 1u, sr_m = hp->flags & 2u, sr_v = hp->flags & 4u;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < static_cast<int64_t>(n); ++i) {
+        const float gi = g_is_f32 ? g32[i] : bf16_to_float(g16[i]);
+        oracle_trace t;
+        oracle_adamw_element(bf16_to_float(p[i]), gi, bf16_to_float(m[i]), bf16_to_float(v[i]), gscale, &sc, &t);
+        const Noise3 r = noise_for(seed, step, tensor_id, elem_offset + static_cast<uint64_t>(i));
+        p[i] = sr_p ? sr_bf16_bits(bits_of(t.x_new), r.rp) : rne_bf16_bits(bits_of(t.x_new));
+        m[i] = sr_m ? sr_bf16_bits(bits_of(t.m_new), r.rm) : rne_bf16_bits(bits_of(t.m_new));
+        v[i] = sr_v ? sr_bf16_bits(bits_of(t.v_new), r.rv) : rne_bf16_bits(bits_of(t.v_new));
+    }
+    return 0;
+}
+
+// Q_SR on an FP32 array; uses the first noise word only.
+void oracle_sr_downcast(const float* src, uint16_t* dst, uint64_t n, uint64_t seed, uint32_t step,
+                        uint32_t tensor_id, uint64_t elem_offset) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < static_cast<int64_t>(n); ++i) {
+        const Noise3 r = noise_for(seed, step, tensor_id, elem_offset + static_cast<uint64_t>(i));
+        dst[i] = sr_bf16_bits(bits_of(src[i]), r.rp);
+    }
+}
+
+// ---- sum of squares with a fixed tree ------------------------------------------------------
+// One reduction pass turns an array of L doubles into ceil(L/8192) doubles.  Inside a block of
+// 8192 consecutive entries there are 256 accumulators; accumulator j adds, in this order, the
+// entries  r*1024 + 4*j + k  for r = 0..7, k = 0..3  (entries past the end are skipped).  The 256
+// accumulators form 8 groups of 32; each group is folded by a butterfly (partner = lane XOR 16,
+// 8, 4, 2, 1; after it every lane of the group holds the same value) and the 8 group values are
+// added in order 0..7.  Passes repeat until one value is left.  The first pass works on the
+// squares g_i*g_i, which are exact in double for FP32 or BF16 g_i.
+static double fold_block(const double* terms, uint64_t count) {
+    double acc[256];
+    for (int j = 0; j < 256; ++j) {
+        double a = 0.0;
+        for (int r = 0; r < 8; ++r)
+            for (int k = 0; k < 4; ++k) {
+                const uint64_t e = static_cast<uint64_t>(r) * 1024u + 4u * static_cast<uint64_t>(j) + static_cast<uint64_t>(k);
+                if (e < count) a += terms[e];
+            }
+        acc[j] = a;
+    }
+    double group[8];
+    for (int w = 0; w < 8; ++w) {
+        double lane[32];
+        for (int l = 0; l < 32; ++l) lane[l] = acc[32 * w + l];
+        for (int s = 16; s >= 1; s >>= 1) {
+            double next[32];
+            for (int l = 0; l < 32; ++l) next[l] = lane[l] + lane[l ^ s];
+            for (int l = 0; l < 32; ++l) lane[l] = next[l];
+        }
+        group[w] = lane[0];
+    }
+    double total = group[0];
+    for (int w = 1; w < 8; ++w) total += group[w];
+    return total;
+}
+
+double oracle_sqnorm(const void* g, int g_is_f32, uint64_t n) {
+    if (n == 0) return 0.0;
+    const uint16_t* g16 = static_cast<const uint16_t*>(g);
+    const float* g32 = static_cast<const float*>(g);
+    uint64_t count = (n + 8191u) / 8192u;
+    double* level = new double[count];
+#pragma omp parallel for schedule(static)
+    for (int64_t c = 0; c < static_cast<int64_t>(count); ++c) {
+        const uint64_t base = static_cast<uint64_t>(c) * 8192u;
+        const uint64_t len = (n - base < 8192u) ? (n - base) : 8192u;
+        double sq[8192];
+        for (uint64_t e = 0; e < len; ++e) {
+            const double gi = g_is_f32 ? static_cast<double>(g32[base + e])
+                                       : static_cast<double>(bf16_to_float(g16[base + e]));
+            sq[e] = gi * gi;
+        }
+        level[c] = fold_block(sq, len);
+    }
+    while (count > 1) {
+        const uint64_t next_count = (count + 8191u) / 8192u;
+        double* next = new double[next_count];
+        for (uint64_t c = 0; c < next_count; ++c) {
+            const uint64_t base = c * 8192u;
+            const uint64_t len = (count - base < 8192u) ? (count - base) : 8192u;
+            next[c] = fold_block(level + base, len);
+        }
+        delete[] level;
+        level = next;
+        count = next_count;
+    }
+    const double result = level[0];
+    delete[] level;
+    return result;
+}
+
+// Same tree applied to an array of doubles (used to check the later passes on their own).
+double oracle_tree_sum(const double* terms, uint64_t n) {
+    if (n == 0) return 0.0;
+    uint64_t count = n;
+    double* level = new double[count];
+    std::memcpy(level, terms, count * sizeof(double));
+    while (count > 1) {
+        const uint64_t next_count = (count + 8191u) / 8192u;
+        double* next = new double[next_count];
+        for (uint64_t c = 0; c < next_count; ++c) {
+            const uint64_t base = c * 8192u;
+            const uint64_t len = (count - base < 8192u) ? (count - base) : 8192u;
+            next[c] = fold_block(level + base, len);
+        }
+        delete[] level;
+        level = next;
+        count = next_count;
+    }
+    const double result = level[0];
+    delete[] level;
+    return result;
+}
+
+// Global-norm clipping with a gradient-accumulation factor: the true gradient is accum_scale * g,
+// its norm is accum_scale * sqrt(S); the factor applied to g is accum_scale * min(1, max_norm /
+// (norm + 1e-6)).  Evaluated in double, returned as FP32.
+float oracle_clip_scale(double sqnorm, float accum_scale, float max_norm) {
+    const double norm = static_cast<double>(accum_scale) * std::sqrt(sqnorm);
+    double coef = static_cast<double>(max_norm) / (norm + 1e-6);
+    if (coef > 1.0) coef = 1.0;
+    return static_cast<float>(static_cast<double>(accum_scale) * coef);
+}
+
+}  // extern "C"
