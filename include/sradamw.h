@@ -1,0 +1,127 @@
+/*
+ * sradamw.h -- C ABI of libsradamw.so: the BF16 + stochastic-rounding AdamW update on one B200.
+ *
+ * The update is Algorithm 1 ("AdamW with Stochastic Rounding and Shared Randomness"): parameters x,
+ * gradients g and both moments m, v are stored in BF16; one iteration reads them, evaluates the
+ * AdamW formulas in FP32 registers and writes x, m, v back to BF16 with stochastic rounding Q_SR
+ * (Eq. 2), implemented the way Section 3 describes: add uniform noise below the kept bits of the
+ * FP32 pattern, then drop the low half.  No FP32 master copy and no auxiliary tensor exists.
+ *
+ * Conventions for every call
+ *   - Data pointers are DEVICE pointers owned by the caller unless a parameter says "host".
+ *     BF16 arrays are passed as uint16_t bit patterns.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls enqueue work and
+ *     return; they never synchronise the device and never allocate device memory, except
+ *     sr_mt_plan_create / sr_mt_plan_destroy.
+ *   - x, m, v are updated in place; g is only read.  Buffers of one call must not overlap each other.
+ *   - n == 0 is a successful no-op.  Any base alignment is accepted; the 16-byte vector path needs
+ *     all buffers of a call 16-byte aligned and otherwise an element-wise path is taken.
+ *   - Errors are returned, never thrown; nothing is written when a call returns an error other
+ *     than SR_ERR_CUDA.  The device must have compute capability 10.x.
+ *
+ * The optimizer's random state (Algorithm 1: r^(opt)_t, equal on every replica) is a pure function
+ * of the arguments: Philox4x32-10 with key (seed[31:0], step) and counter
+ * (index[31:0], index[63:32], tensor_id, seed[63:32]), index = elem_offset + position in the buffer.
+ * Output words 0, 1, 2 serve the roundings of x, m, v; each rounding uses the top 16 bits of its
+ * word.  Two ranks, two shards or two runs with equal (seed, step, tensor_id, index) therefore
+ * round identically, which is what the shared random state of Algorithm 1 is for.
+ */
+#ifndef SRADAMW_H
+#define SRADAMW_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SR_ABI_VERSION 1u
+
+typedef enum {
+    SR_OK = 0,
+    SR_ERR_INVALID_ARG = 1,        /* null pointer, step 0 for AdamW, bad hyper-parameter or struct size */
+    SR_ERR_UNSUPPORTED_DEVICE = 2, /* current device is not compute capability 10.x                      */
+    SR_ERR_WORKSPACE = 3,          /* workspace missing or too small                                     */
+    SR_ERR_CUDA = 4                /* a CUDA runtime call failed; see sr_last_cuda_error()                */
+} sr_status;
+
+typedef enum { SR_DT_BF16 = 0, SR_DT_F32 = 1 } sr_dtype; /* gradient storage; x, m, v are always BF16 */
+
+/* flags of sr_adamw_hparams: which of the three downcasts use Q_SR (Eq. 2); the others use
+ * round-to-nearest-even (Eq. 1).  Algorithm 1 itself needs SR_FLAG_SR_P only. */
+#define SR_FLAG_SR_P 1u
+#define SR_FLAG_SR_M 2u
+#define SR_FLAG_SR_V 4u
+#define SR_FLAGS_DEFAULT 7u
+
+/* Hyper-parameters of one iteration (Algorithm 1, REQUIRE list).  Host memory, read during the call. */
+typedef struct sr_adamw_hparams {
+    uint32_t struct_size;        /* sizeof(sr_adamw_hparams); checked                                        */
+    float lr;                    /* alpha_t, finite, >= 0                                                     */
+    float beta1;                 /* in [0, 1)                                                                 */
+    float beta2;                 /* in [0, 1)                                                                 */
+    float eps;                   /* finite, >= 0; added to sqrt(v-hat), outside the square root               */
+    float weight_decay;          /* lambda, finite; decoupled: the decay term is alpha_t * lambda * x          */
+    float grad_scale;            /* g is multiplied by this before use when grad_scale_dev is NULL (1 = none) */
+    const float* grad_scale_dev; /* optional DEVICE scalar (e.g. from sr_clip_scale); read by the kernel       */
+    uint32_t flags;              /* SR_FLAG_*; other bits must be zero                                         */
+} sr_adamw_hparams;
+
+/* Eq. 2 on an array: dst[i] = Q_SR(src[i]) using noise word 0 at index elem_offset + i.
+ * src: n FP32 values; dst: n BF16 patterns.  step may be 0 here.
+ * NaN inputs give the quiet NaN 0x7FC0; +-0, +-inf and values already representable pass through. */
+sr_status sr_downcast_f32_bf16(const float* src, uint16_t* dst, uint64_t n, uint64_t seed, uint32_t step,
+                               uint32_t tensor_id, uint64_t elem_offset, void* stream);
+
+/* One iteration of Algorithm 1 on a flat buffer of n elements (moment updates, bias-corrected
+ * direction with epsilon outside the square root, decoupled weight decay, rounding of x, m, v).
+ * p, m, v: BF16 in/out.  g: BF16 or FP32 per g_dtype.  step >= 1 is the 1-based iteration t.
+ * elem_offset is the global index of element 0, so a shard of a larger buffer rounds as the whole
+ * buffer would. */
+sr_status sr_adamw_step(uint16_t* p, const void* g, sr_dtype g_dtype, uint16_t* m, uint16_t* v, uint64_t n,
+                        const sr_adamw_hparams* hp, uint64_t seed, uint32_t step, uint32_t tensor_id,
+                        uint64_t elem_offset, void* stream);
+
+/* The same iteration over a list of tensors in one launch.  A plan owns device copies of the
+ * pointer / size table and of the chunk table that maps thread blocks to (tensor, range).
+ * The arrays passed to sr_mt_plan_create are HOST arrays of num_tensors entries holding device
+ * pointers and element counts; they may be freed after the call.  Tensor i uses
+ * tensor_id = tensor_id_base + i and element indices starting at 0.  One hparams set serves the list.
+ * The plan stays valid while the tensors it names stay allocated; destroy it with
+ * sr_mt_plan_destroy (which synchronises nothing: do not destroy while a step using it is in flight). */
+typedef struct sr_mt_plan sr_mt_plan;
+sr_status sr_mt_plan_create(sr_mt_plan** out, uint32_t num_tensors, uint16_t* const* p, const void* const* g,
+                            uint16_t* const* m, uint16_t* const* v, const uint64_t* numel, sr_dtype g_dtype,
+                            void* stream);
+sr_status sr_adamw_multi_tensor(const sr_mt_plan* plan, const sr_adamw_hparams* hp, uint64_t seed, uint32_t step,
+                                uint32_t tensor_id_base, void* stream);
+sr_status sr_mt_plan_destroy(sr_mt_plan* plan);
+uint64_t sr_mt_plan_total_elements(const sr_mt_plan* plan);
+
+/* Sum of squares of the gradient for global-norm clipping (not part of the paper; the usual
+ * companion of the update).  The sum is taken in FP64 over exact squares with a fixed tree that
+ * does not depend on the launch shape: blocks of 8192 consecutive entries; inside a block 256
+ * accumulators, accumulator j adding entries r*1024 + 4j + k (r = 0..7, k = 0..3) in that order;
+ * 8 groups of 32 accumulators folded by an XOR butterfly (16, 8, 4, 2, 1), group values added in
+ * order; the block sums are reduced again by the same rule until one value is left.
+ * out_dev: one double on the device.  workspace: device memory of at least
+ * grad_sqnorm_workspace_bytes(n) bytes, 8-byte aligned (may be NULL when that size is 0). */
+size_t grad_sqnorm_workspace_bytes(uint64_t n);
+sr_status grad_sqnorm(const void* g, sr_dtype g_dtype, uint64_t n, double* out_dev, void* workspace,
+                      size_t workspace_bytes, void* stream);
+
+/* Clipping factor on the device, no host round trip:
+ * gscale = accum_scale * min(1, max_norm / (accum_scale * sqrt(S) + 1e-6)), evaluated in FP64 and
+ * stored as FP32 in *gscale_out_dev; pass that pointer as sr_adamw_hparams.grad_scale_dev. */
+sr_status sr_clip_scale(const double* sqnorm_dev, float accum_scale, float max_norm, float* gscale_out_dev,
+                        void* stream);
+
+const char* sr_status_string(sr_status s);
+int sr_last_cuda_error(void); /* cudaError_t of the last failing runtime call on this thread, else 0 */
+uint32_t sr_abi_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SRADAMW_H */

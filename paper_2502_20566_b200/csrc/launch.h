@@ -1,0 +1,53 @@
+// Internal launcher interface between the C-ABI layer (api.cu) and the kernel translation units.
+#pragma once
+
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "device_math.cuh"
+
+namespace sradamw {
+
+// Device-side tables of a multi-tensor plan.
+struct MtTensor {
+    uint16_t* p;
+    const void* g;
+    uint16_t* m;
+    uint16_t* v;
+    uint64_t n;
+    uint32_t vec_ok;   // all four pointers 16-byte aligned
+    uint32_t pad;
+};
+
+struct MtChunk {
+    uint32_t tensor;   // index into the tensor table
+    uint32_t chunk;    // chunk number inside that tensor; first element = chunk * kMtChunkElems
+};
+
+constexpr uint32_t kMtChunkElems = 16384;   // multiple of 8 * block size
+constexpr int kBlockThreads = 256;
+
+struct DeviceInfo {
+    int sm_count;
+    int cc_major;
+};
+
+cudaError_t launch_downcast(const float* src, uint16_t* dst, uint64_t n, uint64_t elem_offset, uint32_t tensor_id,
+                            uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev, cudaStream_t stream);
+
+cudaError_t launch_adamw_flat(uint16_t* p, const void* g, bool g_f32, uint16_t* m, uint16_t* v, uint64_t n,
+                              uint64_t elem_offset, uint32_t tensor_id, uint32_t seed_hi, uint32_t flags,
+                              const PhiloxKeys& K, const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream);
+
+cudaError_t launch_adamw_mt(const MtTensor* tensors, const MtChunk* chunks, uint32_t num_chunks, bool g_f32,
+                            uint32_t tensor_id_base, uint32_t seed_hi, uint32_t flags, const PhiloxKeys& K,
+                            const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream);
+
+// Squared norm: number of doubles of scratch needed, and the launcher.
+uint64_t sqnorm_scratch_doubles(uint64_t n);
+cudaError_t launch_sqnorm(const void* g, bool g_f32, uint64_t n, double* out, double* scratch,
+                          const DeviceInfo& dev, cudaStream_t stream);
+cudaError_t launch_clip_scale(const double* sqnorm, float accum_scale, float max_norm, float* out,
+                              cudaStream_t stream);
+
+}  // namespace sradamw

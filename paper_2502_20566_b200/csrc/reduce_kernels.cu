@@ -1,0 +1,170 @@
+// Squared gradient norm with a fixed FP64 summation tree, and the clipping factor.
+//
+// The tree is part of the library's contract (the result must not depend on the launch shape):
+// blocks of 8192 consecutive entries; inside a block 256 accumulators, accumulator j adding the
+// entries r*1024 + 4j + k (r = 0..7, k = 0..3) in that order; 8 warps folded by an XOR butterfly
+// (16, 8, 4, 2, 1), warp values added in order 0..7; block sums reduced again by the same rule.
+// A CUDA block of 256 threads is exactly one tree block, so thread j is accumulator j and the
+// loads of one r are 16-byte, fully coalesced.  HBM-bound: 4 (FP32) or 2 (BF16) bytes per element.
+
+#include "launch.h"
+
+namespace sradamw {
+
+namespace {
+
+constexpr uint32_t kTreeBlock = 8192;
+
+// squares are exact in double for FP32 / BF16 inputs, so fma(g, g, acc) rounds once, exactly like
+// acc + g*g
+__device__ __forceinline__ double add_square(double acc, float g) {
+    const double d = static_cast<double>(g);
+    return __fma_rn(d, d, acc);
+}
+
+__device__ __forceinline__ double fold_block(double acc, double* warp_sums) {
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) acc = __dadd_rn(acc, __shfl_xor_sync(0xFFFFFFFFu, acc, s));
+    const int warp = threadIdx.x >> 5;
+    if ((threadIdx.x & 31) == 0) warp_sums[warp] = acc;
+    __syncthreads();
+    double total = 0.0;
+    if (threadIdx.x == 0) {
+        total = warp_sums[0];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) total = __dadd_rn(total, warp_sums[w]);
+    }
+    __syncthreads();
+    return total;   // valid in thread 0
+}
+
+// First pass: out[c] = tree-block sum of squares of entries [c*8192, (c+1)*8192) of g.
+template <bool G32>
+__global__ void __launch_bounds__(kBlockThreads)
+k_sqnorm_pass1(const void* __restrict__ g, uint64_t n, uint64_t num_blocks, bool vec_ok, double* __restrict__ out) {
+    __shared__ double warp_sums[8];
+    const uint32_t j = threadIdx.x;
+    for (uint64_t c = blockIdx.x; c < num_blocks; c += gridDim.x) {
+        const uint64_t base = c * kTreeBlock;
+        double acc = 0.0;
+        if (vec_ok && n - base >= kTreeBlock) {
+            if (G32) {
+                const float4* src = reinterpret_cast<const float4*>(static_cast<const float*>(g) + base) + j;
+                float4 q[8];
+#pragma unroll
+                for (int r = 0; r < 8; ++r) q[r] = __ldcs(src + r * 256);
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    acc = add_square(acc, q[r].x);
+                    acc = add_square(acc, q[r].y);
+                    acc = add_square(acc, q[r].z);
+                    acc = add_square(acc, q[r].w);
+                }
+            } else {
+                const uint2* src = reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(g) + base) + j;
+                uint2 q[8];
+#pragma unroll
+                for (int r = 0; r < 8; ++r) q[r] = __ldcs(src + r * 256);
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    acc = add_square(acc, bf16_lo(q[r].x));
+                    acc = add_square(acc, bf16_hi(q[r].x));
+                    acc = add_square(acc, bf16_lo(q[r].y));
+                    acc = add_square(acc, bf16_hi(q[r].y));
+                }
+            }
+        } else {
+            for (int r = 0; r < 8; ++r)
+                for (int k = 0; k < 4; ++k) {
+                    const uint64_t e = base + static_cast<uint64_t>(r) * 1024u + 4u * j + k;
+                    if (e < n) {
+                        const float gi = G32 ? static_cast<const float*>(g)[e]
+                                             : __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t*>(g)[e]) << 16);
+                        acc = add_square(acc, gi);
+                    }
+                }
+        }
+        const double total = fold_block(acc, warp_sums);
+        if (j == 0) out[c] = total;
+    }
+}
+
+// Later passes: the same rule on an array of doubles (no squaring).
+__global__ void __launch_bounds__(kBlockThreads)
+k_tree_pass(const double* __restrict__ in, uint64_t count, uint64_t num_blocks, double* __restrict__ out) {
+    __shared__ double warp_sums[8];
+    const uint32_t j = threadIdx.x;
+    for (uint64_t c = blockIdx.x; c < num_blocks; c += gridDim.x) {
+        const uint64_t base = c * kTreeBlock;
+        double acc = 0.0;
+        for (int r = 0; r < 8; ++r)
+            for (int k = 0; k < 4; ++k) {
+                const uint64_t e = base + static_cast<uint64_t>(r) * 1024u + 4u * j + k;
+                if (e < count) acc = __dadd_rn(acc, in[e]);
+            }
+        const double total = fold_block(acc, warp_sums);
+        if (j == 0) out[c] = total;
+    }
+}
+
+__global__ void k_clip_scale(const double* __restrict__ sqnorm, float accum_scale, float max_norm,
+                             float* __restrict__ out) {
+    const double a = static_cast<double>(accum_scale);
+    const double norm = __dmul_rn(a, __dsqrt_rn(*sqnorm));
+    double coef = __ddiv_rn(static_cast<double>(max_norm), __dadd_rn(norm, 1e-6));
+    if (coef > 1.0) coef = 1.0;
+    *out = __double2float_rn(__dmul_rn(a, coef));
+}
+
+inline uint64_t blocks_of(uint64_t count) { return (count + kTreeBlock - 1) / kTreeBlock; }
+
+}  // namespace
+
+// Scratch holds every intermediate level: ceil(n/8192) + ceil(that/8192) + ... down to, but not
+// including, the final single value (which goes to the caller's output).
+uint64_t sqnorm_scratch_doubles(uint64_t n) {
+    uint64_t total = 0;
+    uint64_t count = blocks_of(n);
+    while (count > 1) {
+        total += count;
+        count = blocks_of(count);
+    }
+    return total;
+}
+
+cudaError_t launch_sqnorm(const void* g, bool g_f32, uint64_t n, double* out, double* scratch,
+                          const DeviceInfo& dev, cudaStream_t stream) {
+    if (n == 0) return cudaMemsetAsync(out, 0, sizeof(double), stream);
+    uint64_t count = blocks_of(n);
+    double* level_out = count == 1 ? out : scratch;
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(g) & 15u) == 0;
+    const uint64_t cap = static_cast<uint64_t>(dev.sm_count) * 8u;
+    {
+        const unsigned grid = static_cast<unsigned>(count < cap ? count : cap);
+        if (g_f32)
+            k_sqnorm_pass1<true><<<grid, kBlockThreads, 0, stream>>>(g, n, count, vec_ok, level_out);
+        else
+            k_sqnorm_pass1<false><<<grid, kBlockThreads, 0, stream>>>(g, n, count, vec_ok, level_out);
+        cudaError_t err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+    }
+    while (count > 1) {
+        const uint64_t next = blocks_of(count);
+        const double* level_in = level_out;
+        level_out = next == 1 ? out : level_out + count;
+        const unsigned grid = static_cast<unsigned>(next < cap ? next : cap);
+        k_tree_pass<<<grid, kBlockThreads, 0, stream>>>(level_in, count, next, level_out);
+        cudaError_t err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+        count = next;
+    }
+    return cudaSuccess;
+}
+
+cudaError_t launch_clip_scale(const double* sqnorm, float accum_scale, float max_norm, float* out,
+                              cudaStream_t stream) {
+    k_clip_scale<<<1, 1, 0, stream>>>(sqnorm, accum_scale, max_norm, out);
+    return cudaGetLastError();
+}
+
+}  // namespace sradamw
