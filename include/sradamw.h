@@ -83,6 +83,23 @@ sr_status sr_adamw_step(uint16_t* p, const void* g, sr_dtype g_dtype, uint16_t* 
                         const sr_adamw_hparams* hp, uint64_t seed, uint32_t step, uint32_t tensor_id,
                         uint64_t elem_offset, void* stream);
 
+/* The same iteration for state that lives in HOST memory (optimizer state kept off the device):
+ * the buffer is cut into chunks; each chunk is copied host->device into `staging`, stepped by the
+ * same kernel as sr_adamw_step (with elem_offset advanced, so the result equals the in-device
+ * step bit for bit) and its x, m, v copied back.  Two chunks are in flight on two streams (the
+ * caller's and one the library keeps per device) so uploads, kernels and downloads overlap.
+ * p, g, m, v: HOST pointers, page-locked for the copies to be asynchronous; they must stay valid
+ * until `stream` has been synchronised.  staging: DEVICE scratch, 256-byte aligned, at least
+ * sr_adamw_step_host_staging_bytes(g_dtype, chunk_elems) bytes, chunk_elems a non-zero multiple of
+ * 8; larger chunks amortise copy latency (2^24 elements is a reasonable choice).
+ * grad_scale_dev, if set, stays a device pointer.  The first call on a device creates the
+ * library's second stream and two events (kept until the process ends). */
+size_t sr_adamw_step_host_staging_bytes(sr_dtype g_dtype, uint64_t chunk_elems);
+sr_status sr_adamw_step_host(uint16_t* p_host, const void* g_host, sr_dtype g_dtype, uint16_t* m_host,
+                             uint16_t* v_host, uint64_t n, const sr_adamw_hparams* hp, uint64_t seed, uint32_t step,
+                             uint32_t tensor_id, uint64_t elem_offset, void* staging, size_t staging_bytes,
+                             uint64_t chunk_elems, void* stream);
+
 /* The same iteration over a list of tensors in one launch.  A plan owns device copies of the
  * pointer / size table and of the chunk table that maps thread blocks to (tensor, range).
  * The arrays passed to sr_mt_plan_create are HOST arrays of num_tensors entries holding device

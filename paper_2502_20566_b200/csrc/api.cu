@@ -1,0 +1,358 @@
+// C-ABI layer of libsradamw.so: argument checks, per-iteration scalars (Algorithm 1, the m-hat and
+// v-hat steps), Philox round keys, multi-tensor plans; all device work is in the kernel files.
+
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/sradamw.h"
+#include "launch.h"
+
+using namespace sradamw;
+
+namespace {
+
+thread_local int tl_last_cuda_error = 0;
+
+sr_status cuda_fail(cudaError_t e) {
+    tl_last_cuda_error = static_cast<int>(e);
+    return SR_ERR_CUDA;
+}
+
+constexpr int kMaxDevices = 64;
+struct DeviceSlot {
+    bool known = false;
+    DeviceInfo info{};
+};
+DeviceSlot g_devices[kMaxDevices];
+
+// Properties of the current device, queried once per device.  Racing first calls write the same values.
+sr_status current_device(DeviceInfo* out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return SR_ERR_UNSUPPORTED_DEVICE;
+    DeviceSlot& slot = g_devices[dev];
+    if (!slot.known) {
+        int sm = 0, major = 0;
+        e = cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return cuda_fail(e);
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) return cuda_fail(e);
+        slot.info.sm_count = sm;
+        slot.info.cc_major = major;
+        slot.known = true;
+    }
+    if (slot.info.cc_major != 10) return SR_ERR_UNSUPPORTED_DEVICE;
+    *out = slot.info;
+    return SR_OK;
+}
+
+PhiloxKeys make_keys(uint64_t seed, uint32_t step) {
+    PhiloxKeys K;
+    uint32_t k0 = static_cast<uint32_t>(seed), k1 = step;
+    for (int r = 0; r < 10; ++r) {
+        K.k0[r] = k0;
+        K.k1[r] = k1;
+        k0 += kPhiloxW0;
+        k1 += kPhiloxW1;
+    }
+    return K;
+}
+
+// beta^t by square-and-multiply in double (no libm: identical bits on every host)
+double power_u32(double base, uint32_t e) {
+    double r = 1.0;
+    while (e) {
+        if (e & 1u) r *= base;
+        base *= base;
+        e >>= 1;
+    }
+    return r;
+}
+
+bool finite_f(float x) { return std::isfinite(x); }
+
+sr_status make_scalars(const sr_adamw_hparams* hp, uint32_t step, StepScalars* S) {
+    if (hp == nullptr || hp->struct_size != sizeof(sr_adamw_hparams)) return SR_ERR_INVALID_ARG;
+    if (step == 0) return SR_ERR_INVALID_ARG;   // 1 - beta^0 = 0
+    if (!finite_f(hp->lr) || hp->lr < 0.0f) return SR_ERR_INVALID_ARG;
+    if (!(hp->beta1 >= 0.0f && hp->beta1 < 1.0f) || !(hp->beta2 >= 0.0f && hp->beta2 < 1.0f)) return SR_ERR_INVALID_ARG;
+    if (!finite_f(hp->eps) || hp->eps < 0.0f || !finite_f(hp->weight_decay)) return SR_ERR_INVALID_ARG;
+    if (hp->grad_scale_dev == nullptr && !finite_f(hp->grad_scale)) return SR_ERR_INVALID_ARG;
+    if (hp->flags & ~7u) return SR_ERR_INVALID_ARG;
+    const double b1 = hp->beta1, b2 = hp->beta2, lr = hp->lr, wd = hp->weight_decay;
+    const double bc1 = 1.0 - power_u32(b1, step);
+    const double bc2 = 1.0 - power_u32(b2, step);
+    S->beta1 = hp->beta1;
+    S->beta2 = hp->beta2;
+    S->omb1 = 1.0f - hp->beta1;
+    S->omb2 = 1.0f - hp->beta2;
+    S->step_size = static_cast<float>(lr / bc1);
+    S->rsqrt_bc2 = static_cast<float>(1.0 / std::sqrt(bc2));
+    S->eps = hp->eps;
+    S->lr_wd = static_cast<float>(lr * wd);
+    S->gscale = hp->grad_scale;
+    S->gscale_dev = hp->grad_scale_dev;
+    return SR_OK;
+}
+
+}  // namespace
+
+struct sr_mt_plan {
+    MtTensor* d_tensors = nullptr;
+    MtChunk* d_chunks = nullptr;
+    uint32_t num_tensors = 0;
+    uint32_t num_chunks = 0;
+    uint64_t total_elements = 0;
+    bool g_f32 = false;
+    int device = 0;
+};
+
+extern "C" {
+
+sr_status sr_downcast_f32_bf16(const float* src, uint16_t* dst, uint64_t n, uint64_t seed, uint32_t step,
+                               uint32_t tensor_id, uint64_t elem_offset, void* stream) {
+    if (n == 0) return SR_OK;
+    if (src == nullptr || dst == nullptr) return SR_ERR_INVALID_ARG;
+    DeviceInfo dev;
+    sr_status st = current_device(&dev);
+    if (st != SR_OK) return st;
+    const cudaError_t e = launch_downcast(src, dst, n, elem_offset, tensor_id, static_cast<uint32_t>(seed >> 32),
+                                          make_keys(seed, step), dev, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SR_OK : cuda_fail(e);
+}
+
+sr_status sr_adamw_step(uint16_t* p, const void* g, sr_dtype g_dtype, uint16_t* m, uint16_t* v, uint64_t n,
+                        const sr_adamw_hparams* hp, uint64_t seed, uint32_t step, uint32_t tensor_id,
+                        uint64_t elem_offset, void* stream) {
+    StepScalars S;
+    sr_status st = make_scalars(hp, step, &S);
+    if (st != SR_OK) return st;
+    if (g_dtype != SR_DT_BF16 && g_dtype != SR_DT_F32) return SR_ERR_INVALID_ARG;
+    if (n == 0) return SR_OK;
+    if (p == nullptr || g == nullptr || m == nullptr || v == nullptr) return SR_ERR_INVALID_ARG;
+    DeviceInfo dev;
+    st = current_device(&dev);
+    if (st != SR_OK) return st;
+    const cudaError_t e =
+        launch_adamw_flat(p, g, g_dtype == SR_DT_F32, m, v, n, elem_offset, tensor_id, static_cast<uint32_t>(seed >> 32),
+                          hp->flags, make_keys(seed, step), S, dev, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SR_OK : cuda_fail(e);
+}
+
+// ---- host-resident state -------------------------------------------------------------------
+namespace {
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t side = nullptr;     // second stream of the two-deep pipeline
+    cudaEvent_t fork = nullptr, join = nullptr;
+};
+HostPipe g_pipes[kMaxDevices];
+
+size_t slot_bytes(bool g_f32, uint64_t chunk) {
+    // p, m, v (2 bytes each) and g, each region rounded up to 256 bytes
+    auto up = [](uint64_t b) { return (b + 255u) & ~static_cast<uint64_t>(255u); };
+    return static_cast<size_t>(3 * up(chunk * 2) + up(chunk * (g_f32 ? 4 : 2)));
+}
+}  // namespace
+
+size_t sr_adamw_step_host_staging_bytes(sr_dtype g_dtype, uint64_t chunk_elems) {
+    return 2 * slot_bytes(g_dtype == SR_DT_F32, chunk_elems);
+}
+
+sr_status sr_adamw_step_host(uint16_t* p_host, const void* g_host, sr_dtype g_dtype, uint16_t* m_host,
+                             uint16_t* v_host, uint64_t n, const sr_adamw_hparams* hp, uint64_t seed, uint32_t step,
+                             uint32_t tensor_id, uint64_t elem_offset, void* staging, size_t staging_bytes,
+                             uint64_t chunk_elems, void* stream) {
+    StepScalars S;
+    sr_status st = make_scalars(hp, step, &S);
+    if (st != SR_OK) return st;
+    if (g_dtype != SR_DT_BF16 && g_dtype != SR_DT_F32) return SR_ERR_INVALID_ARG;
+    if (n == 0) return SR_OK;
+    if (p_host == nullptr || g_host == nullptr || m_host == nullptr || v_host == nullptr) return SR_ERR_INVALID_ARG;
+    if (chunk_elems == 0 || (chunk_elems & 7u)) return SR_ERR_INVALID_ARG;
+    const bool g_f32 = g_dtype == SR_DT_F32;
+    if (staging == nullptr || (reinterpret_cast<uintptr_t>(staging) & 255u) ||
+        staging_bytes < sr_adamw_step_host_staging_bytes(g_dtype, chunk_elems))
+        return SR_ERR_WORKSPACE;
+    DeviceInfo dev;
+    st = current_device(&dev);
+    if (st != SR_OK) return st;
+    int dev_id = 0;
+    cudaGetDevice(&dev_id);
+    HostPipe& pipe = g_pipes[dev_id];
+    cudaError_t e;
+    if (!pipe.ready) {
+        if ((e = cudaStreamCreateWithFlags(&pipe.side, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventCreateWithFlags(&pipe.fork, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventCreateWithFlags(&pipe.join, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        pipe.ready = true;
+    }
+    cudaStream_t streams[2] = {static_cast<cudaStream_t>(stream), pipe.side};
+    // the side stream starts after whatever the caller queued before this call
+    if ((e = cudaEventRecord(pipe.fork, streams[0])) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(pipe.side, pipe.fork, 0)) != cudaSuccess) return cuda_fail(e);
+
+    const PhiloxKeys K = make_keys(seed, step);
+    const uint32_t seed_hi = static_cast<uint32_t>(seed >> 32);
+    const size_t gsz = g_f32 ? 4 : 2;
+    const size_t slot = slot_bytes(g_f32, chunk_elems);
+    const size_t region = ((chunk_elems * 2 + 255u) / 256u) * 256u;
+    uint64_t k = 0;
+    for (uint64_t start = 0; start < n; start += chunk_elems, ++k) {
+        const uint64_t len = n - start < chunk_elems ? n - start : chunk_elems;
+        cudaStream_t s = streams[k & 1u];
+        char* base = static_cast<char*>(staging) + (k & 1u) * slot;
+        uint16_t* dp = reinterpret_cast<uint16_t*>(base);
+        uint16_t* dm = reinterpret_cast<uint16_t*>(base + region);
+        uint16_t* dv = reinterpret_cast<uint16_t*>(base + 2 * region);
+        void* dg = base + 3 * region;
+        const char* gh = static_cast<const char*>(g_host) + start * gsz;
+        if ((e = cudaMemcpyAsync(dp, p_host + start, len * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpyAsync(dg, gh, len * gsz, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpyAsync(dm, m_host + start, len * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpyAsync(dv, v_host + start, len * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+        e = launch_adamw_flat(dp, dg, g_f32, dm, dv, len, elem_offset + start, tensor_id, seed_hi, hp->flags, K, S, dev, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpyAsync(p_host + start, dp, len * 2, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpyAsync(m_host + start, dm, len * 2, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpyAsync(v_host + start, dv, len * 2, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+    }
+    // the caller's stream finishes only after the side stream has
+    if ((e = cudaEventRecord(pipe.join, pipe.side)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(streams[0], pipe.join, 0)) != cudaSuccess) return cuda_fail(e);
+    return SR_OK;
+}
+
+sr_status sr_mt_plan_create(sr_mt_plan** out, uint32_t num_tensors, uint16_t* const* p, const void* const* g,
+                            uint16_t* const* m, uint16_t* const* v, const uint64_t* numel, sr_dtype g_dtype,
+                            void* stream) {
+    if (out == nullptr) return SR_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (g_dtype != SR_DT_BF16 && g_dtype != SR_DT_F32) return SR_ERR_INVALID_ARG;
+    if (num_tensors != 0 && (p == nullptr || g == nullptr || m == nullptr || v == nullptr || numel == nullptr))
+        return SR_ERR_INVALID_ARG;
+    DeviceInfo dev;
+    sr_status st = current_device(&dev);
+    if (st != SR_OK) return st;
+
+    std::vector<MtTensor> tensors(num_tensors);
+    std::vector<MtChunk> chunks;
+    uint64_t total = 0;
+    for (uint32_t i = 0; i < num_tensors; ++i) {
+        if (numel[i] != 0 && (p[i] == nullptr || g[i] == nullptr || m[i] == nullptr || v[i] == nullptr))
+            return SR_ERR_INVALID_ARG;
+        const uint64_t nchunks = (numel[i] + kMtChunkElems - 1) / kMtChunkElems;
+        if (nchunks > 0xFFFFFFFFull || chunks.size() + nchunks > 0xFFFFFFFFull) return SR_ERR_INVALID_ARG;
+        const uintptr_t bits = reinterpret_cast<uintptr_t>(p[i]) | reinterpret_cast<uintptr_t>(g[i]) |
+                               reinterpret_cast<uintptr_t>(m[i]) | reinterpret_cast<uintptr_t>(v[i]);
+        tensors[i] = MtTensor{p[i], g[i], m[i], v[i], numel[i], (bits & 15u) == 0 ? 1u : 0u, 0u};
+        for (uint64_t c = 0; c < nchunks; ++c) chunks.push_back(MtChunk{i, static_cast<uint32_t>(c)});
+        total += numel[i];
+    }
+
+    sr_mt_plan* plan = new (std::nothrow) sr_mt_plan;
+    if (plan == nullptr) return SR_ERR_INVALID_ARG;
+    plan->num_tensors = num_tensors;
+    plan->num_chunks = static_cast<uint32_t>(chunks.size());
+    plan->total_elements = total;
+    plan->g_f32 = g_dtype == SR_DT_F32;
+    cudaGetDevice(&plan->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaSuccess;
+    if (!chunks.empty()) {
+        e = cudaMalloc(&plan->d_tensors, tensors.size() * sizeof(MtTensor));
+        if (e == cudaSuccess) e = cudaMalloc(&plan->d_chunks, chunks.size() * sizeof(MtChunk));
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(plan->d_tensors, tensors.data(), tensors.size() * sizeof(MtTensor), cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(plan->d_chunks, chunks.data(), chunks.size() * sizeof(MtChunk), cudaMemcpyHostToDevice, s);
+        // the host vectors die at return: wait for the copies (plan creation is not a hot call)
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    }
+    if (e != cudaSuccess) {
+        cudaFree(plan->d_tensors);
+        cudaFree(plan->d_chunks);
+        delete plan;
+        return cuda_fail(e);
+    }
+    *out = plan;
+    return SR_OK;
+}
+
+sr_status sr_adamw_multi_tensor(const sr_mt_plan* plan, const sr_adamw_hparams* hp, uint64_t seed, uint32_t step,
+                                uint32_t tensor_id_base, void* stream) {
+    if (plan == nullptr) return SR_ERR_INVALID_ARG;
+    StepScalars S;
+    sr_status st = make_scalars(hp, step, &S);
+    if (st != SR_OK) return st;
+    if (plan->num_chunks == 0) return SR_OK;
+    DeviceInfo dev;
+    st = current_device(&dev);
+    if (st != SR_OK) return st;
+    const cudaError_t e =
+        launch_adamw_mt(plan->d_tensors, plan->d_chunks, plan->num_chunks, plan->g_f32, tensor_id_base,
+                        static_cast<uint32_t>(seed >> 32), hp->flags, make_keys(seed, step), S, dev,
+                        static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SR_OK : cuda_fail(e);
+}
+
+sr_status sr_mt_plan_destroy(sr_mt_plan* plan) {
+    if (plan == nullptr) return SR_OK;
+    cudaError_t e1 = cudaFree(plan->d_tensors);
+    cudaError_t e2 = cudaFree(plan->d_chunks);
+    delete plan;
+    if (e1 != cudaSuccess) return cuda_fail(e1);
+    if (e2 != cudaSuccess) return cuda_fail(e2);
+    return SR_OK;
+}
+
+uint64_t sr_mt_plan_total_elements(const sr_mt_plan* plan) { return plan ? plan->total_elements : 0; }
+
+size_t grad_sqnorm_workspace_bytes(uint64_t n) { return static_cast<size_t>(sqnorm_scratch_doubles(n) * sizeof(double)); }
+
+sr_status grad_sqnorm(const void* g, sr_dtype g_dtype, uint64_t n, double* out_dev, void* workspace,
+                      size_t workspace_bytes, void* stream) {
+    if (out_dev == nullptr) return SR_ERR_INVALID_ARG;
+    if (g_dtype != SR_DT_BF16 && g_dtype != SR_DT_F32) return SR_ERR_INVALID_ARG;
+    if (n != 0 && g == nullptr) return SR_ERR_INVALID_ARG;
+    const size_t need = grad_sqnorm_workspace_bytes(n);
+    if (need != 0 && (workspace == nullptr || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 7u)))
+        return SR_ERR_WORKSPACE;
+    DeviceInfo dev;
+    sr_status st = current_device(&dev);
+    if (st != SR_OK) return st;
+    const cudaError_t e = launch_sqnorm(g, g_dtype == SR_DT_F32, n, out_dev, static_cast<double*>(workspace), dev,
+                                        static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SR_OK : cuda_fail(e);
+}
+
+sr_status sr_clip_scale(const double* sqnorm_dev, float accum_scale, float max_norm, float* gscale_out_dev,
+                        void* stream) {
+    if (sqnorm_dev == nullptr || gscale_out_dev == nullptr) return SR_ERR_INVALID_ARG;
+    if (!finite_f(accum_scale) || !finite_f(max_norm) || max_norm < 0.0f) return SR_ERR_INVALID_ARG;
+    DeviceInfo dev;
+    sr_status st = current_device(&dev);
+    if (st != SR_OK) return st;
+    const cudaError_t e = launch_clip_scale(sqnorm_dev, accum_scale, max_norm, gscale_out_dev, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SR_OK : cuda_fail(e);
+}
+
+const char* sr_status_string(sr_status s) {
+    switch (s) {
+        case SR_OK: return "ok";
+        case SR_ERR_INVALID_ARG: return "invalid argument";
+        case SR_ERR_UNSUPPORTED_DEVICE: return "unsupported device (compute capability 10.x required)";
+        case SR_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case SR_ERR_CUDA: return "CUDA runtime error (see sr_last_cuda_error)";
+    }
+    return "unknown status";
+}
+
+int sr_last_cuda_error(void) { return tl_last_cuda_error; }
+
+uint32_t sr_abi_version(void) { return SR_ABI_VERSION; }
+
+}  // extern "C"

@@ -1,0 +1,420 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle, bit for bit on
+the same seeded inputs.  Tolerance: 0 mismatching BF16 patterns, exact FP64 norm, exact FP32 scale."""
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+HP = dict(lr=6e-4, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
+
+
+@pytest.fixture(scope="module")
+def env():
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    import oracle
+    from paper_2502_20566_b200 import binding, synth
+    binding.lib()   # raises if the CUDA library is missing: no fallback
+    return oracle, binding, synth, torch.device("cuda", 0)
+
+
+def bits(t: torch.Tensor) -> np.ndarray:
+    return t.detach().view(torch.int16).cpu().numpy().view(np.uint16).copy()
+
+
+def host_g(g: torch.Tensor) -> np.ndarray:
+    return g.cpu().numpy().copy() if g.dtype == torch.float32 else bits(g)
+
+
+def mismatches(a: np.ndarray, b: np.ndarray) -> int:
+    return int(np.count_nonzero(a != b))
+
+
+def run_both(env, p, g, m, v, hp_kw, seed, step, tensor_id=0, elem_offset=0, gscale=1.0, flags=7):
+    """Step the CUDA path in place on (p, m, v) and the oracle on host copies; return mismatch counts."""
+    oracle, binding, _, _ = env
+    hp_o = oracle.hparams(**hp_kw, flags=flags)
+    pb, gb, mb, vb = bits(p), host_g(g), bits(m), bits(v)
+    oracle.adamw_step(pb, gb, mb, vb, hp_o, seed, step, tensor_id, elem_offset, gscale)
+    hp_g = binding.hparams(**hp_kw, grad_scale=gscale, flags=flags)
+    binding.sr_adamw_step(p, g, m, v, hp_g, seed, step, tensor_id, elem_offset)
+    torch.cuda.synchronize()
+    return mismatches(bits(p), pb), mismatches(bits(m), mb), mismatches(bits(v), vb)
+
+
+# ---------------------------------------------------------------------------------------------
+# flat step
+# ---------------------------------------------------------------------------------------------
+
+def test_flat_step_2pow20(env):
+    """One step on 2^20 elements, step 10, seed 1234, SR on x, m and v."""
+    _, _, synth, dev = env
+    p, g, m, v = synth.adamw_state(1 << 20, 1234, dev)
+    p0 = bits(p)
+    assert run_both(env, p, g, m, v, HP, seed=1234, step=10) == (0, 0, 0)
+    assert mismatches(bits(p), p0) > (1 << 19)          # the step really changed the parameters
+
+
+@pytest.mark.parametrize("n", [0, 1, 7, 8, 9, 255, 2047, 2048, 2049, 100003, (1 << 21) + 5])
+@pytest.mark.parametrize("g_dtype", [torch.bfloat16, torch.float32])
+def test_flat_step_ragged_sizes(env, n, g_dtype):
+    _, _, synth, dev = env
+    p, g, m, v = synth.adamw_state(n, 100 + n, dev, g_dtype=g_dtype)
+    assert run_both(env, p, g, m, v, HP, seed=77, step=3, tensor_id=4) == (0, 0, 0)
+
+
+@pytest.mark.parametrize("shift", [1, 3, 4])
+def test_flat_step_unaligned_buffers(env, shift):
+    """Buffers that start 2, 6 or 8 bytes past a 16-byte boundary take the element-wise path."""
+    _, _, synth, dev = env
+    n = 70001
+    p, g, m, v = (t[shift:] for t in synth.adamw_state(n + shift, 5, dev))
+    assert p.data_ptr() % 16 == (2 * shift) % 16
+    assert run_both(env, p, g, m, v, HP, seed=1, step=2) == (0, 0, 0)
+
+
+def test_flat_step_leaves_neighbouring_memory_alone(env):
+    _, binding, synth, dev = env
+    n, pad = 4099, 64
+    bufs = synth.adamw_state(n + 2 * pad, 6, dev)
+    before = [bits(t) for t in bufs]
+    inner = [t[pad:pad + n] for t in bufs]
+    binding.sr_adamw_step(*inner, binding.hparams(**HP), 9, 1)
+    torch.cuda.synchronize()
+    for t, b in zip(bufs, before):
+        a = bits(t)
+        assert np.array_equal(a[:pad], b[:pad]) and np.array_equal(a[pad + n:], b[pad + n:])
+    assert np.array_equal(bits(bufs[1]), before[1])     # the gradient is read-only
+
+
+@pytest.mark.parametrize("offset", [(1 << 32) - 1024, (1 << 32) - 1021, (1 << 33) + 8, 3 * 832300544, (1 << 40) + 5])
+def test_flat_step_index_offsets_cross_32_bits(env, offset):
+    _, _, synth, dev = env
+    p, g, m, v = synth.adamw_state(4096 + 3, 8, dev)
+    assert run_both(env, p, g, m, v, HP, seed=(0xABCD << 32) | 17, step=1000, tensor_id=0xFFFFFFFF, elem_offset=offset) == (0, 0, 0)
+
+
+@pytest.mark.parametrize("flags", range(8))
+@pytest.mark.parametrize("g_dtype", [torch.bfloat16, torch.float32])
+def test_flat_step_rounding_modes(env, flags, g_dtype):
+    """Every choice of stochastic / nearest rounding for x, m, v (flags 1 = the paper's update-only SR)."""
+    _, _, synth, dev = env
+    p, g, m, v = synth.adamw_state(50000 + 1, 12, dev, g_dtype=g_dtype)
+    assert run_both(env, p, g, m, v, HP, seed=3, step=10, gscale=0.125, flags=flags) == (0, 0, 0)
+
+
+def test_flat_step_special_values(env):
+    """NaN, infinities, zeros, subnormals and huge values in every input."""
+    _, _, synth, dev = env
+    n = 1 << 16
+    p, g, m, v = synth.adamw_state(n, 13, dev, g_dtype=torch.float32)
+    mix = synth.downcast_mix(4 * n, 99, dev)
+    sel = torch.rand(4 * n, device=dev, generator=torch.Generator(device=dev).manual_seed(1)) < 0.3
+    for k, t in enumerate((p, g, m, v)):
+        s, x = sel[k * n:(k + 1) * n], mix[k * n:(k + 1) * n]
+        if k == 3:
+            x = x.abs()
+        t[s] = x[s].to(t.dtype)
+    assert run_both(env, p, g, m, v, HP, seed=5, step=2) == (0, 0, 0)
+    assert run_both(env, p, g, m, v, HP, seed=5, step=3, flags=1) == (0, 0, 0)
+
+
+def test_flat_step_hyperparameter_corners(env):
+    _, _, synth, dev = env
+    for kw, step in [(dict(lr=0.0, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.0), 1),
+                     (dict(lr=1e-3, beta1=0.0, beta2=0.0, eps=0.0, weight_decay=0.0), 1),
+                     (dict(lr=7e-4, beta1=0.9, beta2=0.999, eps=1e-6, weight_decay=0.2), 4_000_000_000),
+                     (dict(lr=5.5e-4, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1), 1)]:
+        p, g, m, v = synth.adamw_state(30011, 14, dev)
+        assert run_both(env, p, g, m, v, kw, seed=6, step=step) == (0, 0, 0)
+
+
+def test_shards_equal_whole_and_runs_repeat(env):
+    """Shared random state: 8 shards stepped separately equal the whole buffer; a second run repeats
+    the first bit for bit; another seed does not."""
+    _, binding, synth, dev = env
+    n = 8 * 12500 + 4
+    whole = synth.adamw_state(n, 15, dev)
+    parts = [t.clone() for t in whole]
+    again = [t.clone() for t in whole]
+    other = [t.clone() for t in whole]
+    hp = binding.hparams(**HP)
+    binding.sr_adamw_step(*whole, hp, 21, 7, 3)
+    binding.sr_adamw_step(*again, hp, 21, 7, 3)
+    binding.sr_adamw_step(*other, hp, 22, 7, 3)
+    bounds = np.linspace(0, n, 9).astype(int)
+    for a, b in zip(bounds[:-1], bounds[1:]):
+        binding.sr_adamw_step(*[t[a:b] for t in parts], hp, 21, 7, 3, elem_offset=int(a))
+    torch.cuda.synchronize()
+    for w, q, r in zip(whole, parts, again):
+        assert torch.equal(w.view(torch.int16), q.view(torch.int16))
+        assert torch.equal(w.view(torch.int16), r.view(torch.int16))
+    assert not torch.equal(whole[0].view(torch.int16), other[0].view(torch.int16))
+
+
+def test_checkpoint_resume_is_exact(env):
+    """The random state is a function of (seed, step): 6 steps straight equal 3 steps, a copy out and
+    back, and 3 more."""
+    _, binding, synth, dev = env
+    n = 40000
+    a = synth.adamw_state(n, 16, dev)
+    b = [t.clone() for t in a]
+    hp = binding.hparams(**HP)
+    grads = [synth.state_chunk(synth.ROLE_G, 1000 + s, 0, n, dev) for s in range(1, 7)]
+    for s in range(1, 7):
+        binding.sr_adamw_step(a[0], grads[s - 1], a[2], a[3], hp, 4, s)
+    for s in range(1, 4):
+        binding.sr_adamw_step(b[0], grads[s - 1], b[2], b[3], hp, 4, s)
+    saved = [t.cpu() for t in b]
+    b = [t.to(dev) for t in saved]
+    for s in range(4, 7):
+        binding.sr_adamw_step(b[0], grads[s - 1], b[2], b[3], hp, 4, s)
+    torch.cuda.synchronize()
+    for k in (0, 2, 3):
+        assert torch.equal(a[k].view(torch.int16), b[k].view(torch.int16))
+
+
+# ---------------------------------------------------------------------------------------------
+# standalone stochastic-rounding cast
+# ---------------------------------------------------------------------------------------------
+
+def test_downcast_2pow26_mix(env):
+    oracle, binding, synth, dev = env
+    n = 1 << 26
+    src = synth.downcast_mix(n, 7, dev)
+    dst = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    binding.sr_downcast_f32_bf16(src, dst, seed=7)
+    torch.cuda.synchronize()
+    want = oracle.sr_downcast(src.cpu().numpy(), seed=7)
+    got = bits(dst)
+    assert mismatches(got, want) == 0
+    b = src.cpu().numpy().view(np.uint32)
+    nan = (b & 0x7FFFFFFF) > 0x7F800000
+    assert nan.any() and np.all(got[nan] == 0x7FC0)
+    rep = (b & 0xFFFF) == 0
+    assert np.array_equal(got[rep & ~nan], (b[rep & ~nan] >> 16).astype(np.uint16))
+
+
+@pytest.mark.parametrize("n,offset,shift", [(0, 0, 0), (1, 0, 0), (13, 5, 0), (4097, (1 << 32) - 9, 0), (5000, 16, 1), (5000, 3, 2)])
+def test_downcast_ragged_and_unaligned(env, n, offset, shift):
+    oracle, binding, synth, dev = env
+    src = synth.downcast_mix(n + shift, 8, dev)[shift:]
+    dst = torch.full((n + shift + 8,), -1.0, dtype=torch.bfloat16, device=dev)
+    out = dst[shift:shift + n]
+    binding.sr_downcast_f32_bf16(src, out, seed=(5 << 32) | 1, step=9, tensor_id=2, elem_offset=offset)
+    torch.cuda.synchronize()
+    want = oracle.sr_downcast(src.cpu().numpy().copy(), seed=(5 << 32) | 1, step=9, tensor_id=2, elem_offset=offset)
+    assert mismatches(bits(out), want) == 0
+    assert torch.all(dst[shift + n:] == -1.0) and torch.all(dst[:shift] == -1.0)
+
+
+def test_downcast_unbiased_over_4096_seeds(env):
+    """Mean over 4096 seeds of a 4096-element subset: within 6 sigma of x, sigma^2 = Delta^2 q(1-q)/4096
+    (quantisation-error lemma), and the up-counts follow Binomial(4096, q)."""
+    oracle, binding, synth, dev = env
+    k = 4096
+    src = synth.downcast_mix(1 << 16, 7, dev)
+    b_all = src.cpu().numpy().view(np.uint32)
+    ok = ((b_all & 0x7FFFFFFF) < 0x7F7F0000)                      # finite, below the last BF16 interval
+    idx = np.flatnonzero(ok)[:k]
+    sub = src[torch.from_numpy(idx).to(dev)].contiguous()
+    outs = torch.empty((k, k), dtype=torch.bfloat16, device=dev)
+    for s in range(k):
+        binding.sr_downcast_f32_bf16(sub, outs[s], seed=s)
+    torch.cuda.synchronize()
+    sub_h = sub.cpu().numpy()
+    for s in (0, 1, 4095):
+        assert np.array_equal(bits(outs[s]), oracle.sr_downcast(sub_h, seed=s))
+    x = sub_h.astype(np.float64)
+    b = sub_h.view(np.uint32)
+    lo = (b & 0xFFFF0000).view(np.float32).astype(np.float64)
+    hi = ((b & 0xFFFF0000) + 0x10000).astype(np.uint32).view(np.float32).astype(np.float64)
+    delta = hi - lo
+    q = (b & 0xFFFF) / 65536.0
+    vals = outs.float().double().cpu().numpy()
+    mean = vals.mean(axis=0)
+    sigma = np.abs(delta) * np.sqrt(q * (1 - q) / k)
+    assert np.all(np.abs(mean - x) <= 6 * sigma + 0.0)
+    ups = (bits(outs).reshape(k, k) != (b >> 16).astype(np.uint16)[None, :]).sum(axis=0)
+    var = k * q * (1 - q)
+    assert np.all(ups[var == 0] == 0)
+    wide = var >= 25.0                                     # normal approximation is good there
+    assert wide.sum() > k // 2
+    z = (ups - k * q)[wide] / np.sqrt(var[wide])
+    assert np.abs(z).max() < 6.0 and abs(z.mean()) < 0.1 and 0.9 < z.std() < 1.1
+
+
+# ---------------------------------------------------------------------------------------------
+# squared norm, clipping, and the clipped shard step
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n", [0, 1, 5, 8191, 8192, 8193, 100000, 8192 * 8192 + 12345])
+@pytest.mark.parametrize("g_dtype", [torch.float32, torch.bfloat16])
+def test_sqnorm_bit_exact(env, n, g_dtype):
+    oracle, binding, synth, dev = env
+    g = torch.empty(n, dtype=g_dtype, device=dev)
+    synth.fill_state(g, synth.ROLE_G, 17, outlier_fraction=0.01)
+    ws = torch.empty(max(1, binding.grad_sqnorm_workspace_bytes(n) // 8), dtype=torch.float64, device=dev)
+    out = torch.full((1,), -1.0, dtype=torch.float64, device=dev)
+    binding.grad_sqnorm(g, out, ws)
+    torch.cuda.synchronize()
+    assert float(out.item()).hex() == oracle.sqnorm(host_g(g)).hex()
+
+
+def test_sqnorm_unaligned(env):
+    oracle, binding, synth, dev = env
+    g = torch.empty(30000, dtype=torch.float32, device=dev)
+    synth.fill_state(g, synth.ROLE_G, 18)
+    g = g[1:]
+    ws = torch.empty(16, dtype=torch.float64, device=dev)
+    out = torch.zeros(1, dtype=torch.float64, device=dev)
+    binding.grad_sqnorm(g, out, ws)
+    assert float(out.item()).hex() == oracle.sqnorm(g.cpu().numpy().copy()).hex()
+
+
+def test_clip_scale_bit_exact(env):
+    oracle, binding, _, dev = env
+    out = torch.zeros(1, dtype=torch.float32, device=dev)
+    for S, acc, mx in [(4.0, 0.125, 1.0), (1e6, 0.125, 1.0), (0.0, 1.0, 1.0), (7.3e4, 0.25, 2.0), (832.3004, 0.125, 1.0),
+                       (float("inf"), 1.0, 1.0), (float("nan"), 1.0, 1.0)]:
+        binding.sr_clip_scale(torch.tensor([S], dtype=torch.float64, device=dev), acc, mx, out)
+        got, want = float(out.item()), oracle.clip_scale(S, acc, mx)
+        assert (np.isnan(got) and np.isnan(want)) or np.float32(got).tobytes() == np.float32(want).tobytes()
+
+
+def _clipped_shard(env, n, rank):
+    oracle, binding, synth, dev = env
+    p, g, m, v = synth.adamw_state(n, 19, dev, g_dtype=torch.float32, outlier_fraction=0.01)
+    ws = torch.empty(max(1, binding.grad_sqnorm_workspace_bytes(n) // 8), dtype=torch.float64, device=dev)
+    S = torch.zeros(1, dtype=torch.float64, device=dev)
+    gs = torch.zeros(1, dtype=torch.float32, device=dev)
+    pb, gb, mb, vb = bits(p), host_g(g), bits(m), bits(v)
+    binding.grad_sqnorm(g, S, ws)
+    binding.sr_clip_scale(S, 0.125, 1.0, gs)
+    binding.sr_adamw_step(p, g, m, v, binding.hparams(**HP, grad_scale_dev=gs), 1234, 1000, 0, rank * n)
+    torch.cuda.synchronize()
+    S_o = oracle.sqnorm(gb)
+    gs_o = oracle.clip_scale(S_o, 0.125, 1.0)
+    assert float(S.item()).hex() == S_o.hex()
+    assert np.float32(gs.item()).tobytes() == np.float32(gs_o).tobytes()
+    assert gs_o < 0.125                                       # the outliers make clipping active
+    oracle.adamw_step(pb, gb, mb, vb, oracle.hparams(**HP), 1234, 1000, 0, rank * n, gs_o)
+    return mismatches(bits(p), pb), mismatches(bits(m), mb), mismatches(bits(v), vb)
+
+
+def test_clipped_shard_small(env):
+    assert _clipped_shard(env, (1 << 22) + 13, 3) == (0, 0, 0)
+
+
+def test_clipped_shard_full_size(env):
+    """A 1/8 shard of the 6.7B buffer (832 300 544 elements, FP32 gradients with 1% outliers), rank 3."""
+    _, _, synth, _ = env
+    n = synth.gpt_flat_numel() // 8
+    assert n == 832_300_544
+    assert _clipped_shard(env, n, 3) == (0, 0, 0)
+
+
+# ---------------------------------------------------------------------------------------------
+# tensor list
+# ---------------------------------------------------------------------------------------------
+
+def _run_list(env, specs, steps, seed=1234, grad_seed=4321, shift=0):
+    oracle, binding, synth, dev = env
+    P = [synth.init_param(s, seed, i, dev) for i, s in enumerate(specs)]
+    if shift:
+        P = [torch.cat([t.new_zeros(shift), t])[shift:] if i % 3 == 1 else t for i, t in enumerate(P)]
+    M = [torch.zeros_like(t) for t in P]
+    V = [torch.zeros_like(t) for t in P]
+    G = [torch.zeros_like(t) for t in P]
+    plan = binding.sr_mt_plan_create(P, G, M, V)
+    assert plan.total_elements == sum(s.numel for s in specs)
+    hp_g, hp_o = binding.hparams(**HP), oracle.hparams(**HP)
+    host = [[bits(t) for t in P], None, [bits(t) for t in M], [bits(t) for t in V]]
+    total = [0, 0, 0]
+    for step in range(1, steps + 1):
+        for i, s in enumerate(specs):
+            G[i].copy_(synth.fresh_grad(s, grad_seed, step, i, dev))
+        binding.sr_adamw_multi_tensor(plan, hp_g, seed, step)
+        torch.cuda.synchronize()
+        for i in range(len(specs)):
+            oracle.adamw_step(host[0][i], bits(G[i]), host[2][i], host[3][i], hp_o, seed, step, tensor_id=i)
+        for k, dev_list in ((0, P), (2, M), (3, V)):
+            for i in range(len(specs)):
+                total[0 if k == 0 else k - 1] += mismatches(bits(dev_list[i]), host[k][i])
+        assert total == [0, 0, 0], f"step {step}"
+    plan.destroy()
+    return total
+
+
+def test_multi_tensor_small_list_with_odd_shapes(env):
+    _, _, synth, _ = env
+    T = synth.TensorSpec
+    specs = [T("a", (1,), "normal"), T("b", (7,), "ones"), T("c", (16384,), "normal"), T("d", (16385,), "normal"),
+             T("e", (3, 1111), "normal"), T("f", (0,), "zeros"), T("g", (100000,), "normal"), T("h", (8,), "zeros")]
+    _run_list(env, specs, steps=3)
+    _run_list(env, specs, steps=2, shift=1)      # every third tensor starts 2 bytes off alignment
+
+
+def test_multi_tensor_gpt2_350m_ten_steps(env):
+    """GPT-2 350M parameter list (292 tensors, 354 823 168 elements), 10 iterations with fresh
+    gradients, zero mismatches after every iteration."""
+    _, _, synth, _ = env
+    specs = synth.gpt2_param_list()
+    assert len(specs) == 292 and sum(s.numel for s in specs) == 354_823_168
+    _run_list(env, specs, steps=10)
+
+
+# ---------------------------------------------------------------------------------------------
+# full-size flat buffer: sampled chunks
+# ---------------------------------------------------------------------------------------------
+
+def test_flat_6p7b_sampled_chunks(env):
+    """The 6 658 404 352-element buffer stepped once (step 1000) in the launch shape the benchmark
+    times; chunks sampled across the buffer (first, around index 2^32, last ragged one) are drawn
+    again from the seeded generator, stepped by the oracle and compared bit for bit; untouched
+    guard elements past the end stay intact."""
+    oracle, binding, synth, dev = env
+    n = synth.gpt_flat_numel()
+    assert n == 6_658_404_352
+    guard = 64
+    bufs = [torch.empty(n + guard, dtype=torch.bfloat16, device=dev) for _ in range(4)]
+    roles = (synth.ROLE_P, synth.ROLE_G, synth.ROLE_M, synth.ROLE_V)
+    for t, role in zip(bufs, roles):
+        synth.fill_state(t[:n], role, 1234)
+        t[n:] = 1.5
+    p, g, m, v = (t[:n] for t in bufs)
+    binding.sr_adamw_step(p, g, m, v, binding.hparams(**HP), 1234, 1000)
+    torch.cuda.synchronize()
+    for t in bufs:
+        assert torch.all(t[n:] == 1.5)
+    nchunks = (n + synth.CHUNK - 1) // synth.CHUNK
+    hp_o = oracle.hparams(**HP)
+    for c in sorted({0, 1, 31, 63, 64, 65, nchunks // 2 + 7, nchunks - 2, nchunks - 1}):
+        start = c * synth.CHUNK
+        length = min(synth.CHUNK, n - start)
+        pre = [bits(synth.state_chunk(role, 1234, c, length, dev)) for role in roles]
+        oracle.adamw_step(*pre, hp_o, 1234, 1000, 0, start)
+        for k, t in ((0, p), (2, m), (3, v)):
+            assert mismatches(bits(t[start:start + length]), pre[k]) == 0, (c, k)
+
+
+# ---------------------------------------------------------------------------------------------
+# host-resident state
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("g_dtype", [torch.bfloat16, torch.float32])
+def test_host_resident_step_equals_oracle(env, g_dtype):
+    """State in pinned host memory, staged through the device in chunks: same bits as the oracle
+    (and therefore as the in-device step), including a ragged last chunk and a non-zero offset."""
+    oracle, binding, synth, dev = env
+    n, chunk = 5 * 65536 + 1237, 65536
+    p, g, m, v = (t.pin_memory() for t in synth.adamw_state(n, 23, "cpu", g_dtype=g_dtype))
+    pb, mb, vb = (synth.bits16(t).copy() for t in (p, m, v))
+    gb = g.numpy().copy() if g_dtype == torch.float32 else synth.bits16(g).copy()
+    oracle.adamw_step(pb, gb, mb, vb, oracle.hparams(**HP), 31, 5, 2, 1000)
+    staging = torch.empty(binding.sr_adamw_step_host_staging_bytes(g_dtype, chunk), dtype=torch.uint8, device=dev)
+    binding.sr_adamw_step_host(p, g, m, v, binding.hparams(**HP), 31, 5, staging, chunk, tensor_id=2, elem_offset=1000)
+    torch.cuda.synchronize()
+    assert mismatches(synth.bits16(p), pb) == 0 and mismatches(synth.bits16(m), mb) == 0 and mismatches(synth.bits16(v), vb) == 0
