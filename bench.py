@@ -1,0 +1,335 @@
+#!/usr/bin/env python
+"""Benchmark of the fused SR-AdamW step (Algorithm 1) on the 6.7B-parameter flat buffer.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one sr_adamw_step call over the whole buffer (6 658 404 352 BF16 elements of x, g, m, v
+resident in HBM; 14 algorithmic bytes per element).  Prints ONE JSON line: parameters updated per
+second over all ranks, the HBM roofline of the kernel, an end-to-end figure with host-resident
+state, and the CPU oracle timed on the same box.  With N > 1 (torchrun) every rank steps its own
+full replica, as the data-parallel replicas of Algorithm 1 do; there is no collective in the path.
+`--impl reference` times the CPU oracle (slow by construction) on a bounded sample per step.
+"""
+
+from __future__ import annotations
+
+import argparse
+import datetime as _dt
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "SR-AdamW params/sec and achieved HBM GB/s (% of B200 peak) at 6.7B, 1 GPU"
+HP = dict(lr=6e-4, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
+SEED = 1234
+FIRST_STEP = 1000
+BYTES_PER_ELEMENT = 14          # read x, g, m, v (4 x 2 B) + write x, m, v (3 x 2 B)
+FALLBACK_HBM_GBS = 6650.0       # used only when MEASURED_PEAKS.json is absent
+# dram__bytes_read.sum + dram__bytes_write.sum per element from the committed ncu capture of the
+# current kernel (profiles/); None until a capture of this kernel version exists
+NCU_TRAFFIC_BYTES_PER_ELEMENT = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--elements", type=int, default=0, help="override the buffer length (profiling on a small case)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-elements", type=int, default=1 << 29)
+    return ap.parse_args()
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------------
+
+_SMI_FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+               "clocks_event_reasons.sw_power_cap")
+
+
+class ClockSampler:
+    """nvidia-smi polled in the background; samples are cut to the timed region afterwards."""
+
+    def __init__(self, torch, device_index: int):
+        self.proc = None
+        self.path = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            f = tempfile.NamedTemporaryFile(prefix="clocks_", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", uuid, f"--query-gpu={_SMI_FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=f, stderr=subprocess.DEVNULL)
+            f.close()
+        except Exception:
+            self.proc = None
+
+    def stop(self, t0: _dt.datetime, t1: _dt.datetime) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = []
+        try:
+            with open(self.path) as f:
+                for line in f:
+                    parts = [x.strip() for x in line.split(",")]
+                    if len(parts) != 8:
+                        continue
+                    try:
+                        ts = _dt.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f")
+                        rows.append((ts, float(parts[1]), float(parts[2]), float(parts[3]), parts[4:8]))
+                    except ValueError:
+                        continue
+            os.unlink(self.path)
+        except OSError:
+            return out
+        inside = [r for r in rows if t0 <= r[0] <= t1] or rows[-3:]
+        if not inside:
+            return out
+        out["samples"] = len(inside)
+        out["sm_mhz"] = statistics.median(r[1] for r in inside)
+        out["sm_max_mhz"] = max(r[2] for r in inside)
+        out["power_w_max"] = max(r[3] for r in inside)
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        out["reasons"] = [n for i, n in enumerate(names) if any(r[4][i].lower().startswith("active") for r in inside)]
+        return out
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ---------------------------------------------------------------------------------------------
+
+def _oracle_sample(synth, torch, elements: int):
+    import numpy as np
+    p, g, m, v = synth.adamw_state(elements, SEED, "cpu")
+    return [synth.bits16(t).copy() for t in (p, g, m, v)]
+
+
+def time_oracle(sample_elements: int, budget_s: float = 12.0):
+    """Oracle timed as it stands (OpenMP over elements) on `sample_elements` of the workload."""
+    import torch
+    import oracle
+    from paper_2502_20566_b200 import synth
+    arrs = _oracle_sample(synth, torch, sample_elements)
+    hp = oracle.hparams(**HP)
+    oracle.adamw_step(*[a[:1 << 16].copy() for a in arrs], hp, SEED, FIRST_STEP)      # load + warm
+    times = []
+    t_all = time.perf_counter()
+    rep = 0
+    while rep < 8 and (rep < 1 or time.perf_counter() - t_all < budget_s):
+        t0 = time.perf_counter()
+        oracle.adamw_step(*arrs, hp, SEED, FIRST_STEP + rep)
+        times.append(time.perf_counter() - t0)
+        rep += 1
+    mean = sum(times) / len(times)
+    return {"value": sample_elements / mean, "unit": "params/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{len(times)} x sr_adamw_step on the first {sample_elements} elements of the workload "
+                      f"(same distributions, step {FIRST_STEP}+), OpenMP threads = cores"}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, one bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    import oracle
+    from paper_2502_20566_b200 import synth
+    sample = 1 << 27
+    arrs = _oracle_sample(synth, torch, sample)
+    hp = oracle.hparams(**HP)
+    for w in range(args.warmup):
+        oracle.adamw_step(*arrs, hp, SEED, FIRST_STEP + w)
+    t0 = time.perf_counter()
+    for k in range(args.steps):
+        oracle.adamw_step(*arrs, hp, SEED, FIRST_STEP + args.warmup + k)
+    dt = time.perf_counter() - t0
+    value = sample * args.steps / dt
+    n = args.elements or synth.gpt_flat_numel()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "params/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"6.7B flat buffer ({n} elements, bf16 x/g/m/v, step {FIRST_STEP}); each step runs "
+                               f"the CPU oracle on a {sample}-element sample of it"},
+        "cpu_baseline": {"value": value, "unit": "params/s", "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": f"{sample} elements per step"},
+        "e2e": {"value": value, "unit": "params/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+# CUDA arm
+# ---------------------------------------------------------------------------------------------
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy kernel)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+def run_ours(args):
+    import torch
+    from paper_2502_20566_b200 import binding, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    binding.lib()
+
+    n = args.elements or synth.gpt_flat_numel()
+    bufs = [torch.empty(n, dtype=torch.bfloat16, device=dev) for _ in range(4)]
+    for t, role in zip(bufs, (synth.ROLE_P, synth.ROLE_G, synth.ROLE_M, synth.ROLE_V)):
+        synth.fill_state(t, role, SEED)
+    p, g, m, v = bufs
+    hp = binding.hparams(**HP)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for w in range(args.warmup):
+        binding.sr_adamw_step(p, g, m, v, hp, SEED, FIRST_STEP + w)
+    sampler = ClockSampler(torch, local) if rank == 0 else None
+    if sampler is not None:
+        time.sleep(0.3)          # let the poller start
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    t_begin = _dt.datetime.now()
+    for k in range(args.steps):
+        ev[k][0].record(stream)
+        binding.sr_adamw_step(p, g, m, v, hp, SEED, FIRST_STEP + args.warmup + k)
+        ev[k][1].record(stream)
+    barrier()
+    t_end = _dt.datetime.now()
+    total_ms = ev[0][0].elapsed_time(ev[-1][1])
+    launch_ms = [a.elapsed_time(b) for a, b in ev]
+    clocks = sampler.stop(t_begin, t_end) if sampler is not None else None
+    if dist is not None:
+        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+
+    # end to end: state in pinned host memory, staged through the device by sr_adamw_step_host
+    e2e = None
+    if not args.no_e2e:
+        e = min(args.e2e_elements, n)
+        chunk = 1 << 24
+        host = [t[:e].cpu().pin_memory() for t in bufs]
+        staging = torch.empty(binding.sr_adamw_step_host_staging_bytes(torch.bfloat16, chunk), dtype=torch.uint8, device=dev)
+        reps = max(1, min(args.steps, 5))
+        binding.sr_adamw_step_host(host[0], host[1], host[2], host[3], hp, SEED, 1, staging, chunk)
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for k in range(reps):
+            binding.sr_adamw_step_host(host[0], host[1], host[2], host[3], hp, SEED, 2 + k, staging, chunk)
+        b.record(stream)
+        barrier()
+        e2e_ms = a.elapsed_time(b)
+        checksum = int(host[0][:1024].view(torch.int16).sum())      # the result is read on the host
+        if dist is not None:
+            tt = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e2e_ms = float(tt.item())
+        e2e = {"value": world * e * reps / (e2e_ms * 1e-3), "unit": "params/s", "h2d_bytes_per_step": 8 * e,
+               "d2h_bytes_per_step": 6 * e, "steps": reps, "ms_per_step": e2e_ms / reps,
+               "sample": f"sr_adamw_step_host on {e} elements per rank held in pinned host memory "
+                         f"(x, g, m, v up, x, m, v down every step; {chunk}-element chunks, two streams)",
+               "host_checksum": checksum}
+        del host, staging
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = hbm_peak()
+    avg_launch_ms = sum(launch_ms) / len(launch_ms)
+    achieved = BYTES_PER_ELEMENT * n / (avg_launch_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC,
+        "value": world * n * args.steps / (total_ms * 1e-3),
+        "unit": "params/s",
+        "n_gpus": world,
+        "steps": args.steps,
+        "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps,
+        "higher_is_better": True,
+        "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": "f32",
+        "data": "synthetic",
+        "config": {
+            "workload": f"6.7B flat buffer: {n} elements, bf16 x/g/m/v resident in HBM ({8 * n / 1e9:.1f} GB), "
+                        f"one sr_adamw_step per step at step {FIRST_STEP}+, SR on x, m, v",
+            "elements": n, "bytes_per_element": BYTES_PER_ELEMENT,
+            "l2": "buffers are far larger than the 126 MB L2; no flush between iterations",
+            "replicas": world,
+        },
+        "hbm_gbs": achieved,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": (NCU_TRAFFIC_BYTES_PER_ELEMENT * n if NCU_TRAFFIC_BYTES_PER_ELEMENT else None),
+                     "peak_source": peak_src, "kernel": "k_sr_adamw_flat", "launch_ms_avg": avg_launch_ms,
+                     "launch_ms_min": min(launch_ms), "launch_ms_median": statistics.median(launch_ms),
+                     "algorithmic_bytes_per_launch": BYTES_PER_ELEMENT * n},
+        "gpu_launches": args.steps,
+        "clocks": clocks,
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if world == 1 and not args.no_cpu_baseline:
+        del bufs, p, g, m, v
+        torch.cuda.empty_cache()
+        line["cpu_baseline"] = time_oracle(1 << 28)
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
