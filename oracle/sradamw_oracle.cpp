@@ -93,20 +93,24 @@ void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]
 
 // ---- the optimizer's random state r^(opt)_t ------------------------------------------------
 // Algorithm 1 needs a random state that is the same on every replica at iteration t.  Here the
-// state is a pure function of (seed, step, tensor_id, global element index):
+// state is a pure function of (seed, step, tensor_id, global element index).  One Philox call
+// yields 128 bits while one element needs 3 x 16, so two neighbouring elements share a call:
+//   pair    = index >> 1
 //   key     = (seed[31:0], step)
-//   counter = (index[31:0], index[63:32], tensor_id, seed[63:32])
-// and the four output words serve, in order, the roundings of x, m and v (the fourth is unused).
-// Each rounding consumes the top 16 bits of its word.
+//   counter = (pair[31:0], pair[63:32], tensor_id, seed[63:32])
+// Output words 0, 1, 2 serve the roundings of x, m and v (word 3 is unused); in each word the
+// element with even index takes the low 16 bits and the element with odd index the high 16 bits.
 struct Noise3 { uint32_t rp, rm, rv; };
 
 Noise3 noise_for(uint64_t seed, uint32_t step, uint32_t tensor_id, uint64_t index) {
-    const uint32_t ctr[4] = {static_cast<uint32_t>(index), static_cast<uint32_t>(index >> 32),
+    const uint64_t pair = index >> 1;
+    const uint32_t ctr[4] = {static_cast<uint32_t>(pair), static_cast<uint32_t>(pair >> 32),
                              tensor_id, static_cast<uint32_t>(seed >> 32)};
     const uint32_t key[2] = {static_cast<uint32_t>(seed), step};
     uint32_t w[4];
     philox4x32_10(ctr, key, w);
-    return Noise3{w[0] >> 16, w[1] >> 16, w[2] >> 16};
+    if (index & 1u) return Noise3{w[0] >> 16, w[1] >> 16, w[2] >> 16};
+    return Noise3{w[0] & 0xFFFFu, w[1] & 0xFFFFu, w[2] & 0xFFFFu};
 }
 
 // ---- Eq. 2 by dithering --------------------------------------------------------------------

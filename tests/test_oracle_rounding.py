@@ -49,12 +49,28 @@ def test_philox_is_sensitive_to_every_input_word():
         assert oracle.philox4x32_10([1, 2, 3, 4], k) != base
 
 
+def _half(word, index):
+    return (word >> 16) if index & 1 else (word & 0xFFFF)
+
+
 def test_noise_layout_key_counter_and_words():
-    """key = (seed low, step); counter = (index low, index high, tensor_id, seed high); the noise
-    for x, m, v is the top half of words 0, 1, 2."""
-    seed, step, tid, idx = 0x1234_5678_9ABC_DEF0, 77, 9, (5 << 32) | 0xFFFF_FFF3
-    w = oracle.philox4x32_10([idx & 0xFFFFFFFF, idx >> 32, tid, seed >> 32], [seed & 0xFFFFFFFF, step])
-    assert oracle.noise(seed, step, tid, idx) == (w[0] >> 16, w[1] >> 16, w[2] >> 16)
+    """key = (seed low, step); counter = (pair low, pair high, tensor_id, seed high) with
+    pair = index >> 1; words 0, 1, 2 serve x, m, v; even index -> low half, odd index -> high half."""
+    seed, step, tid = 0x1234_5678_9ABC_DEF0, 77, 9
+    for idx in ((5 << 32) | 0xFFFF_FFF3, (5 << 32) | 0xFFFF_FFF2, (1 << 33) - 1, 1 << 33, 0, 1):
+        pair = idx >> 1
+        w = oracle.philox4x32_10([pair & 0xFFFFFFFF, pair >> 32, tid, seed >> 32], [seed & 0xFFFFFFFF, step])
+        assert oracle.noise(seed, step, tid, idx) == tuple(_half(w[k], idx) for k in range(3))
+
+
+def test_two_elements_of_a_pair_use_disjoint_bits():
+    """The 96 bits a pair consumes are six different 16-bit fields of one call: together the two
+    elements reproduce words 0..2 exactly."""
+    for idx in (0, 2, 10**12):
+        a, b = oracle.noise(3, 4, 5, idx), oracle.noise(3, 4, 5, idx + 1)
+        pair = idx >> 1
+        w = oracle.philox4x32_10([pair & 0xFFFFFFFF, pair >> 32, 5, 0], [3, 4])
+        assert tuple(a[k] | (b[k] << 16) for k in range(3)) == w[:3]
 
 
 def test_noise_streams_differ():
@@ -63,7 +79,7 @@ def test_noise_streams_differ():
     assert [oracle.noise(1, 2, 0, i) for i in range(64)] != ref            # iteration
     assert [oracle.noise(1, 1, 1, i) for i in range(64)] != ref            # tensor
     assert [oracle.noise(1 | (1 << 32), 1, 0, i) for i in range(64)] != ref  # high half of the seed
-    assert [oracle.noise(1, 1, 0, i + (1 << 32)) for i in range(64)] != ref  # high half of the index
+    assert [oracle.noise(1, 1, 0, i + (1 << 33)) for i in range(64)] != ref  # high half of the pair index
     assert len(set(ref)) == 64
 
 
