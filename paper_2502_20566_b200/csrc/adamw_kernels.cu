@@ -20,29 +20,29 @@ __device__ __forceinline__ void st16(void* base, uint64_t vec, uint4 val) {
     __stcs(reinterpret_cast<uint4*>(base) + vec, val);
 }
 
-// Counter words of element `e` (0..7) of a vector whose first global index is (hi:lo).
-// CARRY = false is valid when lo is a multiple of 8 (lo + e cannot wrap).
-template <bool CARRY>
-__device__ __forceinline__ void counter_of(uint32_t lo, uint32_t hi, uint32_t e, uint32_t& c0, uint32_t& c1) {
-    c0 = lo + e;
-    c1 = CARRY ? hi + (c0 < lo ? 1u : 0u) : hi;
-}
-
-// One pair of elements (the two halves of one 32-bit word of each BF16 array).
-template <uint32_t FLAGS, bool CARRY>
+// One pair of elements (the two halves of one 32-bit word of each BF16 array) whose first global
+// index is idx0 + e.  PAIRED = true needs idx0 + e even (then both share one Philox call and, idx0
+// being a multiple of 8, the pair counter low word cannot wrap inside a vector); PAIRED = false
+// draws each element's noise on its own and is valid for any index.
+template <uint32_t FLAGS, bool PAIRED>
 __device__ __forceinline__ void step_pair(uint32_t pw, float g_even, float g_odd, uint32_t mw, uint32_t vw,
-                                          uint32_t lo, uint32_t hi, uint32_t e, uint32_t c2, uint32_t c3, float gscale,
+                                          uint64_t idx0, uint32_t e, uint32_t c2, uint32_t c3, float gscale,
                                           const PhiloxKeys& K, const StepScalars& S, uint32_t& po, uint32_t& mo,
                                           uint32_t& vo) {
     const ElementOut r0 = adamw_element(bf16_lo(pw), g_even, bf16_lo(mw), bf16_lo(vw), gscale, S);
     const ElementOut r1 = adamw_element(bf16_hi(pw), g_odd, bf16_hi(mw), bf16_hi(vw), gscale, S);
     uint32_t a0 = 0, a1 = 0, a2 = 0, b0 = 0, b1 = 0, b2 = 0;
     if (FLAGS != 0) {
-        uint32_t c0, c1;
-        counter_of<CARRY>(lo, hi, e, c0, c1);
-        philox4x32_10(c0, c1, c2, c3, K, a0, a1, a2);
-        counter_of<CARRY>(lo, hi, e + 1, c0, c1);
-        philox4x32_10(c0, c1, c2, c3, K, b0, b1, b2);
+        if (PAIRED) {
+            uint32_t w0, w1, w2;
+            philox4x32_10(static_cast<uint32_t>(idx0 >> 1) + (e >> 1), static_cast<uint32_t>(idx0 >> 33), c2, c3, K,
+                          w0, w1, w2);
+            a0 = noise_even(w0); a1 = noise_even(w1); a2 = noise_even(w2);
+            b0 = noise_odd(w0); b1 = noise_odd(w1); b2 = noise_odd(w2);
+        } else {
+            noise_of_element(idx0 + e, c2, c3, K, a0, a1, a2);
+            noise_of_element(idx0 + e + 1, c2, c3, K, b0, b1, b2);
+        }
     }
     uint32_t sp0, sm0, sv0, sp1, sm1, sv1;
     round_element<FLAGS>(r0, a0, a1, a2, sp0, sm0, sv0);
@@ -53,7 +53,7 @@ __device__ __forceinline__ void step_pair(uint32_t pw, float g_even, float g_odd
 }
 
 // Eight consecutive elements starting at global index idx0; element arrays addressed by `vec`.
-template <bool G32, uint32_t FLAGS, bool CARRY>
+template <bool G32, uint32_t FLAGS, bool PAIRED>
 __device__ __forceinline__ void step_vec8(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t vec,
                                           uint64_t idx0, uint32_t c2, uint32_t c3, float gscale, const PhiloxKeys& K,
                                           const StepScalars& S) {
@@ -75,12 +75,11 @@ __device__ __forceinline__ void step_vec8(uint16_t* p, const void* g, uint16_t* 
         ge[4] = bf16_lo(gv.z); ge[5] = bf16_hi(gv.z);
         ge[6] = bf16_lo(gv.w); ge[7] = bf16_hi(gv.w);
     }
-    const uint32_t lo = static_cast<uint32_t>(idx0), hi = static_cast<uint32_t>(idx0 >> 32);
     uint4 po, mo, vo;
-    step_pair<FLAGS, CARRY>(pv.x, ge[0], ge[1], mv.x, vv.x, lo, hi, 0, c2, c3, gscale, K, S, po.x, mo.x, vo.x);
-    step_pair<FLAGS, CARRY>(pv.y, ge[2], ge[3], mv.y, vv.y, lo, hi, 2, c2, c3, gscale, K, S, po.y, mo.y, vo.y);
-    step_pair<FLAGS, CARRY>(pv.z, ge[4], ge[5], mv.z, vv.z, lo, hi, 4, c2, c3, gscale, K, S, po.z, mo.z, vo.z);
-    step_pair<FLAGS, CARRY>(pv.w, ge[6], ge[7], mv.w, vv.w, lo, hi, 6, c2, c3, gscale, K, S, po.w, mo.w, vo.w);
+    step_pair<FLAGS, PAIRED>(pv.x, ge[0], ge[1], mv.x, vv.x, idx0, 0, c2, c3, gscale, K, S, po.x, mo.x, vo.x);
+    step_pair<FLAGS, PAIRED>(pv.y, ge[2], ge[3], mv.y, vv.y, idx0, 2, c2, c3, gscale, K, S, po.y, mo.y, vo.y);
+    step_pair<FLAGS, PAIRED>(pv.z, ge[4], ge[5], mv.z, vv.z, idx0, 4, c2, c3, gscale, K, S, po.z, mo.z, vo.z);
+    step_pair<FLAGS, PAIRED>(pv.w, ge[6], ge[7], mv.w, vv.w, idx0, 6, c2, c3, gscale, K, S, po.w, mo.w, vo.w);
     st16(p, vec, po);
     st16(m, vec, mo);
     st16(v, vec, vo);
@@ -98,8 +97,7 @@ __device__ __forceinline__ void step_scalar(uint16_t* p, const void* g, uint16_t
                          : __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t*>(g)[i]) << 16);
     const ElementOut r = adamw_element(x, gi, mi, vi, gscale, S);
     uint32_t w0 = 0, w1 = 0, w2 = 0;
-    if (FLAGS != 0)
-        philox4x32_10(static_cast<uint32_t>(idx), static_cast<uint32_t>(idx >> 32), c2, c3, K, w0, w1, w2);
+    if (FLAGS != 0) noise_of_element(idx, c2, c3, K, w0, w1, w2);
     uint32_t sp, sm, sv;
     round_element<FLAGS>(r, w0, w1, w2, sp, sm, sv);
     p[i] = static_cast<uint16_t>(sp >> 16);
@@ -110,7 +108,7 @@ __device__ __forceinline__ void step_scalar(uint16_t* p, const void* g, uint16_t
 // ---- flat buffer ---------------------------------------------------------------------------
 // Persistent grid: thread t of the grid takes vectors t, t + T, t + 2T, ... (T = threads in the
 // grid).  VEC = false is the element-wise kernel for unaligned buffers.
-template <bool G32, uint32_t FLAGS, bool CARRY, bool VEC>
+template <bool G32, uint32_t FLAGS, bool PAIRED, bool VEC>
 __global__ void __launch_bounds__(kBlockThreads)
 k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset,
                 uint32_t tensor_id, uint32_t seed_hi, const __grid_constant__ PhiloxKeys K,
@@ -121,7 +119,7 @@ k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n
     if (VEC) {
         const uint64_t nvec = n >> 3;
         for (uint64_t vec = tid; vec < nvec; vec += stride)
-            step_vec8<G32, FLAGS, CARRY>(p, g, m, v, vec, elem_offset + (vec << 3), tensor_id, seed_hi, gscale, K, S);
+            step_vec8<G32, FLAGS, PAIRED>(p, g, m, v, vec, elem_offset + (vec << 3), tensor_id, seed_hi, gscale, K, S);
         const uint64_t done = nvec << 3;
         if (tid < n - done)
             step_scalar<G32, FLAGS>(p, g, m, v, done + tid, elem_offset + done + tid, tensor_id, seed_hi, gscale, K, S);
@@ -133,8 +131,8 @@ k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n
 
 // ---- tensor list ---------------------------------------------------------------------------
 // Blocks walk the chunk table; a chunk is up to kMtChunkElems consecutive elements of one tensor.
-// Element indices restart at 0 in every tensor and chunk starts are multiples of 8, so the
-// counter needs no carry handling.
+// Element indices restart at 0 in every tensor and chunk starts are multiples of 8, so vectors
+// always hold aligned pairs.
 template <bool G32, uint32_t FLAGS>
 __global__ void __launch_bounds__(kBlockThreads)
 k_sr_adamw_mt(const MtTensor* __restrict__ tensors, const MtChunk* __restrict__ chunks, uint32_t num_chunks,
@@ -152,7 +150,7 @@ k_sr_adamw_mt(const MtTensor* __restrict__ tensors, const MtChunk* __restrict__ 
             const uint32_t nvec = len >> 3;
             const uint64_t vec0 = start >> 3;
             for (uint32_t j = threadIdx.x; j < nvec; j += blockDim.x)
-                step_vec8<G32, FLAGS, false>(T.p, T.g, T.m, T.v, vec0 + j, start + (static_cast<uint64_t>(j) << 3), c2,
+                step_vec8<G32, FLAGS, true>(T.p, T.g, T.m, T.v, vec0 + j, start + (static_cast<uint64_t>(j) << 3), c2,
                                              seed_hi, gscale, K, S);
             const uint32_t done = nvec << 3;
             if (threadIdx.x < len - done) {
@@ -167,20 +165,26 @@ k_sr_adamw_mt(const MtTensor* __restrict__ tensors, const MtChunk* __restrict__ 
 }
 
 // ---- standalone Q_SR cast ------------------------------------------------------------------
-template <bool CARRY>
-__device__ __forceinline__ uint32_t downcast_pair(uint32_t b_even, uint32_t b_odd, uint32_t lo, uint32_t hi, uint32_t e,
+// Uses the x slot (word 0) of the same noise layout: one Philox call per two elements.
+template <bool PAIRED>
+__device__ __forceinline__ uint32_t downcast_pair(uint32_t b_even, uint32_t b_odd, uint64_t idx0, uint32_t e,
                                                   uint32_t c2, uint32_t c3, const PhiloxKeys& K) {
-    uint32_t c0, c1, w0, w1, w2, x0, x1, x2;
-    counter_of<CARRY>(lo, hi, e, c0, c1);
-    philox4x32_10(c0, c1, c2, c3, K, w0, w1, w2);
-    counter_of<CARRY>(lo, hi, e + 1, c0, c1);
-    philox4x32_10(c0, c1, c2, c3, K, x0, x1, x2);
-    const uint32_t s0 = is_nan_bits(b_even) ? (kQuietNaNbf16 << 16) : sr_sum(b_even, w0);
-    const uint32_t s1 = is_nan_bits(b_odd) ? (kQuietNaNbf16 << 16) : sr_sum(b_odd, x0);
+    uint32_t r_even, r_odd, w1, w2;
+    if (PAIRED) {
+        uint32_t w0;
+        philox4x32_10(static_cast<uint32_t>(idx0 >> 1) + (e >> 1), static_cast<uint32_t>(idx0 >> 33), c2, c3, K, w0, w1, w2);
+        r_even = noise_even(w0);
+        r_odd = noise_odd(w0);
+    } else {
+        noise_of_element(idx0 + e, c2, c3, K, r_even, w1, w2);
+        noise_of_element(idx0 + e + 1, c2, c3, K, r_odd, w1, w2);
+    }
+    const uint32_t s0 = is_nan_bits(b_even) ? (kQuietNaNbf16 << 16) : sr_sum(b_even, r_even);
+    const uint32_t s1 = is_nan_bits(b_odd) ? (kQuietNaNbf16 << 16) : sr_sum(b_odd, r_odd);
     return pack_top_halves(s0, s1);
 }
 
-template <bool CARRY, bool VEC>
+template <bool PAIRED, bool VEC>
 __global__ void __launch_bounds__(kBlockThreads)
 k_sr_downcast(const float* __restrict__ src, uint16_t* __restrict__ dst, uint64_t n, uint64_t elem_offset,
               uint32_t tensor_id, uint32_t seed_hi, const __grid_constant__ PhiloxKeys K) {
@@ -193,22 +197,20 @@ k_sr_downcast(const float* __restrict__ src, uint16_t* __restrict__ dst, uint64_
             const uint4 a = ld16(src, 2 * vec);
             const uint4 b = ld16(src, 2 * vec + 1);
             const uint64_t idx0 = elem_offset + (vec << 3);
-            const uint32_t lo = static_cast<uint32_t>(idx0), hi = static_cast<uint32_t>(idx0 >> 32);
             uint4 o;
-            o.x = downcast_pair<CARRY>(a.x, a.y, lo, hi, 0, tensor_id, seed_hi, K);
-            o.y = downcast_pair<CARRY>(a.z, a.w, lo, hi, 2, tensor_id, seed_hi, K);
-            o.z = downcast_pair<CARRY>(b.x, b.y, lo, hi, 4, tensor_id, seed_hi, K);
-            o.w = downcast_pair<CARRY>(b.z, b.w, lo, hi, 6, tensor_id, seed_hi, K);
+            o.x = downcast_pair<PAIRED>(a.x, a.y, idx0, 0, tensor_id, seed_hi, K);
+            o.y = downcast_pair<PAIRED>(a.z, a.w, idx0, 2, tensor_id, seed_hi, K);
+            o.z = downcast_pair<PAIRED>(b.x, b.y, idx0, 4, tensor_id, seed_hi, K);
+            o.w = downcast_pair<PAIRED>(b.z, b.w, idx0, 6, tensor_id, seed_hi, K);
             st16(dst, vec, o);
         }
         done = nvec << 3;
     }
     for (uint64_t i = done + tid; i < n; i += stride) {
-        const uint64_t idx = elem_offset + i;
-        uint32_t w0, w1, w2;
-        philox4x32_10(static_cast<uint32_t>(idx), static_cast<uint32_t>(idx >> 32), tensor_id, seed_hi, K, w0, w1, w2);
+        uint32_t r0, r1, r2;
+        noise_of_element(elem_offset + i, tensor_id, seed_hi, K, r0, r1, r2);
         const uint32_t b = __float_as_uint(src[i]);
-        dst[i] = static_cast<uint16_t>((is_nan_bits(b) ? (kQuietNaNbf16 << 16) : sr_sum(b, w0)) >> 16);
+        dst[i] = static_cast<uint16_t>((is_nan_bits(b) ? (kQuietNaNbf16 << 16) : sr_sum(b, r0)) >> 16);
     }
 }
 
@@ -239,13 +241,13 @@ cudaError_t launch_flat_t(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, 
     const bool vec = aligned16(p) && aligned16(g) && aligned16(m) && aligned16(v);
     const uint64_t vec_items = (n >> 3) + 8;   // the extra 8 keep enough threads for the ragged tail
     if (!vec) {
-        auto k = k_sr_adamw_flat<G32, FLAGS, true, false>;
+        auto k = k_sr_adamw_flat<G32, FLAGS, false, false>;
         k<<<grid_for(k, n, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset, tensor_id, seed_hi, K, S);
     } else if ((elem_offset & 7u) == 0) {
-        auto k = k_sr_adamw_flat<G32, FLAGS, false, true>;
+        auto k = k_sr_adamw_flat<G32, FLAGS, true, true>;
         k<<<grid_for(k, vec_items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset, tensor_id, seed_hi, K, S);
     } else {
-        auto k = k_sr_adamw_flat<G32, FLAGS, true, true>;
+        auto k = k_sr_adamw_flat<G32, FLAGS, false, true>;
         k<<<grid_for(k, vec_items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset, tensor_id, seed_hi, K, S);
     }
     return cudaGetLastError();
@@ -304,13 +306,13 @@ cudaError_t launch_downcast(const float* src, uint16_t* dst, uint64_t n, uint64_
                             uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev, cudaStream_t stream) {
     const bool vec = aligned16(src) && aligned16(dst);
     if (!vec) {
-        auto k = k_sr_downcast<true, false>;
+        auto k = k_sr_downcast<false, false>;
         k<<<grid_for(k, n, dev), kBlockThreads, 0, stream>>>(src, dst, n, elem_offset, tensor_id, seed_hi, K);
     } else if ((elem_offset & 7u) == 0) {
-        auto k = k_sr_downcast<false, true>;
+        auto k = k_sr_downcast<true, true>;
         k<<<grid_for(k, (n >> 3) + 8, dev), kBlockThreads, 0, stream>>>(src, dst, n, elem_offset, tensor_id, seed_hi, K);
     } else {
-        auto k = k_sr_downcast<true, true>;
+        auto k = k_sr_downcast<false, true>;
         k<<<grid_for(k, (n >> 3) + 8, dev), kBlockThreads, 0, stream>>>(src, dst, n, elem_offset, tensor_id, seed_hi, K);
     }
     return cudaGetLastError();
