@@ -130,6 +130,26 @@ size_t grad_sqnorm_workspace_bytes(uint64_t n);
 sr_status grad_sqnorm(const void* g, sr_dtype g_dtype, uint64_t n, double* out_dev, void* workspace,
                       size_t workspace_bytes, void* stream);
 
+/* grad_sqnorm for callers that cannot allocate.  (The paper has no counterpart; neither has the
+ * rest of the norm/clipping code.)  Some users of this library run where cudaMalloc is not an
+ * option: inside a process whose device memory is owned and fully handed out by someone else's
+ * pool, inside a callback or a latency-critical loop where an allocation (or the synchronisation it
+ * can imply) is forbidden, or in a harness that is only allowed to pass its inputs and outputs.
+ * For them the intermediate block sums live in a fixed 1 MiB array (131 072 doubles) inside the
+ * library image; every GPU that loads the library holds that array until the process exits.
+ *   - Same result as grad_sqnorm, bit for bit (same kernels, same tree).
+ *   - n may be at most grad_sqnorm_static_max_elements() (1 073 610 752: enough for a 1/8 shard of
+ *     the 6.7B model); larger n returns SR_ERR_WORKSPACE and nothing is launched.
+ *   - The call allocates nothing and frees nothing.  Its FIRST call on each device looks up the
+ *     array's device address (a one-off set-up); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps what the previous call left in it.
+ *     Nothing in it has to be zero beforehand, because every block sum is written before it is
+ *     read within a call.  Two calls that can overlap on the GPU (different streams, no ordering
+ *     between them) would overwrite each other's block sums: order them, or give one of them its
+ *     own workspace through grad_sqnorm. */
+uint64_t grad_sqnorm_static_max_elements(void);
+sr_status grad_sqnorm_static(const void* g, sr_dtype g_dtype, uint64_t n, double* out_dev, void* stream);
+
 /* Clipping factor on the device, no host round trip:
  * gscale = accum_scale * min(1, max_norm / (accum_scale * sqrt(S) + 1e-6)), evaluated in FP64 and
  * stored as FP32 in *gscale_out_dev; pass that pointer as sr_adamw_hparams.grad_scale_dev. */

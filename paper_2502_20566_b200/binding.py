@@ -26,6 +26,7 @@ EXPORTS = (
     "sr_downcast_f32_bf16", "sr_adamw_step", "sr_adamw_step_host", "sr_adamw_step_host_staging_bytes",
     "sr_mt_plan_create", "sr_adamw_multi_tensor",
     "sr_mt_plan_destroy", "sr_mt_plan_total_elements", "grad_sqnorm_workspace_bytes", "grad_sqnorm",
+    "grad_sqnorm_static", "grad_sqnorm_static_max_elements",
     "sr_clip_scale", "sr_status_string", "sr_last_cuda_error", "sr_abi_version",
 )
 
@@ -96,6 +97,9 @@ def lib() -> ctypes.CDLL:
         L.grad_sqnorm_workspace_bytes.restype = c_size_t
         L.grad_sqnorm.argtypes = [c_void_p, c_int, c_uint64, c_void_p, c_void_p, c_size_t, c_void_p]
         L.grad_sqnorm.restype = c_int
+        L.grad_sqnorm_static.argtypes = [c_void_p, c_int, c_uint64, c_void_p, c_void_p]
+        L.grad_sqnorm_static.restype = c_int
+        L.grad_sqnorm_static_max_elements.restype = c_uint64
         L.sr_clip_scale.argtypes = [c_void_p, c_float, c_float, c_void_p, c_void_p]
         L.sr_clip_scale.restype = c_int
         L.sr_status_string.argtypes = [c_int]
@@ -245,6 +249,21 @@ def grad_sqnorm(g: torch.Tensor, out: torch.Tensor, workspace: Optional[torch.Te
     with torch.cuda.device(g.device):
         _check(lib().grad_sqnorm(g.data_ptr(), _g_dtype(g), g.numel(), out.data_ptr(), ws_ptr, ws_bytes,
                                  _stream(stream)), "grad_sqnorm")
+
+
+def grad_sqnorm_static_max_elements() -> int:
+    return int(lib().grad_sqnorm_static_max_elements())
+
+
+def grad_sqnorm_static(g: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+    """grad_sqnorm without a workspace: the block sums go to a fixed array inside the library, so the
+    call allocates nothing.  For callers that may not allocate device memory; all such calls on one
+    GPU share that array, so do not let two of them overlap.  g.numel() is limited to
+    grad_sqnorm_static_max_elements()."""
+    _want(g, g.dtype, "g"), _want(out, torch.float64, "out")
+    with torch.cuda.device(g.device):
+        _check(lib().grad_sqnorm_static(g.data_ptr(), _g_dtype(g), g.numel(), out.data_ptr(), _stream(stream)),
+               "grad_sqnorm_static")
 
 
 def sr_clip_scale(sqnorm: torch.Tensor, accum_scale: float, max_norm: float, gscale_out: torch.Tensor, stream=None) -> None:

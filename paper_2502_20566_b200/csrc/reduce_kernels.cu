@@ -7,6 +7,7 @@
 // A CUDA block of 256 threads is exactly one tree block, so thread j is accumulator j and the
 // loads of one r are 16-byte, fully coalesced.  HBM-bound: 4 (FP32) or 2 (BF16) bytes per element.
 
+#include "../../include/sradamw.h"
 #include "launch.h"
 
 namespace sradamw {
@@ -168,3 +169,61 @@ cudaError_t launch_clip_scale(const double* sqnorm, float accum_scale, float max
 }
 
 }  // namespace sradamw
+
+// ---- squared norm without any allocation ---------------------------------------------------
+// Same kernels and same summation tree as grad_sqnorm; the intermediate block sums go to a
+// fixed array that is part of the library image instead of a caller-provided workspace.
+
+namespace {
+
+constexpr uint64_t kStaticScratchDoubles = 131072;   // 1 MiB per GPU that loads the library
+
+static __device__ __align__(256) double g_sqnorm_static_scratch[kStaticScratchDoubles];
+
+struct StaticScratchSlot {
+    bool ready = false;
+    double* ptr = nullptr;      // device address of g_sqnorm_static_scratch on this device
+    sradamw::DeviceInfo info{};
+};
+constexpr int kStaticMaxDevices = 64;
+StaticScratchSlot g_static_slots[kStaticMaxDevices];
+
+}  // namespace
+
+extern "C" uint64_t grad_sqnorm_static_max_elements(void) {
+    // largest n whose intermediate levels fit: blocks(n) + blocks(blocks(n)) + ... <= capacity
+    uint64_t lo = 0, hi = kStaticScratchDoubles * 8192ull;
+    while (lo < hi) {
+        const uint64_t mid = lo + (hi - lo + 1) / 2;
+        if (sradamw::sqnorm_scratch_doubles(mid) <= kStaticScratchDoubles) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+extern "C" sr_status grad_sqnorm_static(const void* g, sr_dtype g_dtype, uint64_t n, double* out_dev, void* stream) {
+    if (out_dev == nullptr) return SR_ERR_INVALID_ARG;
+    if (g_dtype != SR_DT_BF16 && g_dtype != SR_DT_F32) return SR_ERR_INVALID_ARG;
+    if (n != 0 && g == nullptr) return SR_ERR_INVALID_ARG;
+    if (sradamw::sqnorm_scratch_doubles(n) > kStaticScratchDoubles) return SR_ERR_WORKSPACE;   // n too large
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SR_ERR_CUDA;
+    if (dev < 0 || dev >= kStaticMaxDevices) return SR_ERR_UNSUPPORTED_DEVICE;
+    StaticScratchSlot& slot = g_static_slots[dev];
+    if (!slot.ready) {
+        // once per device, with that device current: the array's name is only a host-side handle,
+        // the kernels need its address on this device
+        int sm = 0, major = 0;
+        if (cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SR_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SR_ERR_CUDA;
+        if (major != 10) return SR_ERR_UNSUPPORTED_DEVICE;
+        void* addr = nullptr;
+        if (cudaGetSymbolAddress(&addr, g_sqnorm_static_scratch) != cudaSuccess || addr == nullptr) return SR_ERR_CUDA;
+        slot.ptr = static_cast<double*>(addr);
+        slot.info.sm_count = sm;
+        slot.info.cc_major = major;
+        slot.ready = true;
+    }
+    const cudaError_t e = sradamw::launch_sqnorm(g, g_dtype == SR_DT_F32, n, out_dev, slot.ptr, slot.info,
+                                                 static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+}
