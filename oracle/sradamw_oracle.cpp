@@ -94,23 +94,32 @@ void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]
 // ---- the optimizer's random state r^(opt)_t ------------------------------------------------
 // Algorithm 1 needs a random state that is the same on every replica at iteration t.  Here the
 // state is a pure function of (seed, step, tensor_id, global element index).  One Philox call
-// yields 128 bits while one element needs 3 x 16, so two neighbouring elements share a call:
-//   pair    = index >> 1
+// yields 128 bits = eight 16-bit noise values, so one call serves one rounding slot (0: x, 1: m,
+// 2: v) of a group of eight consecutive elements:
+//   group   = index >> 3,   e = index & 7
+//   number  = 4 * group + slot                       (a 64-bit integer)
 //   key     = (seed[31:0], step)
-//   counter = (pair[31:0], pair[63:32], tensor_id, seed[63:32])
-// Output words 0, 1, 2 serve the roundings of x, m and v (word 3 is unused); in each word the
-// element with even index takes the low 16 bits and the element with odd index the high 16 bits.
-struct Noise3 { uint32_t rp, rm, rv; };
-
-Noise3 noise_for(uint64_t seed, uint32_t step, uint32_t tensor_id, uint64_t index) {
-    const uint64_t pair = index >> 1;
-    const uint32_t ctr[4] = {static_cast<uint32_t>(pair), static_cast<uint32_t>(pair >> 32),
+//   counter = (number[31:0], number[63:32], tensor_id, seed[63:32])
+// Elements 2j and 2j+1 of the group share output word j: the even one takes its low 16 bits, the
+// odd one its high 16 bits.  Every bit of every call is used exactly once.
+uint32_t noise_for_slot(uint64_t seed, uint32_t step, uint32_t tensor_id, uint64_t index, uint32_t slot) {
+    const uint64_t group = index >> 3;
+    const uint32_t e = static_cast<uint32_t>(index & 7u);
+    const uint64_t number = 4u * group + slot;
+    const uint32_t ctr[4] = {static_cast<uint32_t>(number), static_cast<uint32_t>(number >> 32),
                              tensor_id, static_cast<uint32_t>(seed >> 32)};
     const uint32_t key[2] = {static_cast<uint32_t>(seed), step};
     uint32_t w[4];
     philox4x32_10(ctr, key, w);
-    if (index & 1u) return Noise3{w[0] >> 16, w[1] >> 16, w[2] >> 16};
-    return Noise3{w[0] & 0xFFFFu, w[1] & 0xFFFFu, w[2] & 0xFFFFu};
+    const uint32_t word = w[e >> 1];
+    return (e & 1u) ? (word >> 16) : (word & 0xFFFFu);
+}
+
+struct Noise3 { uint32_t rp, rm, rv; };
+
+Noise3 noise_for(uint64_t seed, uint32_t step, uint32_t tensor_id, uint64_t index) {
+    return Noise3{noise_for_slot(seed, step, tensor_id, index, 0), noise_for_slot(seed, step, tensor_id, index, 1),
+                  noise_for_slot(seed, step, tensor_id, index, 2)};
 }
 
 // ---- Eq. 2 by dithering --------------------------------------------------------------------
@@ -271,13 +280,13 @@ int oracle_adamw_step(uint16_t* p, const void* g, int g_is_f32, uint16_t* m, uin
     return 0;
 }
 
-// Q_SR on an FP32 array; uses the first noise word only.
+// Q_SR on an FP32 array; uses rounding slot 0 (the x slot) of the noise.
 void oracle_sr_downcast(const float* src, uint16_t* dst, uint64_t n, uint64_t seed, uint32_t step,
                         uint32_t tensor_id, uint64_t elem_offset) {
 #pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < static_cast<int64_t>(n); ++i) {
-        const Noise3 r = noise_for(seed, step, tensor_id, elem_offset + static_cast<uint64_t>(i));
-        dst[i] = sr_bf16_bits(bits_of(src[i]), r.rp);
+        const uint32_t r = noise_for_slot(seed, step, tensor_id, elem_offset + static_cast<uint64_t>(i), 0);
+        dst[i] = sr_bf16_bits(bits_of(src[i]), r);
     }
 }
 

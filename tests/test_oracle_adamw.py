@@ -228,12 +228,13 @@ def _compose_expected(pb, g_f32, mb, vb, hp, seed, step, tensor_id, offset, gsca
         F = lambda h: bits_f32(int(h) << 16)
         t = oracle.adamw_element(F(pb[i]), float(g_f32[i]), F(mb[i]), F(vb[i]), gscale, sc)
         idx = offset + i
-        pair = idx >> 1
-        w = oracle.philox4x32_10([pair & 0xFFFFFFFF, pair >> 32, tensor_id, seed >> 32], [seed & 0xFFFFFFFF, step])
         res = []
         for k, val in enumerate((t.x_new, t.m_new, t.v_new)):
             fb = f32_bits(val)
-            r = (w[k] >> 16) if idx & 1 else (w[k] & 0xFFFF)
+            number = 4 * (idx >> 3) + k
+            w = oracle.philox4x32_10([number & 0xFFFFFFFF, number >> 32, tensor_id, seed >> 32], [seed & 0xFFFFFFFF, step])
+            word = w[(idx & 7) >> 1]
+            r = (word >> 16) if idx & 1 else (word & 0xFFFF)
             res.append(oracle.sr_bf16_bits(fb, r) if flags & (1 << k) else oracle.rne_bf16_bits(fb))
         out.append(res)
     return np.array(out, dtype=np.uint16)
@@ -299,8 +300,8 @@ def test_sr_downcast_array_and_offsets():
     out = oracle.sr_downcast(src, seed=7)
     b = src.view(np.uint32)
     for i in range(0, 5000, 7):
-        w = oracle.philox4x32_10([i >> 1, 0, 0, 0], [7, 0])
-        assert out[i] == oracle.sr_bf16_bits(int(b[i]), (w[0] >> 16) if i & 1 else (w[0] & 0xFFFF))
+        w = oracle.philox4x32_10([4 * (i >> 3), 0, 0, 0], [7, 0])[(i & 7) >> 1]
+        assert out[i] == oracle.sr_bf16_bits(int(b[i]), (w >> 16) if i & 1 else (w & 0xFFFF))
     shifted = oracle.sr_downcast(np.ascontiguousarray(src[1000:2000]), seed=7, elem_offset=1000)
     assert np.array_equal(shifted, out[1000:2000])
     nan = is_nan_bits_array(b)

@@ -49,28 +49,35 @@ def test_philox_is_sensitive_to_every_input_word():
         assert oracle.philox4x32_10([1, 2, 3, 4], k) != base
 
 
-def _half(word, index):
-    return (word >> 16) if index & 1 else (word & 0xFFFF)
+def _expected_noise(seed, step, tid, idx):
+    """Noise layout written out: one call per (group of 8 elements, rounding slot)."""
+    group, e = idx >> 3, idx & 7
+    out = []
+    for slot in range(3):
+        number = 4 * group + slot
+        w = oracle.philox4x32_10([number & 0xFFFFFFFF, number >> 32, tid, seed >> 32], [seed & 0xFFFFFFFF, step])
+        word = w[e >> 1]
+        out.append((word >> 16) if e & 1 else (word & 0xFFFF))
+    return tuple(out)
 
 
 def test_noise_layout_key_counter_and_words():
-    """key = (seed low, step); counter = (pair low, pair high, tensor_id, seed high) with
-    pair = index >> 1; words 0, 1, 2 serve x, m, v; even index -> low half, odd index -> high half."""
+    """key = (seed low, step); counter = (number low, number high, tensor_id, seed high) with
+    number = 4 * (index >> 3) + slot; element e = index & 7 uses word e >> 1, low half if e is even."""
     seed, step, tid = 0x1234_5678_9ABC_DEF0, 77, 9
-    for idx in ((5 << 32) | 0xFFFF_FFF3, (5 << 32) | 0xFFFF_FFF2, (1 << 33) - 1, 1 << 33, 0, 1):
-        pair = idx >> 1
-        w = oracle.philox4x32_10([pair & 0xFFFFFFFF, pair >> 32, tid, seed >> 32], [seed & 0xFFFFFFFF, step])
-        assert oracle.noise(seed, step, tid, idx) == tuple(_half(w[k], idx) for k in range(3))
+    for idx in ((5 << 32) | 0xFFFF_FFF3, (5 << 32) | 0xFFFF_FFF8, (1 << 33) - 1, 1 << 33, (1 << 61) + 5, 0, 1, 7, 8):
+        assert oracle.noise(seed, step, tid, idx) == _expected_noise(seed, step, tid, idx)
 
 
-def test_two_elements_of_a_pair_use_disjoint_bits():
-    """The 96 bits a pair consumes are six different 16-bit fields of one call: together the two
-    elements reproduce words 0..2 exactly."""
-    for idx in (0, 2, 10**12):
-        a, b = oracle.noise(3, 4, 5, idx), oracle.noise(3, 4, 5, idx + 1)
-        pair = idx >> 1
-        w = oracle.philox4x32_10([pair & 0xFFFFFFFF, pair >> 32, 5, 0], [3, 4])
-        assert tuple(a[k] | (b[k] << 16) for k in range(3)) == w[:3]
+def test_a_group_of_eight_uses_every_bit_once():
+    """The eight elements of a group reproduce, slot by slot, all four words of that slot's call."""
+    for base in (0, 8, 8 * 10**12):
+        got = [oracle.noise(3, 4, 5, base + e) for e in range(8)]
+        for slot in range(3):
+            number = 4 * (base >> 3) + slot
+            w = oracle.philox4x32_10([number & 0xFFFFFFFF, number >> 32, 5, 0], [3, 4])
+            words = [got[2 * j][slot] | (got[2 * j + 1][slot] << 16) for j in range(4)]
+            assert tuple(words) == w
 
 
 def test_noise_streams_differ():
@@ -79,7 +86,7 @@ def test_noise_streams_differ():
     assert [oracle.noise(1, 2, 0, i) for i in range(64)] != ref            # iteration
     assert [oracle.noise(1, 1, 1, i) for i in range(64)] != ref            # tensor
     assert [oracle.noise(1 | (1 << 32), 1, 0, i) for i in range(64)] != ref  # high half of the seed
-    assert [oracle.noise(1, 1, 0, i + (1 << 33)) for i in range(64)] != ref  # high half of the pair index
+    assert [oracle.noise(1, 1, 0, i + (1 << 33)) for i in range(64)] != ref  # high half of the call number
     assert len(set(ref)) == 64
 
 
