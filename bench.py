@@ -226,7 +226,7 @@ def run_ours(args):
 
     for w in range(args.warmup):
         binding.sr_adamw_step(p, g, m, v, hp, SEED, FIRST_STEP + w)
-    sampler = ClockSampler(torch, local) if rank == 0 else None
+    sampler = ClockSampler(torch, local) if rank == 0 and not os.environ.get("SRADAMW_NO_CLOCK_SAMPLER") else None
     if sampler is not None:
         time.sleep(0.3)          # let the poller start
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]

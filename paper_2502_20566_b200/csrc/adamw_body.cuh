@@ -1,0 +1,203 @@
+// Vector and element bodies of the fused SR-AdamW step, shared by the flat and the multi-tensor
+// kernels.  One read of x, g, m, v and one write of x, m, v per element; Philox, the FP32 update of
+// Algorithm 1 and the dithering add stay in registers.
+//
+// Each thread moves 8 consecutive elements per iteration with 16-byte loads and stores, so a warp
+// touches 512 contiguous bytes per array; all accesses carry the streaming (evict-first) hint
+// because every byte is used exactly once.
+#pragma once
+
+#include "launch.h"
+
+namespace sradamw {
+
+// ---- 16-byte streaming accesses ------------------------------------------------------------
+__device__ __forceinline__ uint4 ld16(const void* base, uint64_t vec) {
+    return __ldcs(reinterpret_cast<const uint4*>(base) + vec);
+}
+__device__ __forceinline__ void st16(void* base, uint64_t vec, uint4 val) {
+    __stcs(reinterpret_cast<uint4*>(base) + vec, val);
+}
+
+// the eight gradient values of a vector as FP32
+template <bool G32>
+__device__ __forceinline__ void load_grad8(const void* g, uint64_t vec, float (&ge)[8]) {
+    if (G32) {
+        const uint4 g0 = ld16(g, 2 * vec);
+        const uint4 g1 = ld16(g, 2 * vec + 1);
+        ge[0] = __uint_as_float(g0.x); ge[1] = __uint_as_float(g0.y);
+        ge[2] = __uint_as_float(g0.z); ge[3] = __uint_as_float(g0.w);
+        ge[4] = __uint_as_float(g1.x); ge[5] = __uint_as_float(g1.y);
+        ge[6] = __uint_as_float(g1.z); ge[7] = __uint_as_float(g1.w);
+    } else {
+        const uint4 gv = ld16(g, vec);
+        ge[0] = bf16_lo(gv.x); ge[1] = bf16_hi(gv.x);
+        ge[2] = bf16_lo(gv.y); ge[3] = bf16_hi(gv.y);
+        ge[4] = bf16_lo(gv.z); ge[5] = bf16_hi(gv.z);
+        ge[6] = bf16_lo(gv.w); ge[7] = bf16_hi(gv.w);
+    }
+}
+
+__device__ __forceinline__ uint32_t word_of(const uint4& w, int j) { return j == 0 ? w.x : j == 1 ? w.y : j == 2 ? w.z : w.w; }
+
+// ---- reference vector: IEEE square root / division, NaN rule -------------------------------
+// GROUPED = true needs idx0 (global index of the vector's first element) to be a multiple of 8: the
+// vector is then exactly one noise group and three Philox calls serve it.  GROUPED = false draws
+// every element's noise on its own and is valid for any idx0.  Kept out of line: the fast kernels
+// call it only for the rare vector that leaves the fast range.
+template <bool G32, uint32_t FLAGS, bool GROUPED>
+__device__ __noinline__ void step_vec8_reference(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t vec,
+                                                 uint64_t idx0, uint32_t c2, uint32_t c3, float gscale,
+                                                 const PhiloxKeys& K, const StepScalars& S) {
+    const uint4 pv = ld16(p, vec), mv = ld16(m, vec), vv = ld16(v, vec);
+    float ge[8];
+    load_grad8<G32>(g, vec, ge);
+    uint4 wx = make_uint4(0, 0, 0, 0), wm = wx, wv = wx;
+    if (GROUPED) {
+        const uint32_t c0 = static_cast<uint32_t>(idx0 >> 1), c1 = static_cast<uint32_t>(idx0 >> 33);
+        if (FLAGS & 1u) wx = philox4x32_10(c0, c1, c2, c3, K);
+        if (FLAGS & 2u) wm = philox4x32_10(c0 + 1, c1, c2, c3, K);
+        if (FLAGS & 4u) wv = philox4x32_10(c0 + 2, c1, c2, c3, K);
+    }
+    uint32_t po[4], mo[4], vo[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint32_t pw = word_of(pv, j), mw = word_of(mv, j), vw = word_of(vv, j);
+        const ElementOut r0 = adamw_element(bf16_lo(pw), ge[2 * j], bf16_lo(mw), bf16_lo(vw), gscale, S);
+        const ElementOut r1 = adamw_element(bf16_hi(pw), ge[2 * j + 1], bf16_hi(mw), bf16_hi(vw), gscale, S);
+        uint32_t x0, x1, m0, m1, v0, v1;   // 16-bit noise per element and slot
+        if (GROUPED) {
+            const uint32_t ax = word_of(wx, j), am = word_of(wm, j), av = word_of(wv, j);
+            x0 = ax & 0xFFFFu; x1 = ax >> 16; m0 = am & 0xFFFFu; m1 = am >> 16; v0 = av & 0xFFFFu; v1 = av >> 16;
+        } else {
+            const uint64_t i0 = idx0 + 2 * j, i1 = i0 + 1;
+            x0 = (FLAGS & 1u) ? noise_of_element(i0, 0, c2, c3, K) : 0u;
+            x1 = (FLAGS & 1u) ? noise_of_element(i1, 0, c2, c3, K) : 0u;
+            m0 = (FLAGS & 2u) ? noise_of_element(i0, 1, c2, c3, K) : 0u;
+            m1 = (FLAGS & 2u) ? noise_of_element(i1, 1, c2, c3, K) : 0u;
+            v0 = (FLAGS & 4u) ? noise_of_element(i0, 2, c2, c3, K) : 0u;
+            v1 = (FLAGS & 4u) ? noise_of_element(i1, 2, c2, c3, K) : 0u;
+        }
+        po[j] = pack_top_halves(round_sum_r16_nan_safe<(FLAGS & 1u) != 0>(r0.x, x0),
+                                round_sum_r16_nan_safe<(FLAGS & 1u) != 0>(r1.x, x1));
+        mo[j] = pack_top_halves(round_sum_r16_nan_safe<(FLAGS & 2u) != 0>(r0.m, m0),
+                                round_sum_r16_nan_safe<(FLAGS & 2u) != 0>(r1.m, m1));
+        vo[j] = pack_top_halves(round_sum_r16_nan_safe<(FLAGS & 4u) != 0>(r0.v, v0),
+                                round_sum_r16_nan_safe<(FLAGS & 4u) != 0>(r1.v, v1));
+    }
+    st16(p, vec, make_uint4(po[0], po[1], po[2], po[3]));
+    st16(m, vec, make_uint4(mo[0], mo[1], mo[2], mo[3]));
+    st16(v, vec, make_uint4(vo[0], vo[1], vo[2], vo[3]));
+}
+
+// ---- fast vector: branch-free arithmetic, one range test per vector ------------------------
+// idx0 must be a multiple of 8.  c0 = low word of idx0 >> 1, c1 = idx0 >> 33 (uniform over a launch
+// segment or a chunk, which lets the compiler hoist the round-1/round-2 products that depend only
+// on c1, c2 and the keys).
+template <bool G32, uint32_t FLAGS, bool SCALE>
+__device__ __forceinline__ void step_vec8_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t vec,
+                                               uint64_t idx0, uint32_t c1, uint32_t c2, uint32_t c3, float gscale,
+                                               const PhiloxKeys& K, const StepScalars& S) {
+    const uint4 pv = ld16(p, vec), mv = ld16(m, vec), vv = ld16(v, vec);
+    float ge[8];
+    load_grad8<G32>(g, vec, ge);
+    const uint32_t c0 = static_cast<uint32_t>(idx0 >> 1);
+    uint4 wx = make_uint4(0, 0, 0, 0), wm = wx, wv = wx;
+    if (FLAGS & 1u) wx = philox4x32_10(c0, c1, c2, c3, K);
+    if (FLAGS & 2u) wm = philox4x32_10(c0 + 1, c1, c2, c3, K);
+    if (FLAGS & 4u) wv = philox4x32_10(c0 + 2, c1, c2, c3, K);
+    RangeTrack track;
+    track.init();
+    uint32_t po[4], mo[4], vo[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint32_t pw = word_of(pv, j), mw = word_of(mv, j), vw = word_of(vv, j);
+        const ElementOut r0 = adamw_element_in_range<SCALE>(bf16_lo(pw), ge[2 * j], bf16_lo(mw), bf16_lo(vw), gscale, S);
+        const ElementOut r1 = adamw_element_in_range<SCALE>(bf16_hi(pw), ge[2 * j + 1], bf16_hi(mw), bf16_hi(vw), gscale, S);
+        track.add(r0, r1);
+        po[j] = pack_top_halves(round_sum_word<(FLAGS & 1u) != 0, false>(r0.x, word_of(wx, j)),
+                                round_sum_word<(FLAGS & 1u) != 0, true>(r1.x, word_of(wx, j)));
+        mo[j] = pack_top_halves(round_sum_word<(FLAGS & 2u) != 0, false>(r0.m, word_of(wm, j)),
+                                round_sum_word<(FLAGS & 2u) != 0, true>(r1.m, word_of(wm, j)));
+        vo[j] = pack_top_halves(round_sum_word<(FLAGS & 4u) != 0, false>(r0.v, word_of(wv, j)),
+                                round_sum_word<(FLAGS & 4u) != 0, true>(r1.v, word_of(wv, j)));
+    }
+    if (track.left_range()) {
+        // nothing has been stored yet: redo this vector from memory with the reference arithmetic
+        step_vec8_reference<G32, FLAGS, true>(p, g, m, v, vec, idx0, c2, c3, gscale, K, S);
+        return;
+    }
+    st16(p, vec, make_uint4(po[0], po[1], po[2], po[3]));
+    st16(m, vec, make_uint4(mo[0], mo[1], mo[2], mo[3]));
+    st16(v, vec, make_uint4(vo[0], vo[1], vo[2], vo[3]));
+}
+
+// ---- one element with 2-byte accesses: ragged tails, unaligned buffers ---------------------
+template <bool G32, uint32_t FLAGS>
+__device__ __forceinline__ void step_scalar(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t i,
+                                            uint64_t idx, uint32_t c2, uint32_t c3, float gscale, const PhiloxKeys& K,
+                                            const StepScalars& S) {
+    const float x = __uint_as_float(static_cast<uint32_t>(p[i]) << 16);
+    const float mi = __uint_as_float(static_cast<uint32_t>(m[i]) << 16);
+    const float vi = __uint_as_float(static_cast<uint32_t>(v[i]) << 16);
+    const float gi = G32 ? static_cast<const float*>(g)[i]
+                         : __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t*>(g)[i]) << 16);
+    const ElementOut r = adamw_element(x, gi, mi, vi, gscale, S);
+    const uint32_t rx = (FLAGS & 1u) ? noise_of_element(idx, 0, c2, c3, K) : 0u;
+    const uint32_t rm = (FLAGS & 2u) ? noise_of_element(idx, 1, c2, c3, K) : 0u;
+    const uint32_t rv = (FLAGS & 4u) ? noise_of_element(idx, 2, c2, c3, K) : 0u;
+    p[i] = static_cast<uint16_t>(round_sum_r16_nan_safe<(FLAGS & 1u) != 0>(r.x, rx) >> 16);
+    m[i] = static_cast<uint16_t>(round_sum_r16_nan_safe<(FLAGS & 2u) != 0>(r.m, rm) >> 16);
+    v[i] = static_cast<uint16_t>(round_sum_r16_nan_safe<(FLAGS & 4u) != 0>(r.v, rv) >> 16);
+}
+
+// ---- launch helpers ------------------------------------------------------------------------
+inline bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
+
+template <typename Kernel>
+int resident_blocks(Kernel kernel, const DeviceInfo& dev) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kBlockThreads, 0) != cudaSuccess || per_sm < 1)
+        per_sm = 1;
+    return per_sm * dev.sm_count;
+}
+
+// grid for `work_items` thread-items: no more blocks than are resident at once, no more than needed
+template <typename Kernel>
+unsigned grid_for(Kernel kernel, uint64_t work_items, const DeviceInfo& dev) {
+    const uint64_t needed = (work_items + kBlockThreads - 1) / kBlockThreads;
+    const uint64_t resident = static_cast<uint64_t>(resident_blocks(kernel, dev));
+    const uint64_t g = needed < resident ? needed : resident;
+    return static_cast<unsigned>(g < 1 ? 1 : g);
+}
+
+// The branch-free path needs den = sqrt(v1) * rsqrt_bc2 + eps to stay inside the range its
+// division was validated for.
+inline bool fast_path_allowed(const StepScalars& S) {
+    return S.rsqrt_bc2 >= 1.0f && S.rsqrt_bc2 <= 1024.0f && S.eps >= 0.0f && S.eps <= 1.0f;
+}
+inline bool needs_scale(const StepScalars& S) { return S.gscale_dev != nullptr || S.gscale != 1.0f; }
+
+#define SR_DISPATCH_FLAGS(CALL)                    \
+    switch (flags & 7u) {                          \
+        case 0: return CALL(0);                    \
+        case 1: return CALL(1);                    \
+        case 2: return CALL(2);                    \
+        case 3: return CALL(3);                    \
+        case 4: return CALL(4);                    \
+        case 5: return CALL(5);                    \
+        case 6: return CALL(6);                    \
+        default: return CALL(7);                   \
+    }
+
+// per gradient type, defined in adamw_flat_*.cu / adamw_mt_*.cu
+template <bool G32>
+cudaError_t launch_adamw_flat_g(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset,
+                                uint32_t tensor_id, uint32_t seed_hi, uint32_t flags, const PhiloxKeys& K,
+                                const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream);
+template <bool G32>
+cudaError_t launch_adamw_mt_g(const MtTensor* tensors, const MtChunk* chunks, uint32_t num_chunks,
+                              uint32_t tensor_id_base, uint32_t seed_hi, uint32_t flags, const PhiloxKeys& K,
+                              const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream);
+
+}  // namespace sradamw

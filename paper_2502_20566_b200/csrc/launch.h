@@ -25,7 +25,18 @@ struct MtChunk {
 };
 
 constexpr uint32_t kMtChunkElems = 16384;   // multiple of 8 * block size
-constexpr int kBlockThreads = 256;
+#ifndef SR_BLOCK_THREADS
+#define SR_BLOCK_THREADS 128
+#endif
+#ifndef SR_MIN_BLOCKS_PER_SM
+#define SR_MIN_BLOCKS_PER_SM 5
+#endif
+constexpr int kBlockThreads = SR_BLOCK_THREADS;
+// Launch shape of the fused-step kernels, from a sweep on B200 (6.7B flat buffer): 128-thread
+// blocks with at least 5 resident per SM (96 registers per thread, 640 threads per SM) was the
+// best of 64..512 threads x 1..10 blocks; tighter register budgets cost more in instruction
+// scheduling than they gain in occupancy.
+constexpr int kMinBlocksPerSM = SR_MIN_BLOCKS_PER_SM;
 
 struct DeviceInfo {
     int sm_count;

@@ -15,6 +15,7 @@ namespace sradamw {
 namespace {
 
 constexpr uint32_t kTreeBlock = 8192;
+constexpr int kTreeThreads = 256;   // one thread per accumulator of the tree: fixed by the contract
 
 // squares are exact in double for FP32 / BF16 inputs, so fma(g, g, acc) rounds once, exactly like
 // acc + g*g
@@ -41,7 +42,7 @@ __device__ __forceinline__ double fold_block(double acc, double* warp_sums) {
 
 // First pass: out[c] = tree-block sum of squares of entries [c*8192, (c+1)*8192) of g.
 template <bool G32>
-__global__ void __launch_bounds__(kBlockThreads)
+__global__ void __launch_bounds__(kTreeThreads)
 k_sqnorm_pass1(const void* __restrict__ g, uint64_t n, uint64_t num_blocks, bool vec_ok, double* __restrict__ out) {
     __shared__ double warp_sums[8];
     const uint32_t j = threadIdx.x;
@@ -91,7 +92,7 @@ k_sqnorm_pass1(const void* __restrict__ g, uint64_t n, uint64_t num_blocks, bool
 }
 
 // Later passes: the same rule on an array of doubles (no squaring).
-__global__ void __launch_bounds__(kBlockThreads)
+__global__ void __launch_bounds__(kTreeThreads)
 k_tree_pass(const double* __restrict__ in, uint64_t count, uint64_t num_blocks, double* __restrict__ out) {
     __shared__ double warp_sums[8];
     const uint32_t j = threadIdx.x;
@@ -143,9 +144,9 @@ cudaError_t launch_sqnorm(const void* g, bool g_f32, uint64_t n, double* out, do
     {
         const unsigned grid = static_cast<unsigned>(count < cap ? count : cap);
         if (g_f32)
-            k_sqnorm_pass1<true><<<grid, kBlockThreads, 0, stream>>>(g, n, count, vec_ok, level_out);
+            k_sqnorm_pass1<true><<<grid, kTreeThreads, 0, stream>>>(g, n, count, vec_ok, level_out);
         else
-            k_sqnorm_pass1<false><<<grid, kBlockThreads, 0, stream>>>(g, n, count, vec_ok, level_out);
+            k_sqnorm_pass1<false><<<grid, kTreeThreads, 0, stream>>>(g, n, count, vec_ok, level_out);
         cudaError_t err = cudaGetLastError();
         if (err != cudaSuccess) return err;
     }
@@ -154,7 +155,7 @@ cudaError_t launch_sqnorm(const void* g, bool g_f32, uint64_t n, double* out, do
         const double* level_in = level_out;
         level_out = next == 1 ? out : level_out + count;
         const unsigned grid = static_cast<unsigned>(next < cap ? next : cap);
-        k_tree_pass<<<grid, kBlockThreads, 0, stream>>>(level_in, count, next, level_out);
+        k_tree_pass<<<grid, kTreeThreads, 0, stream>>>(level_in, count, next, level_out);
         cudaError_t err = cudaGetLastError();
         if (err != cudaSuccess) return err;
         count = next;
