@@ -20,11 +20,13 @@
  *     than SR_ERR_CUDA.  The device must have compute capability 10.x.
  *
  * The optimizer's random state (Algorithm 1: r^(opt)_t, equal on every replica) is a pure function
- * of the arguments.  With index = elem_offset + position in the buffer and pair = index >> 1, the
- * noise comes from Philox4x32-10 with key (seed[31:0], step) and counter
- * (pair[31:0], pair[63:32], tensor_id, seed[63:32]): two neighbouring elements share one call.
- * Output words 0, 1, 2 serve the roundings of x, m, v (sr_downcast_f32_bf16 uses word 0); the
- * element with even index takes the low 16 bits of each word, the one with odd index the high 16.
+ * of the arguments.  With index = elem_offset + position in the buffer, one Philox4x32-10 call
+ * serves one rounding slot (0: x, 1: m, 2: v) of a group of eight consecutive indices:
+ *   number  = 4 * (index >> 3) + slot                         (64-bit)
+ *   key     = (seed[31:0], step)
+ *   counter = (number[31:0], number[63:32], tensor_id, seed[63:32])
+ * Element e = index & 7 uses output word e >> 1, its low 16 bits if e is even, its high 16 bits if
+ * e is odd; every bit of every call is used once.  sr_downcast_f32_bf16 uses slot 0.
  * Two ranks, two shards or two runs with equal (seed, step, tensor_id, index) therefore round
  * identically, which is what the shared random state of Algorithm 1 is for.
  */
@@ -70,7 +72,7 @@ typedef struct sr_adamw_hparams {
     uint32_t flags;              /* SR_FLAG_*; other bits must be zero                                         */
 } sr_adamw_hparams;
 
-/* Eq. 2 on an array: dst[i] = Q_SR(src[i]) using the x slot of the noise at index elem_offset + i.
+/* Eq. 2 on an array: dst[i] = Q_SR(src[i]) using slot 0 of the noise at index elem_offset + i.
  * src: n FP32 values; dst: n BF16 patterns.  step may be 0 here.
  * NaN inputs give the quiet NaN 0x7FC0; +-0, +-inf and values already representable pass through. */
 sr_status sr_downcast_f32_bf16(const float* src, uint16_t* dst, uint64_t n, uint64_t seed, uint32_t step,
