@@ -33,9 +33,11 @@ SEED = 1234
 FIRST_STEP = 1000
 BYTES_PER_ELEMENT = 14          # read x, g, m, v (4 x 2 B) + write x, m, v (3 x 2 B)
 FALLBACK_HBM_GBS = 6650.0       # used only when MEASURED_PEAKS.json is absent
-# dram__bytes_read.sum + dram__bytes_write.sum per element from the committed ncu capture of the
-# current kernel (profiles/); None until a capture of this kernel version exists
-NCU_TRAFFIC_BYTES_PER_ELEMENT = None
+# (dram__bytes_read.sum + dram__bytes_write.sum) / elements from the ncu capture of the current kernel on
+# the 2^27-element case (profiles/k_sr_adamw_flat__bf16_grads_sr_xmv__2pow27.md); traffic of a streaming
+# kernel grows in proportion to the element count, so the full-size figure is this times n.  Set to
+# None whenever the kernel changes until a new capture exists.
+NCU_TRAFFIC_BYTES_PER_ELEMENT = (1.073966e9 + 0.748455424e9) / (1 << 27)
 
 
 def parse_args():
@@ -48,6 +50,7 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-elements", type=int, default=1 << 29)
+    ap.add_argument("--no-extras", action="store_true", help="skip the secondary kernels (shard step, tensor list, cast)")
     return ap.parse_args()
 
 
@@ -184,6 +187,76 @@ def run_reference(args):
 # CUDA arm
 # ---------------------------------------------------------------------------------------------
 
+def time_extras(torch, binding, synth, dev, peak):
+    """The other calls of the library, each timed alone (CUDA events, 3 warm-ups + 10 launches) on its
+    own workload; bytes are the algorithmic ones.  Reported beside the headline, not part of it."""
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, reps=10):
+        for _ in range(3):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    out = {}
+    # 1/8 shard with FP32 gradients: squared norm -> clip factor -> step (20 B per element over two passes)
+    n = synth.gpt_flat_numel() // 8
+    p, g, m, v = synth.adamw_state(n, SEED, dev, g_dtype=torch.float32, outlier_fraction=0.01)
+    ws = torch.empty(max(1, binding.grad_sqnorm_workspace_bytes(n) // 8), dtype=torch.float64, device=dev)
+    S = torch.zeros(1, dtype=torch.float64, device=dev)
+    gs = torch.zeros(1, dtype=torch.float32, device=dev)
+    hp_clip = binding.hparams(**HP, grad_scale_dev=gs)
+    t_norm = timed(lambda: binding.grad_sqnorm(g, S, ws))
+    t_step = timed(lambda: binding.sr_adamw_step(p, g, m, v, hp_clip, SEED, FIRST_STEP, 0, 3 * n))
+
+    def clipped():
+        binding.grad_sqnorm(g, S, ws)
+        binding.sr_clip_scale(S, 0.125, 1.0, gs)
+        binding.sr_adamw_step(p, g, m, v, hp_clip, SEED, FIRST_STEP, 0, 3 * n)
+    t_all = timed(clipped)
+    out["shard_fp32_grads"] = {
+        "elements": n,
+        "grad_sqnorm": {"ms": t_norm, "gbs": 4 * n / t_norm / 1e6, "frac": 4 * n / t_norm / 1e6 / peak},
+        "sr_adamw_step_f32g": {"ms": t_step, "gbs": 16 * n / t_step / 1e6, "frac": 16 * n / t_step / 1e6 / peak},
+        "norm_clip_step": {"ms": t_all, "params_per_s": n / t_all * 1e3, "gbs": 20 * n / t_all / 1e6,
+                           "frac": 20 * n / t_all / 1e6 / peak},
+    }
+    del p, g, m, v, ws
+    # GPT-2 350M tensor list, one launch per step
+    specs = synth.gpt2_param_list()
+    P = [synth.init_param(sp, SEED, i, dev) for i, sp in enumerate(specs)]
+    G = [synth.fresh_grad(sp, 4321, 1, i, dev) for i, sp in enumerate(specs)]
+    M = [torch.zeros_like(t) for t in P]
+    V = [torch.zeros_like(t) for t in P]
+    plan = binding.sr_mt_plan_create(P, G, M, V)
+    hp = binding.hparams(**HP)
+    step = [0]
+
+    def mt():
+        step[0] += 1
+        binding.sr_adamw_multi_tensor(plan, hp, SEED, step[0])
+    t_mt = timed(mt)
+    ne = plan.total_elements
+    out["tensor_list_gpt2_350m"] = {"tensors": len(specs), "elements": ne, "ms": t_mt, "params_per_s": ne / t_mt * 1e3,
+                                    "gbs": 14 * ne / t_mt / 1e6, "frac": 14 * ne / t_mt / 1e6 / peak}
+    plan.destroy()
+    del P, G, M, V
+    # standalone stochastic-rounding cast, 2^28 FP32 values (6 B per element)
+    nc = 1 << 28
+    src = synth.downcast_mix(nc, 7, dev)
+    dst = torch.empty(nc, dtype=torch.bfloat16, device=dev)
+    t_c = timed(lambda: binding.sr_downcast_f32_bf16(src, dst, seed=7))
+    out["sr_downcast_f32_bf16"] = {"elements": nc, "ms": t_c, "params_per_s": nc / t_c * 1e3, "gbs": 6 * nc / t_c / 1e6,
+                                   "frac": 6 * nc / t_c / 1e6 / peak}
+    return out
+
+
 def hbm_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -314,9 +387,12 @@ def run_ours(args):
     }
     if e2e is not None:
         line["e2e"] = e2e
-    if world == 1 and not args.no_cpu_baseline:
-        del bufs, p, g, m, v
+    del bufs, p, g, m, v
+    torch.cuda.empty_cache()
+    if world == 1 and not args.no_extras and not args.elements:
+        line["extras"] = time_extras(torch, binding, synth, dev, peak)
         torch.cuda.empty_cache()
+    if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = time_oracle(1 << 28)
     print(json.dumps(line), flush=True)
     if dist is not None:
