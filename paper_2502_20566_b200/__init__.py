@@ -5,6 +5,7 @@ Submodules:
   binding  -- ctypes access to the C-ABI library (loads it on first use; fails loudly if absent)
   build    -- compiles the CUDA sources for sm_100a
   synth    -- seeded synthetic workloads (no optimizer arithmetic)
+  dist     -- host-side helpers for several ranks (sharding, rank-ordered norm exchange)
 """
 
-__all__ = ["binding", "build", "synth"]
+__all__ = ["binding", "build", "dist", "synth"]
