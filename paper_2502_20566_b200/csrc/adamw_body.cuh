@@ -19,6 +19,38 @@ __device__ __forceinline__ void st16(void* base, uint64_t vec, uint4 val) {
     __stcs(reinterpret_cast<uint4*>(base) + vec, val);
 }
 
+// ---- asynchronous global -> shared copies (16 bytes, L2 only) ---------------------------------
+// Used to keep a thread's NEXT vector in flight while it computes the current one without
+// spending registers on it.  Each thread copies into and reads from its own shared-memory slots,
+// so no block-level synchronisation is involved; completion is tracked per thread by the
+// hardware's copy groups (commit / wait), not by polling.
+__device__ __forceinline__ void async_copy16(uint4* smem_dst, const void* gmem_src) {
+    const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void async_copy_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// returns once at most PENDING of this thread's committed groups are still in flight
+template <int PENDING>
+__device__ __forceinline__ void async_copy_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
+
+constexpr int kStages = 2;   // vectors per thread in flight or in use (measured: 2 beats 3 and 4)
+
+// unpack a staged gradient vector (one 16-byte piece for BF16, two for FP32)
+template <bool G32>
+__device__ __forceinline__ void unpack_grad8(const uint4 g0, const uint4 g1, float (&ge)[8]) {
+    if (G32) {
+        ge[0] = __uint_as_float(g0.x); ge[1] = __uint_as_float(g0.y);
+        ge[2] = __uint_as_float(g0.z); ge[3] = __uint_as_float(g0.w);
+        ge[4] = __uint_as_float(g1.x); ge[5] = __uint_as_float(g1.y);
+        ge[6] = __uint_as_float(g1.z); ge[7] = __uint_as_float(g1.w);
+    } else {
+        ge[0] = bf16_lo(g0.x); ge[1] = bf16_hi(g0.x);
+        ge[2] = bf16_lo(g0.y); ge[3] = bf16_hi(g0.y);
+        ge[4] = bf16_lo(g0.z); ge[5] = bf16_hi(g0.z);
+        ge[6] = bf16_lo(g0.w); ge[7] = bf16_hi(g0.w);
+    }
+}
+
 // the eight gradient values of a vector as FP32
 template <bool G32>
 __device__ __forceinline__ void load_grad8(const void* g, uint64_t vec, float (&ge)[8]) {
@@ -95,12 +127,10 @@ __device__ __noinline__ void step_vec8_reference(uint16_t* p, const void* g, uin
 // segment or a chunk, which lets the compiler hoist the round-1/round-2 products that depend only
 // on c1, c2 and the keys).
 template <bool G32, uint32_t FLAGS, bool SCALE>
-__device__ __forceinline__ void step_vec8_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t vec,
-                                               uint64_t idx0, uint32_t c1, uint32_t c2, uint32_t c3, float gscale,
-                                               const PhiloxKeys& K, const StepScalars& S) {
-    const uint4 pv = ld16(p, vec), mv = ld16(m, vec), vv = ld16(v, vec);
-    float ge[8];
-    load_grad8<G32>(g, vec, ge);
+__device__ __forceinline__ void step_vec8_fast_loaded(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t vec,
+                                                      uint64_t idx0, const uint4 pv, const uint4 mv, const uint4 vv,
+                                                      const float (&ge)[8], uint32_t c1, uint32_t c2, uint32_t c3,
+                                                      float gscale, const PhiloxKeys& K, const StepScalars& S) {
     const uint32_t c0 = static_cast<uint32_t>(idx0 >> 1);
     uint4 wx = make_uint4(0, 0, 0, 0), wm = wx, wv = wx;
     if (FLAGS & 1u) wx = philox4x32_10(c0, c1, c2, c3, K);
@@ -130,6 +160,17 @@ __device__ __forceinline__ void step_vec8_fast(uint16_t* p, const void* g, uint1
     st16(p, vec, make_uint4(po[0], po[1], po[2], po[3]));
     st16(m, vec, make_uint4(mo[0], mo[1], mo[2], mo[3]));
     st16(v, vec, make_uint4(vo[0], vo[1], vo[2], vo[3]));
+}
+
+// the same, loading the vector straight into registers
+template <bool G32, uint32_t FLAGS, bool SCALE>
+__device__ __forceinline__ void step_vec8_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t vec,
+                                               uint64_t idx0, uint32_t c1, uint32_t c2, uint32_t c3, float gscale,
+                                               const PhiloxKeys& K, const StepScalars& S) {
+    const uint4 pv = ld16(p, vec), mv = ld16(m, vec), vv = ld16(v, vec);
+    float ge[8];
+    load_grad8<G32>(g, vec, ge);
+    step_vec8_fast_loaded<G32, FLAGS, SCALE>(p, g, m, v, vec, idx0, pv, mv, vv, ge, c1, c2, c3, gscale, K, S);
 }
 
 // ---- one element with 2-byte accesses: ragged tails, unaligned buffers ---------------------

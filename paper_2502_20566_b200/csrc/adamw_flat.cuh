@@ -7,13 +7,10 @@ namespace sradamw {
 
 // MODE 0: element-wise (any alignment, any offset)
 //      1: 16-byte vectors, reference arithmetic, per-element noise (elem_offset not a multiple of 8)
-//      2: 16-byte vectors, branch-free arithmetic, gradient used as is
-//      3: 16-byte vectors, branch-free arithmetic, gradient multiplied by gscale
 // Persistent grid: thread t takes vectors t, t + T, t + 2T, ... (T = threads in the grid).
-// For modes 2 and 3 every index of the launch has the same (index >> 33) = c1.
 template <bool G32, uint32_t FLAGS, int MODE>
 __global__ void __launch_bounds__(kBlockThreads, kMinBlocksPerSM)
-k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset, uint32_t c1,
+k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset,
                 uint32_t tensor_id, uint32_t seed_hi, const __grid_constant__ PhiloxKeys K,
                 const __grid_constant__ StepScalars S) {
     const float gscale = S.gscale_dev ? __ldg(S.gscale_dev) : S.gscale;
@@ -25,27 +22,95 @@ k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n
         return;
     }
     const uint64_t nvec = n >> 3;
-    for (uint64_t vec = tid; vec < nvec; vec += stride) {
-        const uint64_t idx0 = elem_offset + (vec << 3);
-        if (MODE == 1)
-            step_vec8_reference<G32, FLAGS, false>(p, g, m, v, vec, idx0, tensor_id, seed_hi, gscale, K, S);
-        else
-            step_vec8_fast<G32, FLAGS, MODE == 3>(p, g, m, v, vec, idx0, c1, tensor_id, seed_hi, gscale, K, S);
+    for (uint64_t vec = tid; vec < nvec; vec += stride)
+        step_vec8_reference<G32, FLAGS, false>(p, g, m, v, vec, elem_offset + (vec << 3), tensor_id, seed_hi, gscale, K, S);
+    const uint64_t done = nvec << 3;
+    if (tid < n - done)
+        step_scalar<G32, FLAGS>(p, g, m, v, done + tid, elem_offset + done + tid, tensor_id, seed_hi, gscale, K, S);
+}
+
+// The hot kernel (modes 2 and 3 of the launcher): 16-byte vectors, branch-free arithmetic, gradient
+// used as is (SCALE = false) or multiplied by gscale.  elem_offset is a multiple of 8 and every
+// index of the launch has the same (index >> 33) = c1.  Same persistent grid.  STAGED = true: each
+// thread keeps its next vector in flight -- while vector k is computed out of shared memory, the
+// asynchronous copies of vector k + T are already under way (kStages slots per thread and array).
+// STAGED = false loads straight into registers.
+template <bool G32, uint32_t FLAGS, bool SCALE, bool STAGED>
+__global__ void __launch_bounds__(kBlockThreads, kMinBlocksPerSM)
+k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset,
+                     uint32_t c1, uint32_t tensor_id, uint32_t seed_hi, const __grid_constant__ PhiloxKeys K,
+                     const __grid_constant__ StepScalars S) {
+    constexpr int kArrays = G32 ? 5 : 4;   // x, m, v and one or two 16-byte pieces of g
+    __shared__ uint4 stage[STAGED ? kStages * kArrays * kBlockThreads : 1];
+    const float gscale = S.gscale_dev ? __ldg(S.gscale_dev) : S.gscale;
+    const uint64_t tid = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
+    const uint64_t nvec = n >> 3;
+    if (STAGED) {
+        uint4* const mine = stage + threadIdx.x;
+        auto slot = [&](int s, int a) -> uint4* { return mine + (s * kArrays + a) * kBlockThreads; };
+        auto issue = [&](uint64_t vec, int s) {
+            if (vec < nvec) {
+                async_copy16(slot(s, 0), reinterpret_cast<const uint4*>(p) + vec);
+                async_copy16(slot(s, 1), reinterpret_cast<const uint4*>(m) + vec);
+                async_copy16(slot(s, 2), reinterpret_cast<const uint4*>(v) + vec);
+                if (G32) {
+                    async_copy16(slot(s, 3), reinterpret_cast<const uint4*>(g) + 2 * vec);
+                    async_copy16(slot(s, 4), reinterpret_cast<const uint4*>(g) + 2 * vec + 1);
+                } else {
+                    async_copy16(slot(s, 3), reinterpret_cast<const uint4*>(g) + vec);
+                }
+            }
+            async_copy_commit();   // one group per iteration, empty past the end: the wait count stays uniform
+        };
+#pragma unroll
+        for (int s = 0; s < kStages - 1; ++s) issue(tid + s * stride, s);
+        int s = 0;
+        for (uint64_t vec = tid; vec < nvec; vec += stride) {
+            int ahead = s + kStages - 1;
+            if (ahead >= kStages) ahead -= kStages;
+            issue(vec + (kStages - 1) * stride, ahead);
+            async_copy_wait<kStages - 1>();   // this vector's group has landed
+            const uint4 pv = *slot(s, 0), mv = *slot(s, 1), vv = *slot(s, 2);
+            float ge[8];
+            unpack_grad8<G32>(*slot(s, 3), G32 ? *slot(s, kArrays - 1) : make_uint4(0, 0, 0, 0), ge);
+            step_vec8_fast_loaded<G32, FLAGS, SCALE>(p, g, m, v, vec, elem_offset + (vec << 3), pv, mv, vv, ge, c1,
+                                                     tensor_id, seed_hi, gscale, K, S);
+            if (++s == kStages) s = 0;
+        }
+        async_copy_wait<0>();
+    } else {
+        for (uint64_t vec = tid; vec < nvec; vec += stride)
+            step_vec8_fast<G32, FLAGS, SCALE>(p, g, m, v, vec, elem_offset + (vec << 3), c1, tensor_id, seed_hi, gscale, K, S);
     }
     const uint64_t done = nvec << 3;
     if (tid < n - done)
         step_scalar<G32, FLAGS>(p, g, m, v, done + tid, elem_offset + done + tid, tensor_id, seed_hi, gscale, K, S);
 }
 
+// which gradient types use the staged variant (compile-time switch for measurements)
+#ifndef SR_STAGE_BF16
+#define SR_STAGE_BF16 1
+#endif
+#ifndef SR_STAGE_F32
+#define SR_STAGE_F32 1
+#endif
+
 template <bool G32, uint32_t FLAGS, int MODE>
 cudaError_t launch_flat_mode(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset,
                              uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K, const StepScalars& S,
                              const DeviceInfo& dev, cudaStream_t stream) {
-    auto k = k_sr_adamw_flat<G32, FLAGS, MODE>;
     const uint64_t items = MODE == 0 ? n : (n >> 3) + 8;   // + 8: enough threads for the ragged tail
-    k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset,
-                                                             static_cast<uint32_t>(elem_offset >> 33), tensor_id,
-                                                             seed_hi, K, S);
+    if (MODE >= 2) {
+        constexpr bool kStaged = G32 ? (SR_STAGE_F32 != 0) : (SR_STAGE_BF16 != 0);
+        auto k = k_sr_adamw_flat_fast<G32, FLAGS, MODE == 3, kStaged>;
+        k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset,
+                                                                 static_cast<uint32_t>(elem_offset >> 33), tensor_id,
+                                                                 seed_hi, K, S);
+    } else {
+        auto k = k_sr_adamw_flat<G32, FLAGS, (MODE < 2 ? MODE : 0)>;
+        k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset, tensor_id, seed_hi, K, S);
+    }
     return cudaGetLastError();
 }
 
