@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0       # used only when MEASURED_PEAKS.json is absent
 # the 2^27-element case (profiles/k_sr_adamw_flat__bf16_grads_sr_xmv__2pow27.md); traffic of a streaming
 # kernel grows in proportion to the element count, so the full-size figure is this times n.  Set to
 # None whenever the kernel changes until a new capture exists.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = (1.073966e9 + 0.748455424e9) / (1 << 27)
+NCU_TRAFFIC_BYTES_PER_ELEMENT = None
 
 
 def parse_args():
@@ -247,6 +247,11 @@ def time_extras(torch, binding, synth, dev, peak):
                                     "gbs": 14 * ne / t_mt / 1e6, "frac": 14 * ne / t_mt / 1e6 / peak}
     plan.destroy()
     del P, G, M, V
+    # the flat kernel on a buffer of the same length, for comparison with the list launch
+    fp, fg, fm, fv = synth.adamw_state(ne, SEED, dev)
+    t_f = timed(lambda: binding.sr_adamw_step(fp, fg, fm, fv, hp, SEED, FIRST_STEP))
+    out["flat_same_length_as_list"] = {"elements": ne, "ms": t_f, "gbs": 14 * ne / t_f / 1e6, "frac": 14 * ne / t_f / 1e6 / peak}
+    del fp, fg, fm, fv
     # standalone stochastic-rounding cast, 2^28 FP32 values (6 B per element)
     nc = 1 << 28
     src = synth.downcast_mix(nc, 7, dev)

@@ -88,12 +88,14 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
         step_scalar<G32, FLAGS>(p, g, m, v, done + tid, elem_offset + done + tid, tensor_id, seed_hi, gscale, K, S);
 }
 
-// which gradient types use the staged variant (compile-time switch for measurements)
+// Which gradient types use the staged variant.  Measured on B200 (same GPU, back to back): BF16
+// gradients 85.3% staged vs 83.8% direct of the copy peak at 6.7B; FP32 gradients (five 16-byte
+// pieces per vector) 77.7% staged vs 93.2% direct at 832M elements, so they stay direct.
 #ifndef SR_STAGE_BF16
 #define SR_STAGE_BF16 1
 #endif
 #ifndef SR_STAGE_F32
-#define SR_STAGE_F32 1
+#define SR_STAGE_F32 0
 #endif
 
 template <bool G32, uint32_t FLAGS, int MODE>
