@@ -34,10 +34,10 @@ FIRST_STEP = 1000
 BYTES_PER_ELEMENT = 14          # read x, g, m, v (4 x 2 B) + write x, m, v (3 x 2 B)
 FALLBACK_HBM_GBS = 6650.0       # used only when MEASURED_PEAKS.json is absent
 # (dram__bytes_read.sum + dram__bytes_write.sum) / elements from the ncu capture of the current kernel on
-# the 2^27-element case (profiles/k_sr_adamw_flat__bf16_grads_sr_xmv__2pow27.md); traffic of a streaming
+# the 2^27-element case (profiles/k_sr_adamw_flat_fast__bf16_grads_sr_xmv__2pow27.md); traffic of a streaming
 # kernel grows in proportion to the element count, so the full-size figure is this times n.  Set to
 # None whenever the kernel changes until a new capture exists.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = None
+NCU_TRAFFIC_BYTES_PER_ELEMENT = (1.073771e9 + 0.747271168e9) / (1 << 27)
 
 
 def parse_args():
@@ -384,7 +384,7 @@ def run_ours(args):
         "hbm_gbs": achieved,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": (NCU_TRAFFIC_BYTES_PER_ELEMENT * n if NCU_TRAFFIC_BYTES_PER_ELEMENT else None),
-                     "peak_source": peak_src, "kernel": "k_sr_adamw_flat", "launch_ms_avg": avg_launch_ms,
+                     "peak_source": peak_src, "kernel": "k_sr_adamw_flat_fast", "launch_ms_avg": avg_launch_ms,
                      "launch_ms_min": min(launch_ms), "launch_ms_median": statistics.median(launch_ms),
                      "algorithmic_bytes_per_launch": BYTES_PER_ELEMENT * n},
         "gpu_launches": args.steps,
