@@ -237,7 +237,7 @@ cudaError_t launch_adamw_flat_g(uint16_t* p, const void* g, uint16_t* m, uint16_
                                 uint32_t tensor_id, uint32_t seed_hi, uint32_t flags, const PhiloxKeys& K,
                                 const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream);
 template <bool G32>
-cudaError_t launch_adamw_mt_g(const MtTensor* tensors, const MtChunk* chunks, uint32_t num_chunks,
+cudaError_t launch_adamw_mt_g(const MtWork* work, uint32_t num_chunks,
                               uint32_t tensor_id_base, uint32_t seed_hi, uint32_t flags, const PhiloxKeys& K,
                               const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream);
 

@@ -11,11 +11,11 @@ cudaError_t launch_adamw_flat(uint16_t* p, const void* g, bool g_f32, uint16_t* 
                  : launch_adamw_flat_g<false>(p, g, m, v, n, elem_offset, tensor_id, seed_hi, flags, K, S, dev, stream);
 }
 
-cudaError_t launch_adamw_mt(const MtTensor* tensors, const MtChunk* chunks, uint32_t num_chunks, bool g_f32,
+cudaError_t launch_adamw_mt(const MtWork* work, uint32_t num_chunks, bool g_f32,
                             uint32_t tensor_id_base, uint32_t seed_hi, uint32_t flags, const PhiloxKeys& K,
                             const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream) {
-    return g_f32 ? launch_adamw_mt_g<true>(tensors, chunks, num_chunks, tensor_id_base, seed_hi, flags, K, S, dev, stream)
-                 : launch_adamw_mt_g<false>(tensors, chunks, num_chunks, tensor_id_base, seed_hi, flags, K, S, dev, stream);
+    return g_f32 ? launch_adamw_mt_g<true>(work, num_chunks, tensor_id_base, seed_hi, flags, K, S, dev, stream)
+                 : launch_adamw_mt_g<false>(work, num_chunks, tensor_id_base, seed_hi, flags, K, S, dev, stream);
 }
 
 // ---- standalone Q_SR cast ------------------------------------------------------------------

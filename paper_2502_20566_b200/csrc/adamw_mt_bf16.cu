@@ -2,6 +2,6 @@
 #include "adamw_mt.cuh"
 
 namespace sradamw {
-template cudaError_t launch_adamw_mt_g<false>(const MtTensor*, const MtChunk*, uint32_t, uint32_t, uint32_t, uint32_t,
+template cudaError_t launch_adamw_mt_g<false>(const MtWork*, uint32_t, uint32_t, uint32_t, uint32_t,
                                             const PhiloxKeys&, const StepScalars&, const DeviceInfo&, cudaStream_t);
 }  // namespace sradamw

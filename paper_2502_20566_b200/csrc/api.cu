@@ -101,8 +101,7 @@ sr_status make_scalars(const sr_adamw_hparams* hp, uint32_t step, StepScalars* S
 }  // namespace
 
 struct sr_mt_plan {
-    MtTensor* d_tensors = nullptr;
-    MtChunk* d_chunks = nullptr;
+    MtWork* d_work = nullptr;
     uint32_t num_tensors = 0;
     uint32_t num_chunks = 0;
     uint64_t total_elements = 0;
@@ -238,18 +237,24 @@ sr_status sr_mt_plan_create(sr_mt_plan** out, uint32_t num_tensors, uint16_t* co
     sr_status st = current_device(&dev);
     if (st != SR_OK) return st;
 
-    std::vector<MtTensor> tensors(num_tensors);
-    std::vector<MtChunk> chunks;
+    if (num_tensors > 0x7FFFFFFFu) return SR_ERR_INVALID_ARG;
+    const size_t gsz = g_dtype == SR_DT_F32 ? 4 : 2;
+    std::vector<MtWork> chunks;
     uint64_t total = 0;
     for (uint32_t i = 0; i < num_tensors; ++i) {
         if (numel[i] != 0 && (p[i] == nullptr || g[i] == nullptr || m[i] == nullptr || v[i] == nullptr))
             return SR_ERR_INVALID_ARG;
         const uint64_t nchunks = (numel[i] + kMtChunkElems - 1) / kMtChunkElems;
-        if (nchunks > 0xFFFFFFFFull || chunks.size() + nchunks > 0xFFFFFFFFull) return SR_ERR_INVALID_ARG;
+        if (chunks.size() + nchunks > 0xFFFFFFFFull) return SR_ERR_INVALID_ARG;
         const uintptr_t bits = reinterpret_cast<uintptr_t>(p[i]) | reinterpret_cast<uintptr_t>(g[i]) |
                                reinterpret_cast<uintptr_t>(m[i]) | reinterpret_cast<uintptr_t>(v[i]);
-        tensors[i] = MtTensor{p[i], g[i], m[i], v[i], numel[i], (bits & 15u) == 0 ? 1u : 0u, 0u};
-        for (uint64_t c = 0; c < nchunks; ++c) chunks.push_back(MtChunk{i, static_cast<uint32_t>(c)});
+        const uint32_t tensor_vec = i | ((bits & 15u) == 0 ? 0x80000000u : 0u);
+        for (uint64_t c = 0; c < nchunks; ++c) {
+            const uint64_t start = c * kMtChunkElems;
+            const uint64_t left = numel[i] - start;
+            chunks.push_back(MtWork{p[i] + start, static_cast<const char*>(g[i]) + start * gsz, m[i] + start, v[i] + start,
+                                    start, static_cast<uint32_t>(left < kMtChunkElems ? left : kMtChunkElems), tensor_vec});
+        }
         total += numel[i];
     }
 
@@ -263,18 +268,14 @@ sr_status sr_mt_plan_create(sr_mt_plan** out, uint32_t num_tensors, uint16_t* co
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaSuccess;
     if (!chunks.empty()) {
-        e = cudaMalloc(&plan->d_tensors, tensors.size() * sizeof(MtTensor));
-        if (e == cudaSuccess) e = cudaMalloc(&plan->d_chunks, chunks.size() * sizeof(MtChunk));
+        e = cudaMalloc(&plan->d_work, chunks.size() * sizeof(MtWork));
         if (e == cudaSuccess)
-            e = cudaMemcpyAsync(plan->d_tensors, tensors.data(), tensors.size() * sizeof(MtTensor), cudaMemcpyHostToDevice, s);
-        if (e == cudaSuccess)
-            e = cudaMemcpyAsync(plan->d_chunks, chunks.data(), chunks.size() * sizeof(MtChunk), cudaMemcpyHostToDevice, s);
+            e = cudaMemcpyAsync(plan->d_work, chunks.data(), chunks.size() * sizeof(MtWork), cudaMemcpyHostToDevice, s);
         // the host vectors die at return: wait for the copies (plan creation is not a hot call)
         if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     }
     if (e != cudaSuccess) {
-        cudaFree(plan->d_tensors);
-        cudaFree(plan->d_chunks);
+        cudaFree(plan->d_work);
         delete plan;
         return cuda_fail(e);
     }
@@ -293,7 +294,7 @@ sr_status sr_adamw_multi_tensor(const sr_mt_plan* plan, const sr_adamw_hparams* 
     st = current_device(&dev);
     if (st != SR_OK) return st;
     const cudaError_t e =
-        launch_adamw_mt(plan->d_tensors, plan->d_chunks, plan->num_chunks, plan->g_f32, tensor_id_base,
+        launch_adamw_mt(plan->d_work, plan->num_chunks, plan->g_f32, tensor_id_base,
                         static_cast<uint32_t>(seed >> 32), hp->flags, make_keys(seed, step), S, dev,
                         static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? SR_OK : cuda_fail(e);
@@ -301,11 +302,9 @@ sr_status sr_adamw_multi_tensor(const sr_mt_plan* plan, const sr_adamw_hparams* 
 
 sr_status sr_mt_plan_destroy(sr_mt_plan* plan) {
     if (plan == nullptr) return SR_OK;
-    cudaError_t e1 = cudaFree(plan->d_tensors);
-    cudaError_t e2 = cudaFree(plan->d_chunks);
+    cudaError_t e1 = cudaFree(plan->d_work);
     delete plan;
     if (e1 != cudaSuccess) return cuda_fail(e1);
-    if (e2 != cudaSuccess) return cuda_fail(e2);
     return SR_OK;
 }
 

@@ -8,23 +8,21 @@
 
 namespace sradamw {
 
-// Device-side tables of a multi-tensor plan.
-struct MtTensor {
+// Device-side work table of a multi-tensor plan: one entry per chunk (up to kMtChunkElems consecutive
+// elements of one tensor) with the four pointers already advanced to the chunk's first element, so a
+// block needs a single 48-byte read per chunk and can fetch the next entry while it works.
+struct MtWork {
     uint16_t* p;
     const void* g;
     uint16_t* m;
     uint16_t* v;
-    uint64_t n;
-    uint32_t vec_ok;   // all four pointers 16-byte aligned
-    uint32_t pad;
+    uint64_t idx0;        // index of the chunk's first element inside its tensor (multiple of kMtChunkElems)
+    uint32_t len;         // elements in this chunk
+    uint32_t tensor_vec;  // tensor index (bits 0..30) | bit 31: all four tensor buffers are 16-byte aligned
 };
+static_assert(sizeof(MtWork) == 48, "three 16-byte loads per entry");
 
-struct MtChunk {
-    uint32_t tensor;   // index into the tensor table
-    uint32_t chunk;    // chunk number inside that tensor; first element = chunk * kMtChunkElems
-};
-
-constexpr uint32_t kMtChunkElems = 16384;   // multiple of 8 * block size
+constexpr uint32_t kMtChunkElems = 8192;   // multiple of 8; never crosses a multiple of 2^33
 #ifndef SR_BLOCK_THREADS
 #define SR_BLOCK_THREADS 128
 #endif
@@ -50,7 +48,7 @@ cudaError_t launch_adamw_flat(uint16_t* p, const void* g, bool g_f32, uint16_t* 
                               uint64_t elem_offset, uint32_t tensor_id, uint32_t seed_hi, uint32_t flags,
                               const PhiloxKeys& K, const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream);
 
-cudaError_t launch_adamw_mt(const MtTensor* tensors, const MtChunk* chunks, uint32_t num_chunks, bool g_f32,
+cudaError_t launch_adamw_mt(const MtWork* work, uint32_t num_chunks, bool g_f32,
                             uint32_t tensor_id_base, uint32_t seed_hi, uint32_t flags, const PhiloxKeys& K,
                             const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream);
 
