@@ -357,6 +357,40 @@ def test_multi_tensor_small_list_with_odd_shapes(env):
     _run_list(env, specs, steps=2, shift=1)      # every third tensor starts 2 bytes off alignment
 
 
+@pytest.mark.parametrize("g_dtype,flags,gscale", [(torch.bfloat16, 7, 1.0), (torch.bfloat16, 1, 0.5), (torch.float32, 7, 1.0),
+                                                 (torch.float32, 0, 0.125)])
+def test_multi_tensor_random_lists(env, g_dtype, flags, gscale):
+    """Lists of many tensors whose sizes straddle every boundary of the kernel: fewer vectors than a
+    block has threads, one more than that, whole chunks, a chunk plus one element, runs of tiny tensors
+    (threads that skip several chunks in a row), empty tensors, and a few unaligned ones."""
+    oracle, binding, synth, dev = env
+    rng = np.random.default_rng(int(flags) * 7 + (g_dtype == torch.float32))
+    sizes = [1, 3, 8, 8 * 127, 8 * 128, 8 * 128 + 1, 8 * 129, 8191, 8192, 8193, 2 * 8192, 2 * 8192 + 7, 0, 5, 5, 5, 5, 5, 5, 16, 24,
+             3 * 8192 + 8 * 64, 40, 100000] + [int(x) for x in rng.integers(1, 30000, 40)] + [int(x) for x in rng.integers(1, 64, 30)]
+    order = rng.permutation(len(sizes))
+    sizes = [sizes[i] for i in order]
+    P, G, M, V = [], [], [], []
+    for i, n in enumerate(sizes):
+        shift = 1 if i % 11 == 3 else 0                 # some tensors start 2 bytes off a 16-byte boundary
+        p, g, m, v = synth.adamw_state(n + shift, 900 + i, dev, g_dtype=g_dtype)
+        P.append(p[shift:]); G.append(g[shift:]); M.append(m[shift:]); V.append(v[shift:])
+    plan = binding.sr_mt_plan_create(P, G, M, V)
+    assert plan.total_elements == sum(sizes)
+    hp_o = oracle.hparams(**HP, flags=flags)
+    hp_g = binding.hparams(**HP, grad_scale=gscale, flags=flags)
+    host = [[bits(t) for t in P], [host_g(t) for t in G], [bits(t) for t in M], [bits(t) for t in V]]
+    for step in (1, 2):
+        binding.sr_adamw_multi_tensor(plan, hp_g, 99, step, tensor_id_base=1000)
+        torch.cuda.synchronize()
+        bad = 0
+        for i in range(len(sizes)):
+            oracle.adamw_step(host[0][i], host[1][i], host[2][i], host[3][i], hp_o, 99, step, 1000 + i, 0, gscale)
+            bad += mismatches(bits(P[i]), host[0][i]) + mismatches(bits(M[i]), host[2][i]) + mismatches(bits(V[i]), host[3][i])
+            assert np.array_equal(host_g(G[i]), host[1][i])
+        assert bad == 0, f"step {step}"
+    plan.destroy()
+
+
 def test_multi_tensor_gpt2_350m_ten_steps(env):
     """GPT-2 350M parameter list (292 tensors, 354 823 168 elements), 10 iterations with fresh
     gradients, zero mismatches after every iteration."""
