@@ -82,6 +82,9 @@ def lib() -> ctypes.CDLL:
         L.oracle_adamw_step.argtypes = [c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_uint64,
                                         POINTER(HParams), c_float, c_uint64, c_uint32, c_uint32, c_uint64]
         L.oracle_adamw_step.restype = c_int
+        L.oracle_master_adamw_step.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_uint64,
+                                               POINTER(HParams), c_float, c_uint32]
+        L.oracle_master_adamw_step.restype = c_int
         L.oracle_sr_downcast.argtypes = [c_void_p, c_void_p, c_uint64, c_uint64, c_uint32, c_uint32, c_uint64]
         L.oracle_sqnorm.argtypes = [c_void_p, c_int, c_uint64]
         L.oracle_sqnorm.restype = c_double
@@ -161,6 +164,24 @@ def adamw_step(p, g, m, v, hp: HParams, seed, step, tensor_id=0, elem_offset=0, 
                                  gscale, seed, step, tensor_id, elem_offset)
     if rc != 0:
         raise ValueError("AdamW is not defined for step 0")
+
+
+def master_adamw_step(p, g, m, v, hp: HParams, step, gscale=1.0):
+    """FP32 master recipe, in place on float32 arrays p, m, v; g is uint16 (BF16 bits) or float32.
+    Returns the BF16 copy of the updated parameters (uint16 bit patterns)."""
+    _check(p, np.float32), _check(m, np.float32), _check(v, np.float32)
+    g_is_f32 = 1 if g.dtype == np.float32 else 0
+    if not g_is_f32:
+        _check(g, np.uint16)
+    n = p.size
+    if not (g.size == m.size == v.size == n):
+        raise ValueError("size mismatch")
+    p16 = np.empty(p.shape, dtype=np.uint16)
+    rc = lib().oracle_master_adamw_step(_ptr(p), _ptr(p16), _ptr(g), g_is_f32, _ptr(m), _ptr(v), n, ctypes.byref(hp),
+                                        gscale, step)
+    if rc != 0:
+        raise ValueError("AdamW is not defined for step 0")
+    return p16
 
 
 def sr_downcast(src, seed, step=0, tensor_id=0, elem_offset=0):

@@ -280,6 +280,29 @@ int oracle_adamw_step(uint16_t* p, const void* g, int g_is_f32, uint16_t* m, uin
     return 0;
 }
 
+// The mixed-precision comparison recipe the paper measures against (its "O2": FP32 master weights
+// and FP32 optimizer states, a BF16 copy of the weights for the forward/backward pass): the same
+// element function, results kept in FP32 without any rounding, plus x rounded to nearest (Eq. 1)
+// into the BF16 copy.  No random state is involved.
+int oracle_master_adamw_step(float* p, uint16_t* p_bf16, const void* g, int g_is_f32, float* m, float* v, uint64_t n,
+                             const oracle_hparams* hp, float gscale, uint32_t step) {
+    oracle_scalars sc;
+    if (oracle_adamw_scalars(hp, step, &sc) != 0) return 1;
+    const uint16_t* g16 = static_cast<const uint16_t*>(g);
+    const float* g32 = static_cast<const float*>(g);
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < static_cast<int64_t>(n); ++i) {
+        const float gi = g_is_f32 ? g32[i] : bf16_to_float(g16[i]);
+        oracle_trace t;
+        oracle_adamw_element(p[i], gi, m[i], v[i], gscale, &sc, &t);
+        p[i] = t.x_new;
+        m[i] = t.m_new;
+        v[i] = t.v_new;
+        p_bf16[i] = rne_bf16_bits(bits_of(t.x_new));
+    }
+    return 0;
+}
+
 // Q_SR on an FP32 array; uses rounding slot 0 (the x slot) of the noise.
 void oracle_sr_downcast(const float* src, uint16_t* dst, uint64_t n, uint64_t seed, uint32_t step,
                         uint32_t tensor_id, uint64_t elem_offset) {

@@ -314,6 +314,46 @@ def is_nan_bits_array(b):
     return (b & 0x7FFFFFFF) > 0x7F800000
 
 
+def test_master_recipe_tracks_library_adamw_over_several_steps():
+    """FP32-master recipe (the paper's mixed-precision comparison): eight consecutive steps stay within
+    FP32 rounding of torch.optim.AdamW, and the BF16 copy is the nearest-rounded parameter."""
+    n = 4096
+    p0, _, _, _ = synth.adamw_state(n, 61, "cpu")
+    p = p0.float().numpy().copy()
+    m = np.zeros(n, dtype=np.float32)
+    v = np.zeros(n, dtype=np.float32)
+    param = torch.nn.Parameter(torch.from_numpy(p.copy()))
+    opt = torch.optim.AdamW([param], lr=HP["lr"], betas=(HP["beta1"], HP["beta2"]), eps=HP["eps"],
+                            weight_decay=HP["weight_decay"])
+    hp = oracle.hparams(**HP)
+    for step in range(1, 9):
+        g = synth.state_chunk(synth.ROLE_G, 600 + step, 0, n, "cpu", g_dtype=torch.float32)
+        param.grad = g.clone()
+        opt.step()
+        p16 = oracle.master_adamw_step(p, g.numpy().copy(), m, v, hp, step)
+        np.testing.assert_allclose(p, param.detach().numpy(), rtol=2e-6, atol=2e-8)
+        want16 = torch.from_numpy(p.copy()).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+        assert np.array_equal(p16, want16)
+    st = opt.state[param]
+    np.testing.assert_allclose(m, st["exp_avg"].numpy(), rtol=2e-5, atol=1e-9)
+    np.testing.assert_allclose(v, st["exp_avg_sq"].numpy(), rtol=2e-5, atol=1e-13)
+
+
+def test_master_recipe_is_the_element_function():
+    n = 333
+    p0, g, m0, v0 = synth.adamw_state(n, 62, "cpu")
+    p, m, v = (t.float().numpy().copy() for t in (p0, m0, v0))
+    before = (p.copy(), m.copy(), v.copy())
+    hp = oracle.hparams(**HP)
+    sc = oracle.adamw_scalars(hp, 5)
+    gb = synth.bits16(g).copy()
+    p16 = oracle.master_adamw_step(p, gb, m, v, hp, 5, gscale=f32(0.25))
+    for i in range(n):
+        t = oracle.adamw_element(float(before[0][i]), float(g[i]), float(before[1][i]), float(before[2][i]), f32(0.25), sc)
+        assert (p[i], m[i], v[i]) == (t.x_new, t.m_new, t.v_new)
+        assert p16[i] == oracle.rne_bf16_bits(f32_bits(t.x_new))
+
+
 # ---------------------------------------------------------------------------------------------
 # squared norm and clipping
 # ---------------------------------------------------------------------------------------------
