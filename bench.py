@@ -227,7 +227,20 @@ def time_extras(torch, binding, synth, dev, peak):
         "norm_clip_step": {"ms": t_all, "params_per_s": n / t_all * 1e3, "gbs": 20 * n / t_all / 1e6,
                            "frac": 20 * n / t_all / 1e6 / peak},
     }
-    del p, g, m, v, ws
+    del p, m, v, ws
+    # the mixed-precision comparison recipe on the same shard: FP32 master weights and moments + BF16 copy
+    p32, m32, v32 = (torch.empty(n, dtype=torch.float32, device=dev) for _ in range(3))
+    for t, role in ((p32, synth.ROLE_P), (m32, synth.ROLE_M), (v32, synth.ROLE_V)):
+        for c, start, length in synth.chunks(n):
+            t[start:start + length] = synth.state_chunk(role, SEED, c, length, dev).float()
+    p16 = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    hp_plain = binding.hparams(**HP)
+    t_mp = timed(lambda: binding.sr_master_adamw_step(p32, p16, g, m32, v32, hp_plain, FIRST_STEP))
+    out["fp32_master_recipe_same_shard"] = {
+        "elements": n, "bytes_per_element": 30, "ms": t_mp, "params_per_s": n / t_mp * 1e3, "gbs": 30 * n / t_mp / 1e6,
+        "frac": 30 * n / t_mp / 1e6 / peak, "state_bytes_per_param": 14, "sr_state_bytes_per_param": 6,
+        "time_vs_sr_step": t_mp / t_step}
+    del p32, m32, v32, p16, g
     # GPT-2 350M tensor list, one launch per step
     specs = synth.gpt2_param_list()
     P = [synth.init_param(sp, SEED, i, dev) for i, sp in enumerate(specs)]

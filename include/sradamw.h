@@ -87,6 +87,14 @@ sr_status sr_adamw_step(uint16_t* p, const void* g, sr_dtype g_dtype, uint16_t* 
                         const sr_adamw_hparams* hp, uint64_t seed, uint32_t step, uint32_t tensor_id,
                         uint64_t elem_offset, void* stream);
 
+/* The mixed-precision recipe the paper compares against (Section 3: FP32 master weights and FP32
+ * optimizer states, BF16 copy of the weights), provided so that both recipes can be measured with
+ * the same arithmetic on the same GPU.  p, m, v: FP32 in/out; p_bf16: BF16 copy of the updated x,
+ * rounded to nearest (Eq. 1), written only; g: BF16 or FP32.  Same element function as
+ * sr_adamw_step, no noise; hp->flags is ignored.  28 (30) bytes per element instead of 14 (16). */
+sr_status sr_master_adamw_step(float* p, uint16_t* p_bf16, const void* g, sr_dtype g_dtype, float* m, float* v,
+                               uint64_t n, const sr_adamw_hparams* hp, uint32_t step, void* stream);
+
 /* The same iteration for state that lives in HOST memory (optimizer state kept off the device):
  * the buffer is cut into chunks; each chunk is copied host->device into `staging`, stepped by the
  * same kernel as sr_adamw_step (with elem_offset advanced, so the result equals the in-device

@@ -23,7 +23,7 @@ SR_FLAG_SR_P, SR_FLAG_SR_M, SR_FLAG_SR_V = 1, 2, 4
 SR_FLAGS_DEFAULT = 7
 
 EXPORTS = (
-    "sr_downcast_f32_bf16", "sr_adamw_step", "sr_adamw_step_host", "sr_adamw_step_host_staging_bytes",
+    "sr_downcast_f32_bf16", "sr_adamw_step", "sr_master_adamw_step", "sr_adamw_step_host", "sr_adamw_step_host_staging_bytes",
     "sr_mt_plan_create", "sr_adamw_multi_tensor",
     "sr_mt_plan_destroy", "sr_mt_plan_total_elements", "grad_sqnorm_workspace_bytes", "grad_sqnorm",
     "grad_sqnorm_static", "grad_sqnorm_static_max_elements",
@@ -79,6 +79,9 @@ def lib() -> ctypes.CDLL:
         L.sr_adamw_step.argtypes = [c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_uint64, POINTER(HParams),
                                     c_uint64, c_uint32, c_uint32, c_uint64, c_void_p]
         L.sr_adamw_step.restype = c_int
+        L.sr_master_adamw_step.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_uint64,
+                                           POINTER(HParams), c_uint32, c_void_p]
+        L.sr_master_adamw_step.restype = c_int
         L.sr_adamw_step_host_staging_bytes.argtypes = [c_int, c_uint64]
         L.sr_adamw_step_host_staging_bytes.restype = c_size_t
         L.sr_adamw_step_host.argtypes = [c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_uint64, POINTER(HParams),
@@ -155,6 +158,21 @@ def sr_adamw_step(p: torch.Tensor, g: torch.Tensor, m: torch.Tensor, v: torch.Te
         _check(lib().sr_adamw_step(p.data_ptr(), g.data_ptr(), _g_dtype(g), m.data_ptr(), v.data_ptr(), n,
                                    ctypes.byref(hp), seed, step, tensor_id, elem_offset, _stream(stream)),
                "sr_adamw_step")
+
+
+def sr_master_adamw_step(p: torch.Tensor, p_bf16: torch.Tensor, g: torch.Tensor, m: torch.Tensor, v: torch.Tensor,
+                         hp: HParams, step: int, stream=None) -> None:
+    """FP32 master weights / moments (in place) with a nearest-rounded BF16 copy of x: the paper's
+    mixed-precision comparison recipe."""
+    _want(p, torch.float32, "p"), _want(m, torch.float32, "m"), _want(v, torch.float32, "v")
+    _want(p_bf16, torch.bfloat16, "p_bf16"), _want(g, g.dtype, "g")
+    n = p.numel()
+    if not (g.numel() == m.numel() == v.numel() == p_bf16.numel() == n):
+        raise ValueError("size mismatch")
+    with torch.cuda.device(p.device):
+        _check(lib().sr_master_adamw_step(p.data_ptr(), p_bf16.data_ptr(), g.data_ptr(), _g_dtype(g), m.data_ptr(),
+                                          v.data_ptr(), n, ctypes.byref(hp), step, _stream(stream)),
+               "sr_master_adamw_step")
 
 
 def sr_adamw_step_host_staging_bytes(g_dtype: torch.dtype, chunk_elems: int) -> int:

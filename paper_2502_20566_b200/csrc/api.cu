@@ -141,6 +141,22 @@ sr_status sr_adamw_step(uint16_t* p, const void* g, sr_dtype g_dtype, uint16_t* 
     return e == cudaSuccess ? SR_OK : cuda_fail(e);
 }
 
+sr_status sr_master_adamw_step(float* p, uint16_t* p_bf16, const void* g, sr_dtype g_dtype, float* m, float* v,
+                               uint64_t n, const sr_adamw_hparams* hp, uint32_t step, void* stream) {
+    StepScalars S;
+    sr_status st = make_scalars(hp, step, &S);
+    if (st != SR_OK) return st;
+    if (g_dtype != SR_DT_BF16 && g_dtype != SR_DT_F32) return SR_ERR_INVALID_ARG;
+    if (n == 0) return SR_OK;
+    if (p == nullptr || p_bf16 == nullptr || g == nullptr || m == nullptr || v == nullptr) return SR_ERR_INVALID_ARG;
+    DeviceInfo dev;
+    st = current_device(&dev);
+    if (st != SR_OK) return st;
+    const cudaError_t e = launch_master_adamw(p, p_bf16, g, g_dtype == SR_DT_F32, m, v, n, S, dev,
+                                              static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SR_OK : cuda_fail(e);
+}
+
 // ---- host-resident state -------------------------------------------------------------------
 namespace {
 struct HostPipe {

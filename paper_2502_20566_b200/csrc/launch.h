@@ -52,6 +52,9 @@ cudaError_t launch_adamw_mt(const MtWork* work, uint32_t num_chunks, bool g_f32,
                             uint32_t tensor_id_base, uint32_t seed_hi, uint32_t flags, const PhiloxKeys& K,
                             const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream);
 
+cudaError_t launch_master_adamw(float* p, uint16_t* p16, const void* g, bool g_f32, float* m, float* v, uint64_t n,
+                                const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream);
+
 // Squared norm: number of doubles of scratch needed, and the launcher.
 uint64_t sqnorm_scratch_doubles(uint64_t n);
 cudaError_t launch_sqnorm(const void* g, bool g_f32, uint64_t n, double* out, double* scratch,

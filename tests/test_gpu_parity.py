@@ -452,3 +452,36 @@ def test_host_resident_step_equals_oracle(env, g_dtype):
     binding.sr_adamw_step_host(p, g, m, v, binding.hparams(**HP), 31, 5, staging, chunk, tensor_id=2, elem_offset=1000)
     torch.cuda.synchronize()
     assert mismatches(synth.bits16(p), pb) == 0 and mismatches(synth.bits16(m), mb) == 0 and mismatches(synth.bits16(v), vb) == 0
+
+
+# ---------------------------------------------------------------------------------------------
+# FP32-master comparison recipe
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n,shift", [(0, 0), (5, 0), (8 * 4096 + 3, 0), ((1 << 22) + 11, 0), (9001, 1)])
+@pytest.mark.parametrize("g_dtype,gscale", [(torch.bfloat16, 1.0), (torch.float32, 0.125)])
+def test_master_recipe_bit_exact(env, n, shift, g_dtype, gscale):
+    """FP32 master weights and moments + nearest-rounded BF16 copy (the paper's mixed-precision
+    comparison): two consecutive steps, every FP32 word and every BF16 pattern equal to the oracle's."""
+    oracle, binding, synth, dev = env
+    p0, g, m0, v0 = synth.adamw_state(n + shift, 31 + n, dev, g_dtype=g_dtype)
+    p, m, v = (t.float()[shift:] for t in (p0, m0, v0))
+    g = g[shift:]
+    if n > 100:
+        p[7], m[11], v[13], v[17] = float("nan"), float("inf"), 0.0, 1e-30      # vectors that leave the fast range
+    p16 = torch.zeros(n + shift, dtype=torch.bfloat16, device=dev)[shift:]
+    ph, mh, vh = (t.cpu().numpy().copy() for t in (p, m, v))
+    gh = host_g(g)
+    hp_kw = dict(HP)
+    for step in (1, 2):
+        want16 = oracle.master_adamw_step(ph, gh, mh, vh, oracle.hparams(**hp_kw), step, gscale)
+        binding.sr_master_adamw_step(p, p16, g, m, v, binding.hparams(**hp_kw, grad_scale=gscale), step)
+        torch.cuda.synchronize()
+        for dev_t, host_t in ((p, ph), (m, mh), (v, vh)):
+            got = dev_t.cpu().numpy().view(np.uint32)
+            want = host_t.view(np.uint32)
+            nan = (want & 0x7FFFFFFF) > 0x7F800000                      # NaN payloads may differ between platforms
+            assert np.array_equal(got[~nan], want[~nan])
+            assert np.all((got[nan] & 0x7FFFFFFF) > 0x7F800000)
+            host_t[nan] = dev_t.cpu().numpy()[nan]                      # keep both sides on the same NaN bits
+        assert mismatches(bits(p16), want16) == 0
