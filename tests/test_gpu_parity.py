@@ -89,7 +89,8 @@ def test_flat_step_leaves_neighbouring_memory_alone(env):
     assert np.array_equal(bits(bufs[1]), before[1])     # the gradient is read-only
 
 
-@pytest.mark.parametrize("offset", [(1 << 32) - 1024, (1 << 32) - 1021, (1 << 33) + 8, 3 * 832300544, (1 << 40) + 5])
+@pytest.mark.parametrize("offset", [(1 << 32) - 1024, (1 << 32) - 1021, (1 << 33) + 8, (1 << 33) - 2048, (1 << 33) - 2045,
+                                    3 * 832300544, (1 << 40) + 5])
 def test_flat_step_index_offsets_cross_32_bits(env, offset):
     _, _, synth, dev = env
     p, g, m, v = synth.adamw_state(4096 + 3, 8, dev)
@@ -244,6 +245,33 @@ def test_downcast_unbiased_over_4096_seeds(env):
     assert wide.sum() > k // 2
     z = (ups - k * q)[wide] / np.sqrt(var[wide])
     assert np.abs(z).max() < 6.0 and abs(z.mean()) < 0.1 and 0.9 < z.std() < 1.1
+
+
+def test_random_walk_example_on_the_gpu(env):
+    """Section 2.2, first example, run with the library's cast: walkers start on a BF16 level, take two
+    half-level steps and then steps of epsilon levels.  P(T <= 2) = 3/4 and E[T] = 3/2 + 1/(4 eps)."""
+    _, binding, _, dev = env
+    walkers, eps, horizon = 1 << 20, 1.0 / 16.0, 400
+    level, delta = 1.0, 2.0 ** -7                                   # 1.0 and 1 + 2^-7 are consecutive BF16 values
+    x = torch.full((walkers,), level, dtype=torch.float32, device=dev)
+    out = torch.empty(walkers, dtype=torch.bfloat16, device=dev)
+    hit = torch.zeros(walkers, dtype=torch.int32, device=dev)
+    for t in range(1, horizon + 1):
+        u = delta / 2 if t <= 2 else delta * eps
+        binding.sr_downcast_f32_bf16(x + u, out, seed=2024, step=t)
+        x = out.float()
+        hit = torch.where((hit == 0) & (x > level), torch.full_like(hit, t), hit)
+        x = torch.where(hit > 0, torch.full_like(x, level + delta), x)   # absorbed at the upper level
+    assert int((hit == 0).sum()) == 0                               # (15/16)^398 is far below 2^-20
+    p_le_2 = float((hit <= 2).float().mean())
+    assert abs(p_le_2 - 0.75) < 5 * (0.75 * 0.25 / walkers) ** 0.5
+    mean_T = float(hit.double().mean())
+    want = 1.5 + 0.25 / eps
+    var_T = 0.25 * (1 - eps) / eps ** 2 + 5.0                        # generous bound on Var[T]
+    assert abs(mean_T - want) < 5 * (var_T / walkers) ** 0.5
+    for n in (3, 4, 6):
+        p_n = float((hit == n).float().mean())
+        assert abs(p_n - 0.25 * (1 - eps) ** (n - 3) * eps) < 5 * (0.02 / walkers) ** 0.5
 
 
 # ---------------------------------------------------------------------------------------------
