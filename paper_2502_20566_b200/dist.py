@@ -56,3 +56,59 @@ def max_over_ranks(value: float, device, group=None) -> float:
     t = torch.tensor([value], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX, group=group)
     return float(t.item())
+
+
+def sharded_clipped_step(shard_p, shard_m, shard_v, full_grad, hp_kwargs: dict, seed: int, step: int, *, max_norm: float,
+                         accum_scale: float = 1.0, tensor_id: int = 0, group=None, full_param_out=None, ops=None):
+    """One optimizer iteration with the state sharded over the ranks of ``group`` (ZeRO-1 shape):
+
+        reduce-scatter(full_grad) -> grad_sqnorm -> rank-ordered global norm -> sr_clip_scale
+        -> sr_adamw_step on this rank's slice with elem_offset = slice start -> all-gather(x)
+
+    ``shard_p/m/v``: this rank's BF16 slice (length = partition(n)[rank][1]); ``full_grad``: this
+    rank's full-length local gradient (FP32; summed over ranks by the reduce-scatter, the factor
+    1/world belongs in ``accum_scale``); ``full_param_out``: optional full-length BF16 buffer that
+    receives every rank's updated slice.  All slices must have equal length (n divisible by
+    8 * world), which is what the collectives need.  The collectives are torch.distributed calls
+    (NCCL over NVLink on GPUs); every arithmetic step runs in the library's kernels.  ``ops`` lets a
+    test substitute the four kernel calls; by default they are the CUDA binding's.
+    Returns the global squared norm (one float64 tensor, identical on every rank).
+    """
+    world = dist.get_world_size(group)
+    rank = dist.get_rank(group)
+    n = full_grad.numel()
+    if n % (8 * world) != 0:
+        raise ValueError("buffer length must be a multiple of 8 * world size")
+    per = n // world
+    if not (shard_p.numel() == shard_m.numel() == shard_v.numel() == per):
+        raise ValueError("shard length mismatch")
+    if ops is None:
+        from . import binding
+
+        class ops:  # noqa: N801 - namespace of the four kernel calls
+            @staticmethod
+            def sqnorm(g, out):
+                ws = torch.empty(max(1, binding.grad_sqnorm_workspace_bytes(g.numel()) // 8), dtype=torch.float64, device=g.device)
+                binding.grad_sqnorm(g, out, ws)
+
+            @staticmethod
+            def clip_scale(total, accum, mx, out):
+                binding.sr_clip_scale(total, accum, mx, out)
+
+            @staticmethod
+            def step(p, g, m, v, gscale_dev, offset):
+                binding.sr_adamw_step(p, g, m, v, binding.hparams(**hp_kwargs, grad_scale_dev=gscale_dev), seed, step,
+                                      tensor_id, offset)
+
+    dev = full_grad.device
+    shard_g = torch.empty(per, dtype=full_grad.dtype, device=dev)
+    dist.reduce_scatter_tensor(shard_g, full_grad.contiguous(), op=dist.ReduceOp.SUM, group=group)
+    local = torch.zeros(1, dtype=torch.float64, device=dev)
+    ops.sqnorm(shard_g, local)
+    total = global_sqnorm(local, group)
+    gscale = torch.zeros(1, dtype=torch.float32, device=dev)
+    ops.clip_scale(total, accum_scale, max_norm, gscale)
+    ops.step(shard_p, shard_g, shard_m, shard_v, gscale, rank * per)
+    if full_param_out is not None:
+        dist.all_gather_into_tensor(full_param_out, shard_p.contiguous(), group=group)
+    return total

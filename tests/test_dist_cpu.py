@@ -46,6 +46,81 @@ def _worker(rank, world, port, out_dir):
     dist.destroy_process_group()
 
 
+def _sharded_worker(rank, world, port, out_dir):
+    """sharded_clipped_step with the kernel calls replaced by the oracle (CPU tensors, gloo)."""
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import oracle
+    from paper_2502_20566_b200 import synth
+    from paper_2502_20566_b200.dist import sharded_clipped_step
+    n = 8 * world * 1500
+    p, _, m, v = synth.adamw_state(n, 88, "cpu")
+    g_local = synth.state_chunk(synth.ROLE_G, 500 + rank, 0, n, "cpu", g_dtype=torch.float32, outlier_fraction=0.01)
+    per = n // world
+    sl = slice(rank * per, (rank + 1) * per)
+    sp, sm, sv = (t[sl].clone() for t in (p, m, v))
+
+    class ops:
+        @staticmethod
+        def sqnorm(g, out):
+            out[0] = oracle.sqnorm(g.numpy().copy())
+
+        @staticmethod
+        def clip_scale(total, accum, mx, out):
+            out[0] = oracle.clip_scale(float(total.item()), accum, mx)
+
+        @staticmethod
+        def step(pp, gg, mm, vv, gscale_dev, offset):
+            pb, mb, vb = (synth.bits16(t) for t in (pp, mm, vv))       # views: updated in place
+            oracle.adamw_step(pb, gg.numpy().copy(), mb, vb, oracle.hparams(**HP), 1234, 7, 0, offset, float(gscale_dev.item()))
+
+    full = torch.empty(n, dtype=torch.bfloat16)
+    # gloo has no reduce_scatter_tensor / all_gather_into_tensor on every build: fall back to the list forms
+    if not hasattr(dist, "_orig_rs"):
+        def rs(out, inp, op=dist.ReduceOp.SUM, group=None):
+            t = inp.clone()
+            dist.all_reduce(t, op=op, group=group)
+            out.copy_(t[dist.get_rank(group) * out.numel():(dist.get_rank(group) + 1) * out.numel()])
+
+        def ag(out, inp, group=None):
+            parts = [torch.empty_like(inp) for _ in range(dist.get_world_size(group))]
+            dist.all_gather(parts, inp, group=group)
+            out.copy_(torch.cat(parts))
+        dist._orig_rs = dist.reduce_scatter_tensor
+        dist.reduce_scatter_tensor, dist.all_gather_into_tensor = rs, ag
+    total = sharded_clipped_step(sp, sm, sv, g_local, HP, 1234, 7, max_norm=1.0, accum_scale=1.0 / world,
+                                 full_param_out=full, ops=ops)
+    np.savez(os.path.join(out_dir, f"s{rank}.npz"), full=synth.bits16(full), m=synth.bits16(sm), v=synth.bits16(sv),
+             total=total.numpy(), g=g_local.numpy())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_sharded_clipped_step_orchestration(tmp_path):
+    """reduce-scatter -> norm exchange -> clip -> shard step -> all-gather on two gloo ranks equals the
+    single-process computation on the summed gradient."""
+    world, port = 2, _free_port()
+    mp.spawn(_sharded_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    sys.path.insert(0, ROOT)
+    import oracle
+    from paper_2502_20566_b200 import synth
+    r = [np.load(tmp_path / f"s{k}.npz") for k in range(world)]
+    n = 8 * world * 1500
+    per = n // world
+    p, _, m, v = synth.adamw_state(n, 88, "cpu")
+    g_sum = r[0]["g"] + r[1]["g"]
+    S = sum(oracle.sqnorm(np.ascontiguousarray(g_sum[k * per:(k + 1) * per])) for k in range(world))
+    assert float(r[0]["total"][0]) == S and r[0]["total"].tobytes() == r[1]["total"].tobytes()
+    gscale = oracle.clip_scale(S, 1.0 / world, 1.0)
+    pb, mb, vb = (synth.bits16(t).copy() for t in (p, m, v))
+    oracle.adamw_step(pb, g_sum.copy(), mb, vb, oracle.hparams(**HP), 1234, 7, 0, 0, gscale)
+    assert np.array_equal(r[0]["full"], pb) and np.array_equal(r[1]["full"], pb)
+    assert np.array_equal(np.concatenate([r[0]["m"], r[1]["m"]]), mb)
+    assert np.array_equal(np.concatenate([r[0]["v"], r[1]["v"]]), vb)
+
+
 def test_partition_properties():
     sys.path.insert(0, ROOT)
     from paper_2502_20566_b200.dist import partition

@@ -513,3 +513,34 @@ def test_master_recipe_bit_exact(env, n, shift, g_dtype, gscale):
             assert np.all((got[nan] & 0x7FFFFFFF) > 0x7F800000)
             host_t[nan] = dev_t.cpu().numpy()[nan]                      # keep both sides on the same NaN bits
         assert mismatches(bits(p16), want16) == 0
+
+
+# ---------------------------------------------------------------------------------------------
+# sharded step through torch.distributed (one rank here; two ranks are covered on CPU with gloo)
+# ---------------------------------------------------------------------------------------------
+
+def test_sharded_clipped_step_single_rank_nccl(env):
+    import os
+    import socket
+    import torch.distributed as dist
+    oracle, binding, synth, dev = env
+    from paper_2502_20566_b200.dist import sharded_clipped_step
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=dev)
+    try:
+        n = 8 * 40000
+        p, g, m, v = synth.adamw_state(n, 91, dev, g_dtype=torch.float32, outlier_fraction=0.01)
+        pb, gb, mb, vb = bits(p), host_g(g), bits(m), bits(v)
+        full = torch.empty(n, dtype=torch.bfloat16, device=dev)
+        total = sharded_clipped_step(p, m, v, g, HP, 1234, 3, max_norm=1.0, accum_scale=0.125, full_param_out=full)
+        torch.cuda.synchronize()
+        S = oracle.sqnorm(gb)
+        assert float(total.item()).hex() == S.hex()
+        oracle.adamw_step(pb, gb, mb, vb, oracle.hparams(**HP), 1234, 3, 0, 0, oracle.clip_scale(S, 0.125, 1.0))
+        assert mismatches(bits(p), pb) == 0 and mismatches(bits(full), pb) == 0
+        assert mismatches(bits(m), mb) == 0 and mismatches(bits(v), vb) == 0
+    finally:
+        dist.destroy_process_group()
