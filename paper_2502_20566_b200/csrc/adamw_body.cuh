@@ -33,8 +33,6 @@ __device__ __forceinline__ void async_copy_commit() { asm volatile("cp.async.com
 template <int PENDING>
 __device__ __forceinline__ void async_copy_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
 
-constexpr int kStages = 2;   // vectors per thread in flight or in use (measured: 2 beats 3 and 4)
-
 // unpack a staged gradient vector (one 16-byte piece for BF16, two for FP32)
 template <bool G32>
 __device__ __forceinline__ void unpack_grad8(const uint4 g0, const uint4 g1, float (&ge)[8]) {
@@ -196,18 +194,18 @@ __device__ __forceinline__ void step_scalar(uint16_t* p, const void* g, uint16_t
 inline bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
 
 template <typename Kernel>
-int resident_blocks(Kernel kernel, const DeviceInfo& dev) {
+int resident_blocks(Kernel kernel, const DeviceInfo& dev, int threads = kBlockThreads) {
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kBlockThreads, 0) != cudaSuccess || per_sm < 1)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, 0) != cudaSuccess || per_sm < 1)
         per_sm = 1;
     return per_sm * dev.sm_count;
 }
 
 // grid for `work_items` thread-items: no more blocks than are resident at once, no more than needed
 template <typename Kernel>
-unsigned grid_for(Kernel kernel, uint64_t work_items, const DeviceInfo& dev) {
-    const uint64_t needed = (work_items + kBlockThreads - 1) / kBlockThreads;
-    const uint64_t resident = static_cast<uint64_t>(resident_blocks(kernel, dev));
+unsigned grid_for(Kernel kernel, uint64_t work_items, const DeviceInfo& dev, int threads = kBlockThreads) {
+    const uint64_t needed = (work_items + threads - 1) / threads;
+    const uint64_t resident = static_cast<uint64_t>(resident_blocks(kernel, dev, threads));
     const uint64_t g = needed < resident ? needed : resident;
     return static_cast<unsigned>(g < 1 ? 1 : g);
 }

@@ -32,23 +32,27 @@ k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n
 // The hot kernel (modes 2 and 3 of the launcher): 16-byte vectors, branch-free arithmetic, gradient
 // used as is (SCALE = false) or multiplied by gscale.  elem_offset is a multiple of 8 and every
 // index of the launch has the same (index >> 33) = c1.  Same persistent grid.  STAGED = true: each
-// thread keeps its next vector in flight -- while vector k is computed out of shared memory, the
-// asynchronous copies of vector k + T are already under way (kStages slots per thread and array).
-// STAGED = false loads straight into registers.
-template <bool G32, uint32_t FLAGS, bool SCALE, bool STAGED>
-__global__ void __launch_bounds__(kBlockThreads, kMinBlocksPerSM)
+// thread keeps its next vectors in flight -- while vector k is computed out of shared memory, the
+// asynchronous copies of vectors k + T, ... are already under way (kFlatStages slots per thread and
+// array).  SHAPE 0: direct loads into registers, kBlockThreads x kMinBlocksPerSM; 1: staged, same
+// block shape, kShortStages; 2: staged, kFlatStagedThreads x kFlatStagedMinBlocks, kFlatStages.
+template <bool G32, uint32_t FLAGS, bool SCALE, int SHAPE>
+__global__ void __launch_bounds__(SHAPE == 2 ? kFlatStagedThreads : kBlockThreads, SHAPE == 2 ? kFlatStagedMinBlocks : kMinBlocksPerSM)
 k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset,
                      uint32_t c1, uint32_t tensor_id, uint32_t seed_hi, const __grid_constant__ PhiloxKeys K,
                      const __grid_constant__ StepScalars S) {
     constexpr int kArrays = G32 ? 5 : 4;   // x, m, v and one or two 16-byte pieces of g
-    __shared__ uint4 stage[STAGED ? kStages * kArrays * kBlockThreads : 1];
+    constexpr bool STAGED = SHAPE != 0;
+    constexpr int kThreads = SHAPE == 2 ? kFlatStagedThreads : kBlockThreads;
+    constexpr int kStages = SHAPE == 2 ? kFlatStages : kShortStages;
+    __shared__ uint4 stage[STAGED ? kStages * kArrays * kThreads : 1];
     const float gscale = S.gscale_dev ? __ldg(S.gscale_dev) : S.gscale;
     const uint64_t tid = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
     const uint64_t nvec = n >> 3;
     if (STAGED) {
         uint4* const mine = stage + threadIdx.x;
-        auto slot = [&](int s, int a) -> uint4* { return mine + (s * kArrays + a) * kBlockThreads; };
+        auto slot = [&](int s, int a) -> uint4* { return mine + (s * kArrays + a) * kThreads; };
         auto issue = [&](uint64_t vec, int s) {
             if (vec < nvec) {
                 async_copy16(slot(s, 0), reinterpret_cast<const uint4*>(p) + vec);
@@ -80,8 +84,20 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
         }
         async_copy_wait<0>();
     } else {
-        for (uint64_t vec = tid; vec < nvec; vec += stride)
+        for (uint64_t vec = tid; vec < nvec; vec += stride) {
+#ifdef SR_L2_PREFETCH_AHEAD
+            {
+                const uint64_t pf = vec + SR_L2_PREFETCH_AHEAD * stride;
+                if (pf < nvec) {
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint4*>(p) + pf));
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint4*>(m) + pf));
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint4*>(v) + pf));
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint4*>(g) + (G32 ? 2 : 1) * pf));
+                }
+            }
+#endif
             step_vec8_fast<G32, FLAGS, SCALE>(p, g, m, v, vec, elem_offset + (vec << 3), c1, tensor_id, seed_hi, gscale, K, S);
+        }
     }
     const uint64_t done = nvec << 3;
     if (tid < n - done)
@@ -105,10 +121,15 @@ cudaError_t launch_flat_mode(uint16_t* p, const void* g, uint16_t* m, uint16_t* 
     const uint64_t items = MODE == 0 ? n : (n >> 3) + 8;   // + 8: enough threads for the ragged tail
     if (MODE >= 2) {
         constexpr bool kStaged = G32 ? (SR_STAGE_F32 != 0) : (SR_STAGE_BF16 != 0);
-        auto k = k_sr_adamw_flat_fast<G32, FLAGS, MODE == 3, kStaged>;
-        k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset,
-                                                                 static_cast<uint32_t>(elem_offset >> 33), tensor_id,
-                                                                 seed_hi, K, S);
+        const uint32_t c1 = static_cast<uint32_t>(elem_offset >> 33);
+        if (kStaged && n >= kLongLaunchElems) {
+            auto k = k_sr_adamw_flat_fast<G32, FLAGS, MODE == 3, kStaged ? 2 : 0>;
+            constexpr int kThreads = kStaged ? kFlatStagedThreads : kBlockThreads;
+            k<<<grid_for(k, items, dev, kThreads), kThreads, 0, stream>>>(p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
+        } else {
+            auto k = k_sr_adamw_flat_fast<G32, FLAGS, MODE == 3, kStaged ? 1 : 0>;
+            k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
+        }
     } else {
         auto k = k_sr_adamw_flat<G32, FLAGS, (MODE < 2 ? MODE : 0)>;
         k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset, tensor_id, seed_hi, K, S);

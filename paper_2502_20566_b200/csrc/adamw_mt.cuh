@@ -53,8 +53,8 @@ k_sr_adamw_mt(const MtWork* __restrict__ work, uint32_t num_chunks, uint32_t ten
               const __grid_constant__ PhiloxKeys K, const __grid_constant__ StepScalars S) {
     constexpr int kArrays = G32 ? 5 : 4;
     constexpr bool kStage = STAGED && MODE >= 2;
-    __shared__ uint4 stage[kStage ? kStages * kArrays * kBlockThreads : 1];
-    static_assert(kStages == 2, "slot bookkeeping below assumes two stages");
+    __shared__ uint4 stage[kStage ? kMtStages * kArrays * kBlockThreads : 1];
+    static_assert(kMtStages == 2, "slot bookkeeping below assumes two stages");
     const float gscale = S.gscale_dev ? __ldg(S.gscale_dev) : S.gscale;
     const uint32_t tid = threadIdx.x;
     uint4* const mine = stage + tid;

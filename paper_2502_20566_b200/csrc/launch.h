@@ -23,18 +23,40 @@ struct MtWork {
 static_assert(sizeof(MtWork) == 48, "three 16-byte loads per entry");
 
 constexpr uint32_t kMtChunkElems = 8192;   // multiple of 8; never crosses a multiple of 2^33
+// Launch shapes, from sweeps on B200 with the 6.7B flat buffer (64..512 threads x 1..10 blocks/SM x
+// 2..6 stages on the real kernels).  Every kernel's arithmetic needs about 96 registers; tighter
+// budgets cost more in instruction scheduling than they gain in occupancy.
+//  - kernels that load straight into registers: 128 threads, >= 5 blocks/SM (640 threads/SM);
+//  - the staged flat kernel has two shapes.  Long launches (>= 2^30 elements, tens of milliseconds,
+//    which run into the board's power cap): 256 threads, 2 blocks/SM, 3 vectors per thread in
+//    flight or in use (48 KB of shared memory per block) -- with the memory latency covered by the
+//    staging, fewer resident warps ran faster under the cap (90% vs 86% of the copy peak at 6.7B).
+//    Shorter launches, which finish before the cap bites: 128 x 5 with 2 stages (93% vs 87% at
+//    355M elements);
+//  - the staged multi-tensor kernel keeps 128 x 5 with 2 stages.
 #ifndef SR_BLOCK_THREADS
 #define SR_BLOCK_THREADS 128
 #endif
 #ifndef SR_MIN_BLOCKS_PER_SM
 #define SR_MIN_BLOCKS_PER_SM 5
 #endif
+#ifndef SR_FLAT_STAGED_THREADS
+#define SR_FLAT_STAGED_THREADS 256
+#endif
+#ifndef SR_FLAT_STAGED_MIN_BLOCKS
+#define SR_FLAT_STAGED_MIN_BLOCKS 2
+#endif
+#ifndef SR_FLAT_STAGES
+#define SR_FLAT_STAGES 3
+#endif
 constexpr int kBlockThreads = SR_BLOCK_THREADS;
-// Launch shape of the fused-step kernels, from a sweep on B200 (6.7B flat buffer): 128-thread
-// blocks with at least 5 resident per SM (96 registers per thread, 640 threads per SM) was the
-// best of 64..512 threads x 1..10 blocks; tighter register budgets cost more in instruction
-// scheduling than they gain in occupancy.
 constexpr int kMinBlocksPerSM = SR_MIN_BLOCKS_PER_SM;
+constexpr int kFlatStagedThreads = SR_FLAT_STAGED_THREADS;
+constexpr int kFlatStagedMinBlocks = SR_FLAT_STAGED_MIN_BLOCKS;
+constexpr int kFlatStages = SR_FLAT_STAGES;
+constexpr int kMtStages = 2;
+constexpr int kShortStages = 2;
+constexpr uint64_t kLongLaunchElems = static_cast<uint64_t>(1) << 30;
 
 struct DeviceInfo {
     int sm_count;
