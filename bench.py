@@ -33,11 +33,11 @@ SEED = 1234
 FIRST_STEP = 1000
 BYTES_PER_ELEMENT = 14          # read x, g, m, v (4 x 2 B) + write x, m, v (3 x 2 B)
 FALLBACK_HBM_GBS = 6650.0       # used only when MEASURED_PEAKS.json is absent
-# (dram__bytes_read.sum + dram__bytes_write.sum) / elements from the ncu capture of the current kernel on
-# the 2^27-element case (profiles/k_sr_adamw_flat_fast__bf16_grads_sr_xmv__2pow27.md); traffic of a streaming
-# kernel grows in proportion to the element count, so the full-size figure is this times n.  Set to
-# None whenever the kernel changes until a new capture exists.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = (1.073771e9 + 0.747271168e9) / (1 << 27)
+# DRAM bytes (read + write) per element from the ncu capture of the current kernel and launch shape on the
+# 2^30-element case (profiles/k_sr_adamw_flat_fast__long_launch_shape__2pow30.md: 5.794371 TB/s x 2.584544 ms);
+# the traffic of a streaming kernel grows in proportion to the element count, so the full-size figure is
+# this times n.  Set to None whenever the kernel changes until a new capture exists.
+NCU_TRAFFIC_BYTES_PER_ELEMENT = 5.794371e12 * 2.584544e-3 / (1 << 30)
 
 
 def parse_args():
