@@ -132,6 +132,33 @@ def test_flat_step_hyperparameter_corners(env):
         assert run_both(env, p, g, m, v, kw, seed=6, step=step) == (0, 0, 0)
 
 
+@pytest.mark.parametrize("kw,step", [
+    (dict(lr=1e-3, beta1=0.9, beta2=0.999999, eps=1.0, weight_decay=0.01), 1),      # 1/sqrt(1-beta2^t) = 1000, eps at its bound
+    (dict(lr=1e-3, beta1=0.5, beta2=0.999, eps=0.0, weight_decay=0.0), 1),
+    (dict(lr=3e-4, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1), 1000),
+    (dict(lr=1e-3, beta1=0.9, beta2=0.9999999, eps=1e-8, weight_decay=0.0), 1),     # beyond the gate: reference arithmetic
+])
+def test_in_range_arithmetic_over_its_whole_operand_range(env, kw, step):
+    """Moments spread log-uniformly over and beyond the operand range of the branch-free square root
+    and division (v, |m| from 2^-70 to 2^70, both gradient types), with the scalars at the limits
+    under which that path is chosen: every vector inside the range must equal IEEE sqrt/div, every
+    vector outside must have been redone."""
+    _, _, synth, dev = env
+    n = 1 << 20
+    gen = torch.Generator(device=dev).manual_seed(1234 + step)
+    for g_dtype in (torch.bfloat16, torch.float32):
+        p, g, m, v = synth.adamw_state(n, 17, dev, g_dtype=g_dtype)
+        span = 70.0 if g_dtype == torch.bfloat16 else 59.0      # second pass: (almost) every vector stays inside
+        ev = (torch.rand(n, generator=gen, device=dev) * 2.0 - 1.0) * span
+        em = (torch.rand(n, generator=gen, device=dev) * 2.0 - 1.0) * span
+        sign = torch.where(torch.rand(n, generator=gen, device=dev) < 0.5, -1.0, 1.0)
+        v.copy_(torch.exp2(ev).to(torch.bfloat16))
+        m.copy_((sign * torch.exp2(em)).to(torch.bfloat16))
+        g.mul_(0)                                   # m', v' are then beta * m, beta * v: the spread survives
+        g[::7] = 1e-3
+        assert run_both(env, p, g, m, v, kw, seed=8, step=step) == (0, 0, 0)
+
+
 def test_shards_equal_whole_and_runs_repeat(env):
     """Shared random state: 8 shards stepped separately equal the whole buffer; a second run repeats
     the first bit for bit; another seed does not."""
