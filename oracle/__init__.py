@@ -85,6 +85,11 @@ def lib() -> ctypes.CDLL:
         L.oracle_master_adamw_step.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_uint64,
                                                POINTER(HParams), c_float, c_uint32]
         L.oracle_master_adamw_step.restype = c_int
+        L.oracle_sr_fp8_bits.argtypes = [c_uint32, c_uint32, c_int]
+        L.oracle_sr_fp8_bits.restype = ctypes.c_uint8
+        L.oracle_noise32.argtypes = [c_uint64, c_uint32, c_uint32, c_uint64]
+        L.oracle_noise32.restype = c_uint32
+        L.oracle_sr_downcast_fp8.argtypes = [c_void_p, c_void_p, c_uint64, c_int, c_uint64, c_uint32, c_uint32, c_uint64]
         L.oracle_sr_downcast.argtypes = [c_void_p, c_void_p, c_uint64, c_uint64, c_uint32, c_uint32, c_uint64]
         L.oracle_sqnorm.argtypes = [c_void_p, c_int, c_uint64]
         L.oracle_sqnorm.restype = c_double
@@ -188,6 +193,21 @@ def sr_downcast(src, seed, step=0, tensor_id=0, elem_offset=0):
     _check(src, np.float32)
     dst = np.empty(src.shape, dtype=np.uint16)
     lib().oracle_sr_downcast(_ptr(src), _ptr(dst), src.size, seed, step, tensor_id, elem_offset)
+    return dst
+
+
+def sr_fp8_bits(fbits: int, r32: int, e5m2: bool) -> int:
+    return int(lib().oracle_sr_fp8_bits(fbits & 0xFFFFFFFF, r32 & 0xFFFFFFFF, 1 if e5m2 else 0))
+
+
+def noise32(seed: int, step: int, tensor_id: int, index: int) -> int:
+    return int(lib().oracle_noise32(seed, step, tensor_id, index))
+
+
+def sr_downcast_fp8(src, e5m2: bool, seed, step=0, tensor_id=0, elem_offset=0):
+    _check(src, np.float32)
+    dst = np.empty(src.shape, dtype=np.uint8)
+    lib().oracle_sr_downcast_fp8(_ptr(src), _ptr(dst), src.size, 1 if e5m2 else 0, seed, step, tensor_id, elem_offset)
     return dst
 
 

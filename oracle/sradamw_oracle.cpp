@@ -303,6 +303,68 @@ int oracle_master_adamw_step(float* p, uint16_t* p_bf16, const void* g, int g_is
     return 0;
 }
 
+// ---- Eq. 2 onto an 8-bit floating-point grid -------------------------------------------------
+// The paper's closing remark: the method carries over to FP8.  Formats: E4M3 (4 exponent bits,
+// bias 7, 3 mantissa bits, no infinity, largest finite 448, S.1111.111 = NaN) and E5M2 (5 exponent
+// bits, bias 15, 2 mantissa bits, IEEE-like, largest finite 57344).  For |x| = a with binary
+// exponent E, the two neighbouring levels are spaced Delta = 2^(Eq - M), Eq = max(E, 1 - bias)
+// (subnormal levels share the spacing of the smallest normal binade).  y = a / Delta = k + f with
+// integer k and 0 <= f < 1; Eq. 2 moves to level k + 1 with probability f.  With a uniform 32-bit
+// integer r the move happens iff r < floor(f * 2^32), which is exactly probability f whenever f has
+// at most 32 fractional bits (every FP32 input down to 2^-12 of the smallest subnormal level) and
+// rounds the probability down by less than 2^-32 otherwise.  Magnitudes at or beyond the largest
+// finite level saturate to it (E5M2 keeps infinity); NaN gives the pattern 0x7F.
+// The code of level k' in binade Eq is ((Eq + bias - 1) << M) + k' for normal and subnormal levels
+// alike, and a carry to k' = 2^(M+1) lands on the first level of the next binade.
+uint8_t sr_fp8_bits(uint32_t fbits, uint32_t r32, int e5m2) {
+    const int M = e5m2 ? 2 : 3, bias = e5m2 ? 15 : 7;
+    const uint32_t max_code = e5m2 ? 0x7Bu : 0x7Eu;
+    const float max_value = e5m2 ? 57344.0f : 448.0f;
+    const uint8_t sign = static_cast<uint8_t>((fbits >> 24) & 0x80u);
+    if (is_nan_bits(fbits)) return 0x7F;
+    const float a = float_of(fbits & 0x7FFFFFFFu);
+    if (std::isinf(a)) return static_cast<uint8_t>(sign | (e5m2 ? 0x7Cu : max_code));
+    if (a >= max_value) return static_cast<uint8_t>(sign | max_code);
+    if (a == 0.0f) return sign;
+    int E;
+    std::frexp(a, &E);      // a = mant * 2^E with mant in [0.5, 1): binary exponent is E - 1
+    E -= 1;
+    const int Eq = E > 1 - bias ? E : 1 - bias;
+    const double y = std::ldexp(static_cast<double>(a), M - Eq);      // exact: power-of-two scaling
+    const double k = std::floor(y);
+    const double f = y - k;
+    const double threshold = std::floor(std::ldexp(f, 32));
+    const uint32_t up = static_cast<double>(r32) < threshold ? 1u : 0u;
+    uint32_t code = static_cast<uint32_t>((Eq + bias - 1) << M) + static_cast<uint32_t>(k) + up;
+    if (code > max_code) code = max_code;
+    return static_cast<uint8_t>(sign | code);
+}
+
+// 32 noise bits per element: one Philox call per four consecutive elements, counter number =
+// index >> 2, element index & 3 takes output word index & 3 (key and the other counter words as above).
+uint32_t noise32_for(uint64_t seed, uint32_t step, uint32_t tensor_id, uint64_t index) {
+    const uint64_t number = index >> 2;
+    const uint32_t ctr[4] = {static_cast<uint32_t>(number), static_cast<uint32_t>(number >> 32),
+                             tensor_id, static_cast<uint32_t>(seed >> 32)};
+    const uint32_t key[2] = {static_cast<uint32_t>(seed), step};
+    uint32_t w[4];
+    philox4x32_10(ctr, key, w);
+    return w[index & 3u];
+}
+
+void oracle_sr_downcast_fp8(const float* src, uint8_t* dst, uint64_t n, int e5m2, uint64_t seed, uint32_t step,
+                            uint32_t tensor_id, uint64_t elem_offset) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < static_cast<int64_t>(n); ++i)
+        dst[i] = sr_fp8_bits(bits_of(src[i]), noise32_for(seed, step, tensor_id, elem_offset + static_cast<uint64_t>(i)), e5m2);
+}
+
+uint8_t oracle_sr_fp8_bits(uint32_t fbits, uint32_t r32, int e5m2) { return sr_fp8_bits(fbits, r32, e5m2); }
+
+uint32_t oracle_noise32(uint64_t seed, uint32_t step, uint32_t tensor_id, uint64_t index) {
+    return noise32_for(seed, step, tensor_id, index);
+}
+
 // Q_SR on an FP32 array; uses rounding slot 0 (the x slot) of the noise.
 void oracle_sr_downcast(const float* src, uint16_t* dst, uint64_t n, uint64_t seed, uint32_t step,
                         uint32_t tensor_id, uint64_t elem_offset) {
