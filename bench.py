@@ -272,6 +272,11 @@ def time_extras(torch, binding, synth, dev, peak):
     t_c = timed(lambda: binding.sr_downcast_f32_bf16(src, dst, seed=7))
     out["sr_downcast_f32_bf16"] = {"elements": nc, "ms": t_c, "params_per_s": nc / t_c * 1e3, "gbs": 6 * nc / t_c / 1e6,
                                    "frac": 6 * nc / t_c / 1e6 / peak}
+    # FP8 stochastic-rounding cast (5 B per element)
+    dst8 = torch.empty(nc, dtype=torch.uint8, device=dev).view(torch.float8_e4m3fn)
+    t_8 = timed(lambda: binding.sr_downcast_f32_fp8(src, dst8, seed=7))
+    out["sr_downcast_f32_fp8_e4m3"] = {"elements": nc, "ms": t_8, "params_per_s": nc / t_8 * 1e3, "gbs": 5 * nc / t_8 / 1e6,
+                                       "frac": 5 * nc / t_8 / 1e6 / peak}
     return out
 
 

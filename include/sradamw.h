@@ -78,6 +78,19 @@ typedef struct sr_adamw_hparams {
 sr_status sr_downcast_f32_bf16(const float* src, uint16_t* dst, uint64_t n, uint64_t seed, uint32_t step,
                                uint32_t tensor_id, uint64_t elem_offset, void* stream);
 
+/* Eq. 2 onto an 8-bit floating-point grid (the extension the paper's conclusion names): dst[i] =
+ * Q_SR(src[i]) with the two neighbouring levels taken from E4M3 (bias 7, no infinity, largest finite
+ * 448, NaN = S.1111.111) or E5M2 (bias 15, IEEE-like, largest finite 57344).  With a = |x| in the
+ * binade Eq = max(E, 1 - bias), y = a / 2^(Eq - M) = k + f: the value moves to level k + 1 iff
+ * r < floor(f * 2^32) for a uniform 32-bit r, i.e. with probability f (exact whenever f has at most
+ * 32 fractional bits).  Magnitudes at or beyond the largest finite level saturate to it (E5M2 keeps
+ * +-inf), NaN gives 0x7F.  Noise: one Philox call per four consecutive indices, counter number =
+ * index >> 2 (other counter and key words as above), element index & 3 takes output word index & 3.
+ * src: n FP32 values; dst: n bytes. */
+typedef enum { SR_FP8_E4M3 = 0, SR_FP8_E5M2 = 1 } sr_fp8_format;
+sr_status sr_downcast_f32_fp8(const float* src, uint8_t* dst, uint64_t n, sr_fp8_format format, uint64_t seed,
+                              uint32_t step, uint32_t tensor_id, uint64_t elem_offset, void* stream);
+
 /* One iteration of Algorithm 1 on a flat buffer of n elements (moment updates, bias-corrected
  * direction with epsilon outside the square root, decoupled weight decay, rounding of x, m, v).
  * p, m, v: BF16 in/out.  g: BF16 or FP32 per g_dtype.  step >= 1 is the 1-based iteration t.

@@ -23,7 +23,7 @@ SR_FLAG_SR_P, SR_FLAG_SR_M, SR_FLAG_SR_V = 1, 2, 4
 SR_FLAGS_DEFAULT = 7
 
 EXPORTS = (
-    "sr_downcast_f32_bf16", "sr_adamw_step", "sr_master_adamw_step", "sr_adamw_step_host", "sr_adamw_step_host_staging_bytes",
+    "sr_downcast_f32_bf16", "sr_downcast_f32_fp8", "sr_adamw_step", "sr_master_adamw_step", "sr_adamw_step_host", "sr_adamw_step_host_staging_bytes",
     "sr_mt_plan_create", "sr_adamw_multi_tensor",
     "sr_mt_plan_destroy", "sr_mt_plan_total_elements", "grad_sqnorm_workspace_bytes", "grad_sqnorm",
     "grad_sqnorm_static", "grad_sqnorm_static_max_elements",
@@ -76,6 +76,8 @@ def lib() -> ctypes.CDLL:
         L = ctypes.CDLL(LIB_PATH)
         L.sr_downcast_f32_bf16.argtypes = [c_void_p, c_void_p, c_uint64, c_uint64, c_uint32, c_uint32, c_uint64, c_void_p]
         L.sr_downcast_f32_bf16.restype = c_int
+        L.sr_downcast_f32_fp8.argtypes = [c_void_p, c_void_p, c_uint64, c_int, c_uint64, c_uint32, c_uint32, c_uint64, c_void_p]
+        L.sr_downcast_f32_fp8.restype = c_int
         L.sr_adamw_step.argtypes = [c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_uint64, POINTER(HParams),
                                     c_uint64, c_uint32, c_uint32, c_uint64, c_void_p]
         L.sr_adamw_step.restype = c_int
@@ -145,6 +147,23 @@ def sr_downcast_f32_bf16(src: torch.Tensor, dst: torch.Tensor, seed: int, step: 
     with torch.cuda.device(src.device):
         _check(lib().sr_downcast_f32_bf16(src.data_ptr(), dst.data_ptr(), src.numel(), seed, step, tensor_id,
                                           elem_offset, _stream(stream)), "sr_downcast_f32_bf16")
+
+
+SR_FP8_E4M3, SR_FP8_E5M2 = 0, 1
+
+
+def sr_downcast_f32_fp8(src: torch.Tensor, dst: torch.Tensor, seed: int, step: int = 0, tensor_id: int = 0,
+                        elem_offset: int = 0, stream=None) -> None:
+    """dst: torch.float8_e4m3fn, torch.float8_e5m2 (the format follows the dtype) or uint8 (E4M3)."""
+    _want(src, torch.float32, "src")
+    if not dst.is_cuda or not dst.is_contiguous() or dst.element_size() != 1:
+        raise TypeError("dst: expected a contiguous CUDA tensor of an 8-bit type")
+    fmt = SR_FP8_E5M2 if dst.dtype == torch.float8_e5m2 else SR_FP8_E4M3
+    if src.numel() != dst.numel():
+        raise ValueError("size mismatch")
+    with torch.cuda.device(src.device):
+        _check(lib().sr_downcast_f32_fp8(src.data_ptr(), dst.data_ptr(), src.numel(), fmt, seed, step, tensor_id,
+                                         elem_offset, _stream(stream)), "sr_downcast_f32_fp8")
 
 
 def sr_adamw_step(p: torch.Tensor, g: torch.Tensor, m: torch.Tensor, v: torch.Tensor, hp: HParams, seed: int,

@@ -123,6 +123,20 @@ sr_status sr_downcast_f32_bf16(const float* src, uint16_t* dst, uint64_t n, uint
     return e == cudaSuccess ? SR_OK : cuda_fail(e);
 }
 
+sr_status sr_downcast_f32_fp8(const float* src, uint8_t* dst, uint64_t n, sr_fp8_format format, uint64_t seed,
+                              uint32_t step, uint32_t tensor_id, uint64_t elem_offset, void* stream) {
+    if (format != SR_FP8_E4M3 && format != SR_FP8_E5M2) return SR_ERR_INVALID_ARG;
+    if (n == 0) return SR_OK;
+    if (src == nullptr || dst == nullptr) return SR_ERR_INVALID_ARG;
+    DeviceInfo dev;
+    sr_status st = current_device(&dev);
+    if (st != SR_OK) return st;
+    const cudaError_t e = launch_downcast_fp8(src, dst, n, format == SR_FP8_E5M2, elem_offset, tensor_id,
+                                              static_cast<uint32_t>(seed >> 32), make_keys(seed, step), dev,
+                                              static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SR_OK : cuda_fail(e);
+}
+
 sr_status sr_adamw_step(uint16_t* p, const void* g, sr_dtype g_dtype, uint16_t* m, uint16_t* v, uint64_t n,
                         const sr_adamw_hparams* hp, uint64_t seed, uint32_t step, uint32_t tensor_id,
                         uint64_t elem_offset, void* stream) {

@@ -1,0 +1,110 @@
+// Stochastic-rounding cast FP32 -> FP8 (E4M3 / E5M2): Eq. 2 on the 8-bit grids, the extension the
+// paper's conclusion names.  5 bytes per element (4 read, 1 written).  32 noise bits per element,
+// one Philox call per four consecutive elements (counter number = index >> 2, word = index & 3).
+
+#include "adamw_body.cuh"
+
+namespace sradamw {
+
+namespace {
+
+template <bool E5M2>
+struct Fp8 {
+    static constexpr int M = E5M2 ? 2 : 3;
+    static constexpr int kBias = E5M2 ? 15 : 7;
+    static constexpr uint32_t kMaxCode = E5M2 ? 0x7Bu : 0x7Eu;
+    static constexpr uint32_t kMaxBits = E5M2 ? 0x47600000u : 0x43E00000u;   // 57344.0f, 448.0f
+    static constexpr uint32_t kInfCode = E5M2 ? 0x7Cu : 0x7Eu;               // E4M3 has no infinity
+    static constexpr uint32_t kMinBiasedExp = 127 + 1 - kBias;               // FP32 exponent field of the smallest normal level
+};
+
+// One value.  a = |x| lies in the binade Eq = max(E, 1 - bias); y = a / 2^(Eq - M) = k + f; move to
+// level k + 1 iff r < floor(f * 2^32).  In integers: with the 24-bit significand `mant` of a and
+// D = (23 - M) + (Eq - E) dropped bits, (mant * 2^32) >> D holds k in its high word and
+// floor(f * 2^32) in its low word (for D >= 56 both are zero: the probability is below 2^-32).
+// The code of level k' is ((Eq + bias - 1) << M) + k' for subnormal and normal levels alike.
+template <bool E5M2>
+__device__ __forceinline__ uint32_t sr_fp8_code(uint32_t fbits, uint32_t r) {
+    using F = Fp8<E5M2>;
+    const uint32_t sign = (fbits >> 24) & 0x80u;
+    const uint32_t abits = fbits & 0x7FFFFFFFu;
+    const uint32_t e_raw = abits >> 23;                             // biased FP32 exponent
+    const uint32_t e = e_raw == 0 ? 1u : e_raw;                     // FP32 subnormals sit at 2^-126 without implicit bit
+    const uint32_t mant = (abits & 0x7FFFFFu) | (e_raw == 0 ? 0u : 0x800000u);
+    const uint32_t eq = e < F::kMinBiasedExp ? F::kMinBiasedExp : e;  // Eq + 127
+    uint32_t dropped = (23u - F::M) + (eq - e);
+    dropped = dropped > 63u ? 63u : dropped;
+    // (mant : 0) >> dropped as two clamped funnel shifts: high word = k, low word = floor(f * 2^32)
+    const uint32_t d_lo = dropped > 32u ? 32u : dropped, d_hi = dropped - d_lo;
+    const uint32_t k = __funnelshift_rc(mant, 0u, d_lo);
+    const uint32_t threshold = __funnelshift_rc(0u, mant, d_lo) >> d_hi;
+    uint32_t code = ((eq - 127u + F::kBias - 1u) << F::M) + k + (r < threshold ? 1u : 0u);
+    code = code > F::kMaxCode ? F::kMaxCode : code;                 // saturation, also for every |x| >= the largest level
+    if (E5M2) code = abits == 0x7F800000u ? F::kInfCode : code;
+    return abits > 0x7F800000u ? 0x7Fu : (sign | code);
+}
+
+__device__ __forceinline__ uint32_t noise32_of_element(uint64_t idx, uint32_t c2, uint32_t c3, const PhiloxKeys& K) {
+    const uint64_t number = idx >> 2;
+    const uint4 w = philox4x32_10(static_cast<uint32_t>(number), static_cast<uint32_t>(number >> 32), c2, c3, K);
+    const uint32_t e = static_cast<uint32_t>(idx) & 3u;
+    return e == 0 ? w.x : e == 1 ? w.y : e == 2 ? w.z : w.w;
+}
+
+template <bool E5M2>
+__device__ __forceinline__ uint32_t cast4(const uint4 x, const uint4 w) {
+    return sr_fp8_code<E5M2>(x.x, w.x) | (sr_fp8_code<E5M2>(x.y, w.y) << 8) | (sr_fp8_code<E5M2>(x.z, w.z) << 16) |
+           (sr_fp8_code<E5M2>(x.w, w.w) << 24);
+}
+
+// VEC: 16 elements per thread-iteration (4 x 16-byte loads, 1 x 16-byte store); needs both buffers
+// 16-byte aligned and elem_offset a multiple of 4 (whole noise groups).
+template <bool E5M2, bool VEC>
+__global__ void __launch_bounds__(kBlockThreads)
+k_sr_downcast_fp8(const float* __restrict__ src, uint8_t* __restrict__ dst, uint64_t n, uint64_t elem_offset,
+                  uint32_t tensor_id, uint32_t seed_hi, const __grid_constant__ PhiloxKeys K) {
+    const uint64_t tid = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
+    uint64_t done = 0;
+    if (VEC) {
+        const uint64_t nvec = n >> 4;
+        for (uint64_t vec = tid; vec < nvec; vec += stride) {
+            const uint4 a = ld16(src, 4 * vec), b = ld16(src, 4 * vec + 1), c = ld16(src, 4 * vec + 2), d = ld16(src, 4 * vec + 3);
+            const uint64_t number = (elem_offset + (vec << 4)) >> 2;
+            const uint32_t c0 = static_cast<uint32_t>(number), c1 = static_cast<uint32_t>(number >> 32);
+            uint4 o;
+            o.x = cast4<E5M2>(a, philox4x32_10(c0, c1, tensor_id, seed_hi, K));
+            o.y = cast4<E5M2>(b, philox4x32_10(c0 + 1, c1, tensor_id, seed_hi, K));
+            o.z = cast4<E5M2>(c, philox4x32_10(c0 + 2, c1, tensor_id, seed_hi, K));
+            o.w = cast4<E5M2>(d, philox4x32_10(c0 + 3, c1, tensor_id, seed_hi, K));
+            st16(dst, vec, o);
+        }
+        done = nvec << 4;
+    }
+    for (uint64_t i = done + tid; i < n; i += stride)
+        dst[i] = static_cast<uint8_t>(sr_fp8_code<E5M2>(__float_as_uint(src[i]), noise32_of_element(elem_offset + i, tensor_id, seed_hi, K)));
+}
+
+template <bool E5M2, bool VEC>
+cudaError_t launch_fp8_t(const float* src, uint8_t* dst, uint64_t n, uint64_t elem_offset, uint32_t tensor_id,
+                         uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev, cudaStream_t stream) {
+    auto k = k_sr_downcast_fp8<E5M2, VEC>;
+    const uint64_t items = VEC ? (n >> 4) + 16 : n;
+    k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(src, dst, n, elem_offset, tensor_id, seed_hi, K);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_downcast_fp8(const float* src, uint8_t* dst, uint64_t n, bool e5m2, uint64_t elem_offset,
+                                uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev,
+                                cudaStream_t stream) {
+    // the low word of the group number must not wrap inside a 16-element vector: offset multiple of 16
+    const bool vec = aligned16(src) && aligned16(dst) && (elem_offset & 15u) == 0;
+    if (e5m2) return vec ? launch_fp8_t<true, true>(src, dst, n, elem_offset, tensor_id, seed_hi, K, dev, stream)
+                         : launch_fp8_t<true, false>(src, dst, n, elem_offset, tensor_id, seed_hi, K, dev, stream);
+    return vec ? launch_fp8_t<false, true>(src, dst, n, elem_offset, tensor_id, seed_hi, K, dev, stream)
+               : launch_fp8_t<false, false>(src, dst, n, elem_offset, tensor_id, seed_hi, K, dev, stream);
+}
+
+}  // namespace sradamw

@@ -74,6 +74,10 @@ cudaError_t launch_adamw_mt(const MtWork* work, uint32_t num_chunks, bool g_f32,
                             uint32_t tensor_id_base, uint32_t seed_hi, uint32_t flags, const PhiloxKeys& K,
                             const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream);
 
+cudaError_t launch_downcast_fp8(const float* src, uint8_t* dst, uint64_t n, bool e5m2, uint64_t elem_offset,
+                                uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev,
+                                cudaStream_t stream);
+
 cudaError_t launch_master_adamw(float* p, uint16_t* p16, const void* g, bool g_f32, float* m, float* v, uint64_t n,
                                 const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream);
 

@@ -571,3 +571,53 @@ def test_sharded_clipped_step_single_rank_nccl(env):
         assert mismatches(bits(m), mb) == 0 and mismatches(bits(v), vb) == 0
     finally:
         dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------------
+# FP8 stochastic-rounding cast
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype", [torch.float8_e4m3fn, torch.float8_e5m2])
+@pytest.mark.parametrize("n,offset,shift", [(0, 0, 0), (3, 0, 0), (1 << 22, 0, 0), ((1 << 20) + 13, 16 * 77, 0), (70001, 5, 0),
+                                            (70001, 32, 1), (5000, (1 << 34) - 64, 0)])
+def test_fp8_cast_bit_exact(env, dtype, n, offset, shift):
+    oracle, binding, synth, dev = env
+    e5m2 = dtype == torch.float8_e5m2
+    src = synth.downcast_mix(n + shift, 21, dev)[shift:]
+    if n > 1000:                                   # most of the mix lies outside the FP8 range: add in-range values
+        k = n // 2
+        scale = torch.pow(10.0, torch.rand(k, device=dev, generator=torch.Generator(device=dev).manual_seed(4)) * 8 - 6)
+        src[:k] = torch.randn(k, device=dev, generator=torch.Generator(device=dev).manual_seed(3)) * scale
+    dst = torch.zeros(n + shift + 16, dtype=torch.uint8, device=dev).view(dtype)
+    out = dst[shift:shift + n]
+    binding.sr_downcast_f32_fp8(src, out, seed=(9 << 32) | 5, step=2, tensor_id=7, elem_offset=offset)
+    torch.cuda.synchronize()
+    want = oracle.sr_downcast_fp8(src.cpu().numpy().copy(), e5m2, (9 << 32) | 5, 2, 7, offset)
+    got = out.view(torch.uint8).cpu().numpy()
+    assert int(np.count_nonzero(got != want)) == 0
+    assert int(dst.view(torch.uint8)[shift + n:].sum()) == 0 and int(dst.view(torch.uint8)[:shift].sum()) == 0
+    if n > 1000:
+        assert len(np.unique(got)) > 100           # the cast really spreads over the grid
+
+
+def test_fp8_cast_is_unbiased_over_seeds(env):
+    """Mean over 2048 seeds of 4096 in-range values: within 6 sigma of x, sigma^2 = Delta^2 f (1 - f) / seeds."""
+    _, binding, _, dev = env
+    k, seeds = 4096, 2048
+    gen = torch.Generator(device=dev).manual_seed(11)
+    x = (torch.rand(k, device=dev, generator=gen) * 2 - 1) * torch.pow(2.0, torch.rand(k, device=dev, generator=gen) * 12 - 6)
+    for dtype in (torch.float8_e4m3fn, torch.float8_e5m2):
+        outs = torch.empty((seeds, k), dtype=torch.uint8, device=dev).view(dtype)
+        for s in range(seeds):
+            binding.sr_downcast_f32_fp8(x, outs[s], seed=s)
+        torch.cuda.synchronize()
+        vals = outs.to(torch.float32).double()
+        M, bias = (2, 15) if dtype == torch.float8_e5m2 else (3, 7)
+        a = x.double().abs()
+        eq = torch.clamp(torch.floor(torch.log2(a)), min=1 - bias)            # binade that sets the spacing
+        delta = torch.exp2(eq - M)
+        lo = torch.floor(a / delta) * delta
+        f = (a - lo) / delta
+        assert torch.all((vals.abs() == lo) | (vals.abs() == lo + delta))      # the two neighbouring levels only
+        sigma = delta * torch.sqrt(f * (1 - f) / seeds)
+        assert torch.all((vals.mean(dim=0) - x.double()).abs() <= 6 * sigma + 1e-300)
