@@ -84,20 +84,8 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
         }
         async_copy_wait<0>();
     } else {
-        for (uint64_t vec = tid; vec < nvec; vec += stride) {
-#ifdef SR_L2_PREFETCH_AHEAD
-            {
-                const uint64_t pf = vec + SR_L2_PREFETCH_AHEAD * stride;
-                if (pf < nvec) {
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint4*>(p) + pf));
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint4*>(m) + pf));
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint4*>(v) + pf));
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint4*>(g) + (G32 ? 2 : 1) * pf));
-                }
-            }
-#endif
+        for (uint64_t vec = tid; vec < nvec; vec += stride)
             step_vec8_fast<G32, FLAGS, SCALE>(p, g, m, v, vec, elem_offset + (vec << 3), c1, tensor_id, seed_hi, gscale, K, S);
-        }
     }
     const uint64_t done = nvec << 3;
     if (tid < n - done)
