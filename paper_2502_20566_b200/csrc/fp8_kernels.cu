@@ -18,30 +18,35 @@ struct Fp8 {
     static constexpr uint32_t kMinBiasedExp = 127 + 1 - kBias;               // FP32 exponent field of the smallest normal level
 };
 
-// One value.  a = |x| lies in the binade Eq = max(E, 1 - bias); y = a / 2^(Eq - M) = k + f; move to
-// level k + 1 iff r < floor(f * 2^32).  In integers: with the 24-bit significand `mant` of a and
-// D = (23 - M) + (Eq - E) dropped bits, (mant * 2^32) >> D holds k in its high word and
-// floor(f * 2^32) in its low word (for D >= 56 both are zero: the probability is below 2^-32).
-// The code of level k' is ((Eq + bias - 1) << M) + k' for subnormal and normal levels alike.
+// The magnitude code of one value (sign handled by the caller).  a = |x| lies in the binade
+// Eq = max(E, 1 - bias); y = a / 2^(Eq - M) = k + f; move to level k + 1 iff r < floor(f * 2^32).
+// In integers: with the 24-bit significand `mant` of a and D = (23 - M) + (Eq - E) dropped bits,
+// (mant * 2^32) >> D holds k in its high word and floor(f * 2^32) in its low word; both are zero once
+// D >= 56, which also covers zero and the FP32 subnormals (their exponent field is 0, so D is far
+// beyond 56 whatever their significand).  The code of level k' is ((Eq + bias - 1) << M) + k' for
+// subnormal and normal levels alike; the clamp saturates every finite |x| beyond the largest level.
+template <bool E5M2>
+__device__ __forceinline__ uint32_t sr_fp8_magnitude(uint32_t abits, uint32_t r) {
+    using F = Fp8<E5M2>;
+    const uint32_t e = abits >> 23;                                    // biased FP32 exponent
+    const uint32_t mant = (abits & 0x7FFFFFu) | 0x800000u;
+    const uint32_t eq = e < F::kMinBiasedExp ? F::kMinBiasedExp : e;   // Eq + 127
+    const uint32_t dropped = (23u - F::M) + (eq - e);                  // 20 or 21 in the normal range
+    // (mant : 0) >> dropped with clamped funnel shifts (a shift of 32 or more yields what is left)
+    const uint32_t k = __funnelshift_rc(mant, 0u, dropped);
+    const uint32_t low = __funnelshift_rc(0u, mant, dropped);
+    const uint32_t threshold = dropped > 32u ? __funnelshift_rc(mant, 0u, dropped - 32u) : low;
+    uint32_t code = ((eq - 127u + F::kBias - 1u) << F::M) + k + (r < threshold ? 1u : 0u);
+    code = code > F::kMaxCode ? F::kMaxCode : code;
+    if (E5M2) code = abits == 0x7F800000u ? F::kInfCode : code;
+    return abits > 0x7F800000u ? 0x7Fu : code;                         // NaN -> 0x7F (its sign is dropped below)
+}
+
 template <bool E5M2>
 __device__ __forceinline__ uint32_t sr_fp8_code(uint32_t fbits, uint32_t r) {
-    using F = Fp8<E5M2>;
-    const uint32_t sign = (fbits >> 24) & 0x80u;
     const uint32_t abits = fbits & 0x7FFFFFFFu;
-    const uint32_t e_raw = abits >> 23;                             // biased FP32 exponent
-    const uint32_t e = e_raw == 0 ? 1u : e_raw;                     // FP32 subnormals sit at 2^-126 without implicit bit
-    const uint32_t mant = (abits & 0x7FFFFFu) | (e_raw == 0 ? 0u : 0x800000u);
-    const uint32_t eq = e < F::kMinBiasedExp ? F::kMinBiasedExp : e;  // Eq + 127
-    uint32_t dropped = (23u - F::M) + (eq - e);
-    dropped = dropped > 63u ? 63u : dropped;
-    // (mant : 0) >> dropped as two clamped funnel shifts: high word = k, low word = floor(f * 2^32)
-    const uint32_t d_lo = dropped > 32u ? 32u : dropped, d_hi = dropped - d_lo;
-    const uint32_t k = __funnelshift_rc(mant, 0u, d_lo);
-    const uint32_t threshold = __funnelshift_rc(0u, mant, d_lo) >> d_hi;
-    uint32_t code = ((eq - 127u + F::kBias - 1u) << F::M) + k + (r < threshold ? 1u : 0u);
-    code = code > F::kMaxCode ? F::kMaxCode : code;                 // saturation, also for every |x| >= the largest level
-    if (E5M2) code = abits == 0x7F800000u ? F::kInfCode : code;
-    return abits > 0x7F800000u ? 0x7Fu : (sign | code);
+    const uint32_t sign = abits > 0x7F800000u ? 0u : ((fbits >> 24) & 0x80u);
+    return sign | sr_fp8_magnitude<E5M2>(abits, r);
 }
 
 __device__ __forceinline__ uint32_t noise32_of_element(uint64_t idx, uint32_t c2, uint32_t c3, const PhiloxKeys& K) {
@@ -51,10 +56,17 @@ __device__ __forceinline__ uint32_t noise32_of_element(uint64_t idx, uint32_t c2
     return e == 0 ? w.x : e == 1 ? w.y : e == 2 ? w.z : w.w;
 }
 
+// four values -> four bytes; the four sign bits are gathered with two byte permutes
 template <bool E5M2>
 __device__ __forceinline__ uint32_t cast4(const uint4 x, const uint4 w) {
-    return sr_fp8_code<E5M2>(x.x, w.x) | (sr_fp8_code<E5M2>(x.y, w.y) << 8) | (sr_fp8_code<E5M2>(x.z, w.z) << 16) |
-           (sr_fp8_code<E5M2>(x.w, w.w) << 24);
+    const uint32_t ax = x.x & 0x7FFFFFFFu, ay = x.y & 0x7FFFFFFFu, az = x.z & 0x7FFFFFFFu, aw = x.w & 0x7FFFFFFFu;
+    const uint32_t m0 = sr_fp8_magnitude<E5M2>(ax, w.x), m1 = sr_fp8_magnitude<E5M2>(ay, w.y);
+    const uint32_t m2 = sr_fp8_magnitude<E5M2>(az, w.z), m3 = sr_fp8_magnitude<E5M2>(aw, w.w);
+    const uint32_t mags = __byte_perm(__byte_perm(m0, m1, 0x0040), __byte_perm(m2, m3, 0x0040), 0x5410);
+    const uint32_t tops = __byte_perm(__byte_perm(x.x, x.y, 0x0073), __byte_perm(x.z, x.w, 0x0073), 0x5410);
+    // a NaN code (0x7F) keeps no sign: mask the sign bit where the magnitude byte is 0x7F with all of bits 0..6 set
+    const uint32_t is_nan = ((mags & 0x7F7F7F7Fu) + 0x01010101u) & 0x80808080u;
+    return mags | (tops & 0x80808080u & ~is_nan);
 }
 
 // VEC: 16 elements per thread-iteration (4 x 16-byte loads, 1 x 16-byte store); needs both buffers
