@@ -301,6 +301,48 @@ def test_random_walk_example_on_the_gpu(env):
         assert abs(p_n - 0.25 * (1 - eps) ** (n - 3) * eps) < 5 * (0.02 / walkers) ** 0.5
 
 
+def test_linear_loss_toy_qualitative(env):
+    """Section 2.2, second example, run on the library: Adam on the linear loss f(x) = -(x - 2) + 1 for
+    x < 3 (0 beyond), from x0 = 2, with a decaying learning rate.  The paper does not give the decay
+    schedule, so only the qualitative statements are checked, with an assumed schedule (linear decay over
+    5000 steps, chosen so that FP32 reaches x = 3 in about 4600 steps at minimum rate 1e-5): BF16 with
+    stochastic rounding needs more steps than FP32 on average, and fewer when the minimum rate is higher."""
+    _, binding, _, dev = env
+    runs, horizon = 1024, 40000
+
+    def schedule(t, lr_min):
+        lr_max = 3.94e-4
+        return max(lr_min, lr_max - (lr_max - 1e-5) * t / 5000.0)
+
+    def steps_to_converge(lr_min, sr):
+        kw = dict(beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
+        x = torch.full((runs,), 2.0, device=dev, dtype=torch.bfloat16 if sr else torch.float32)
+        m, v = torch.zeros_like(x), torch.zeros_like(x)
+        x16 = torch.empty(runs, dtype=torch.bfloat16, device=dev)
+        hit = torch.zeros(runs, dtype=torch.int32, device=dev)
+        for t in range(1, horizon + 1):
+            g = torch.where(x < 3.0, -1.0, 0.0).to(torch.bfloat16)
+            hp = binding.hparams(lr=schedule(t - 1, lr_min), **kw)
+            if sr:
+                binding.sr_adamw_step(x, g, m, v, hp, seed=77, step=t)
+            else:
+                binding.sr_master_adamw_step(x, x16, g, m, v, hp, t)
+            hit = torch.where((hit == 0) & (x >= 3.0), torch.full_like(hit, t), hit)
+            if t % 500 == 0 and int((hit == 0).sum()) == 0:
+                break
+        # a run still short of x = 3 at the horizon counts as the horizon: its mean is then a lower bound
+        return torch.where(hit == 0, torch.full_like(hit, horizon), hit).double()
+
+    fp32 = steps_to_converge(1e-5, sr=False)
+    assert float(fp32.min()) == float(fp32.max()) and 4500 <= float(fp32[0]) <= 4700
+    assert float(fp32[0]) < horizon
+    sr_slow = steps_to_converge(1e-5, sr=True)
+    sr_fast = steps_to_converge(5e-5, sr=True)
+    assert float(sr_slow.mean()) > 1.1 * float(fp32[0])          # stagnation at small learning rates
+    assert float(sr_fast.mean()) < float(sr_slow.mean())          # a higher minimum rate closes the gap
+    assert float(sr_slow.std()) > 0                               # runs differ: the rounding is stochastic
+
+
 # ---------------------------------------------------------------------------------------------
 # squared norm, clipping, and the clipped shard step
 # ---------------------------------------------------------------------------------------------
