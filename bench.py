@@ -51,6 +51,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-elements", type=int, default=1 << 29)
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary kernels (shard step, tensor list, cast)")
+    ap.add_argument("--case", choices=EXTRA_CASES, default=None,
+                    help="run one secondary call alone (with --elements: on a small case) instead of the headline step")
     return ap.parse_args()
 
 
@@ -187,13 +189,19 @@ def run_reference(args):
 # CUDA arm
 # ---------------------------------------------------------------------------------------------
 
-def time_extras(torch, binding, synth, dev, peak):
-    """The other calls of the library, each timed alone (CUDA events, 3 warm-ups + 10 launches) on its
-    own workload; bytes are the algorithmic ones.  Reported beside the headline, not part of it."""
-    stream = torch.cuda.current_stream()
+EXTRA_CASES = ("shard_fp32_grads", "fp32_master_recipe", "tensor_list", "cast_bf16", "cast_fp8")
 
-    def timed(fn, reps=10):
-        for _ in range(3):
+
+def time_extras(torch, binding, synth, dev, peak, only=None, elements=0, reps=10, warmup=3):
+    """The other calls of the library, each timed alone (CUDA events, 3 warm-ups + 10 launches) on its
+    own workload; bytes are the algorithmic ones.  Reported beside the headline, not part of it.
+    `only` names one case of EXTRA_CASES (the others are skipped) and `elements` shrinks its buffers:
+    the small single-kernel runs that profiler captures are taken on."""
+    stream = torch.cuda.current_stream()
+    want = lambda *cases: only is None or only in cases
+
+    def timed(fn, reps=reps):
+        for _ in range(warmup):
             fn()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
@@ -205,9 +213,28 @@ def time_extras(torch, binding, synth, dev, peak):
         return a.elapsed_time(b) / reps
 
     out = {}
+    if want("shard_fp32_grads", "fp32_master_recipe"):
+        _extras_shard(torch, binding, synth, dev, peak, timed, out, want, elements)
+    if want("tensor_list"):
+        _extras_list(torch, binding, synth, dev, peak, timed, out, compare_flat=only is None)
+    if want("cast_bf16", "cast_fp8"):
+        _extras_casts(torch, binding, synth, dev, peak, timed, out, want, elements)
+    return out
+
+
+def _extras_shard(torch, binding, synth, dev, peak, timed, out, want, elements):
     # 1/8 shard with FP32 gradients: squared norm -> clip factor -> step (20 B per element over two passes)
-    n = synth.gpt_flat_numel() // 8
+    n = elements or synth.gpt_flat_numel() // 8
     p, g, m, v = synth.adamw_state(n, SEED, dev, g_dtype=torch.float32, outlier_fraction=0.01)
+    if want("shard_fp32_grads"):
+        _extras_shard_sr(torch, binding, dev, peak, timed, out, n, p, g, m, v)
+    del p, m, v
+    if want("fp32_master_recipe"):
+        _extras_master(torch, binding, synth, dev, peak, timed, out, n, g)
+    out.pop("sr_step_ms_same_shard", None)
+
+
+def _extras_shard_sr(torch, binding, dev, peak, timed, out, n, p, g, m, v):
     ws = torch.empty(max(1, binding.grad_sqnorm_workspace_bytes(n) // 8), dtype=torch.float64, device=dev)
     S = torch.zeros(1, dtype=torch.float64, device=dev)
     gs = torch.zeros(1, dtype=torch.float32, device=dev)
@@ -220,6 +247,7 @@ def time_extras(torch, binding, synth, dev, peak):
         binding.sr_clip_scale(S, 0.125, 1.0, gs)
         binding.sr_adamw_step(p, g, m, v, hp_clip, SEED, FIRST_STEP, 0, 3 * n)
     t_all = timed(clipped)
+    out["sr_step_ms_same_shard"] = t_step
     out["shard_fp32_grads"] = {
         "elements": n,
         "grad_sqnorm": {"ms": t_norm, "gbs": 4 * n / t_norm / 1e6, "frac": 4 * n / t_norm / 1e6 / peak},
@@ -227,7 +255,9 @@ def time_extras(torch, binding, synth, dev, peak):
         "norm_clip_step": {"ms": t_all, "params_per_s": n / t_all * 1e3, "gbs": 20 * n / t_all / 1e6,
                            "frac": 20 * n / t_all / 1e6 / peak},
     }
-    del p, m, v, ws
+
+
+def _extras_master(torch, binding, synth, dev, peak, timed, out, n, g):
     # the mixed-precision comparison recipe on the same shard: FP32 master weights and moments + BF16 copy
     p32, m32, v32 = (torch.empty(n, dtype=torch.float32, device=dev) for _ in range(3))
     for t, role in ((p32, synth.ROLE_P), (m32, synth.ROLE_M), (v32, synth.ROLE_V)):
@@ -239,8 +269,10 @@ def time_extras(torch, binding, synth, dev, peak):
     out["fp32_master_recipe_same_shard"] = {
         "elements": n, "bytes_per_element": 30, "ms": t_mp, "params_per_s": n / t_mp * 1e3, "gbs": 30 * n / t_mp / 1e6,
         "frac": 30 * n / t_mp / 1e6 / peak, "state_bytes_per_param": 14, "sr_state_bytes_per_param": 6,
-        "time_vs_sr_step": t_mp / t_step}
-    del p32, m32, v32, p16, g
+        "time_vs_sr_step": t_mp / out["sr_step_ms_same_shard"] if "sr_step_ms_same_shard" in out else None}
+
+
+def _extras_list(torch, binding, synth, dev, peak, timed, out, compare_flat):
     # GPT-2 350M tensor list, one launch per step
     specs = synth.gpt2_param_list()
     P = [synth.init_param(sp, SEED, i, dev) for i, sp in enumerate(specs)]
@@ -260,24 +292,28 @@ def time_extras(torch, binding, synth, dev, peak):
                                     "gbs": 14 * ne / t_mt / 1e6, "frac": 14 * ne / t_mt / 1e6 / peak}
     plan.destroy()
     del P, G, M, V
+    if not compare_flat:
+        return
     # the flat kernel on a buffer of the same length, for comparison with the list launch
     fp, fg, fm, fv = synth.adamw_state(ne, SEED, dev)
     t_f = timed(lambda: binding.sr_adamw_step(fp, fg, fm, fv, hp, SEED, FIRST_STEP))
     out["flat_same_length_as_list"] = {"elements": ne, "ms": t_f, "gbs": 14 * ne / t_f / 1e6, "frac": 14 * ne / t_f / 1e6 / peak}
-    del fp, fg, fm, fv
-    # standalone stochastic-rounding cast, 2^28 FP32 values (6 B per element)
-    nc = 1 << 28
+
+
+def _extras_casts(torch, binding, synth, dev, peak, timed, out, want, elements):
+    # standalone stochastic-rounding casts of 2^28 FP32 values: BF16 (6 B per element), FP8 (5 B per element)
+    nc = elements or 1 << 28
     src = synth.downcast_mix(nc, 7, dev)
-    dst = torch.empty(nc, dtype=torch.bfloat16, device=dev)
-    t_c = timed(lambda: binding.sr_downcast_f32_bf16(src, dst, seed=7))
-    out["sr_downcast_f32_bf16"] = {"elements": nc, "ms": t_c, "params_per_s": nc / t_c * 1e3, "gbs": 6 * nc / t_c / 1e6,
-                                   "frac": 6 * nc / t_c / 1e6 / peak}
-    # FP8 stochastic-rounding cast (5 B per element)
-    dst8 = torch.empty(nc, dtype=torch.uint8, device=dev).view(torch.float8_e4m3fn)
-    t_8 = timed(lambda: binding.sr_downcast_f32_fp8(src, dst8, seed=7))
-    out["sr_downcast_f32_fp8_e4m3"] = {"elements": nc, "ms": t_8, "params_per_s": nc / t_8 * 1e3, "gbs": 5 * nc / t_8 / 1e6,
-                                       "frac": 5 * nc / t_8 / 1e6 / peak}
-    return out
+    if want("cast_bf16"):
+        dst = torch.empty(nc, dtype=torch.bfloat16, device=dev)
+        t_c = timed(lambda: binding.sr_downcast_f32_bf16(src, dst, seed=7))
+        out["sr_downcast_f32_bf16"] = {"elements": nc, "ms": t_c, "params_per_s": nc / t_c * 1e3,
+                                       "gbs": 6 * nc / t_c / 1e6, "frac": 6 * nc / t_c / 1e6 / peak}
+    if want("cast_fp8"):
+        dst8 = torch.empty(nc, dtype=torch.uint8, device=dev).view(torch.float8_e4m3fn)
+        t_8 = timed(lambda: binding.sr_downcast_f32_fp8(src, dst8, seed=7))
+        out["sr_downcast_f32_fp8_e4m3"] = {"elements": nc, "ms": t_8, "params_per_s": nc / t_8 * 1e3,
+                                           "gbs": 5 * nc / t_8 / 1e6, "frac": 5 * nc / t_8 / 1e6 / peak}
 
 
 def hbm_peak():
@@ -305,6 +341,14 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     binding.lib()
+
+    if args.case:   # one secondary call alone: the run a profiler capture of that kernel is taken on
+        peak, peak_src = hbm_peak()
+        res = time_extras(torch, binding, synth, dev, peak, only=args.case, elements=args.elements,
+                          reps=args.steps, warmup=args.warmup)
+        print(json.dumps({"case": args.case, "steps": args.steps, "warmup": args.warmup, "peak": peak,
+                          "peak_source": peak_src, "result": res}), flush=True)
+        return
 
     n = args.elements or synth.gpt_flat_numel()
     bufs = [torch.empty(n, dtype=torch.bfloat16, device=dev) for _ in range(4)]
