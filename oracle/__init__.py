@@ -91,6 +91,15 @@ def lib() -> ctypes.CDLL:
         L.oracle_noise32.restype = c_uint32
         L.oracle_sr_downcast_fp8.argtypes = [c_void_p, c_void_p, c_uint64, c_int, c_uint64, c_uint32, c_uint32, c_uint64]
         L.oracle_sr_downcast.argtypes = [c_void_p, c_void_p, c_uint64, c_uint64, c_uint32, c_uint32, c_uint64]
+        L.oracle_sr_fp4_bits.argtypes = [c_uint32, c_uint32]
+        L.oracle_sr_fp4_bits.restype = ctypes.c_uint8
+        L.oracle_sr_downcast_fp4.argtypes = [c_void_p, c_void_p, c_uint64, c_uint64, c_uint32, c_uint32, c_uint64]
+        L.oracle_noise_slot.argtypes = [c_uint64, c_uint32, c_uint32, c_uint64, c_uint32]
+        L.oracle_noise_slot.restype = c_uint32
+        L.oracle_accumulate_element.argtypes = [ctypes.c_uint16, c_float, c_float, c_uint32, c_int]
+        L.oracle_accumulate_element.restype = ctypes.c_uint16
+        L.oracle_sr_accumulate.argtypes = [c_void_p, c_void_p, c_int, c_uint64, c_float, c_int, c_uint64, c_uint32,
+                                           c_uint32, c_uint64]
         L.oracle_sqnorm.argtypes = [c_void_p, c_int, c_uint64]
         L.oracle_sqnorm.restype = c_double
         L.oracle_tree_sum.argtypes = [c_void_p, c_uint64]
@@ -209,6 +218,43 @@ def sr_downcast_fp8(src, e5m2: bool, seed, step=0, tensor_id=0, elem_offset=0):
     dst = np.empty(src.shape, dtype=np.uint8)
     lib().oracle_sr_downcast_fp8(_ptr(src), _ptr(dst), src.size, 1 if e5m2 else 0, seed, step, tensor_id, elem_offset)
     return dst
+
+
+def sr_fp4_bits(fbits: int, r32: int) -> int:
+    """Code (sign bit 3, magnitude bits 0..2) of Q_SR on the E2M1 grid for one FP32 pattern and one noise word."""
+    return int(lib().oracle_sr_fp4_bits(fbits & 0xFFFFFFFF, r32 & 0xFFFFFFFF))
+
+
+def sr_downcast_fp4(src, seed, step=0, tensor_id=0, elem_offset=0):
+    """Packed E2M1 codes, two per byte (even element in the low half)."""
+    _check(src, np.float32)
+    dst = np.empty((src.size + 1) // 2, dtype=np.uint8)
+    lib().oracle_sr_downcast_fp4(_ptr(src), _ptr(dst), src.size, seed, step, tensor_id, elem_offset)
+    return dst
+
+
+def noise_slot(seed: int, step: int, tensor_id: int, index: int, slot: int) -> int:
+    """16-bit noise of rounding slot 0..3 of one element."""
+    return int(lib().oracle_noise_slot(seed, step, tensor_id, index, slot))
+
+
+def accumulate_element(acc_bits: int, g: float, scale: float, r16: int, stochastic: bool = True) -> int:
+    return int(lib().oracle_accumulate_element(acc_bits & 0xFFFF, g, scale, r16 & 0xFFFF, 1 if stochastic else 0))
+
+
+def sr_accumulate(acc, g, scale, seed, step, tensor_id=0, elem_offset=0, stochastic=True):
+    """In place: acc (BF16 bit patterns, uint16) <- rounding(acc + scale * g); g is uint16 (BF16) or float32."""
+    _check(acc, np.uint16)
+    if g.dtype == np.float32:
+        _check(g, np.float32)
+        is32 = 1
+    else:
+        _check(g, np.uint16)
+        is32 = 0
+    assert g.size == acc.size
+    lib().oracle_sr_accumulate(_ptr(acc), _ptr(g), is32, acc.size, scale, 1 if stochastic else 0, seed, step, tensor_id,
+                               elem_offset)
+    return acc
 
 
 def sqnorm(g) -> float:

@@ -21,6 +21,11 @@
 //                             direction, decoupled decay), in FP32, before any rounding.
 //   oracle_adamw_step         Algorithm 1 over an array: element function + Q_SR on x, m and v.
 //   oracle_sr_downcast        Q_SR applied to an FP32 array.
+//   oracle_sr_downcast_fp8    Q_SR of Eq. 2 on the 8-bit grids E4M3 and E5M2, and
+//   oracle_sr_downcast_fp4    on the 4-bit grid E2M1 (the conclusion names FP8/4 as the next targets).
+//   oracle_sr_accumulate      Q_SR (or Q) applied to a BF16 accumulator plus a new term (Section 3
+//                             keeps the accumulated gradient in BF16 too).
+//   oracle_master_adamw_step  the mixed-precision recipe the paper compares against.
 //   oracle_sqnorm             sum of squares of the gradient with a fixed summation tree
 //   oracle_clip_scale         global-norm clipping coefficient.  (Neither is in the paper; they
 //                             are the usual companions of the update and are defined below.)
@@ -217,6 +222,10 @@ void oracle_noise(uint64_t seed, uint32_t step, uint32_t tensor_id, uint64_t ind
     out[0] = r.rp; out[1] = r.rm; out[2] = r.rv;
 }
 
+uint32_t oracle_noise_slot(uint64_t seed, uint32_t step, uint32_t tensor_id, uint64_t index, uint32_t slot) {
+    return noise_for_slot(seed, step, tensor_id, index, slot);
+}
+
 uint16_t oracle_sr_bf16_bits(uint32_t fbits, uint32_t r16) { return sr_bf16_bits(fbits, r16); }
 
 uint16_t oracle_rne_bf16_bits(uint32_t fbits) { return rne_bf16_bits(fbits); }
@@ -363,6 +372,83 @@ uint8_t oracle_sr_fp8_bits(uint32_t fbits, uint32_t r32, int e5m2) { return sr_f
 
 uint32_t oracle_noise32(uint64_t seed, uint32_t step, uint32_t tensor_id, uint64_t index) {
     return noise32_for(seed, step, tensor_id, index);
+}
+
+// ---- Eq. 2 onto the 4-bit grid E2M1 ----------------------------------------------------------
+// The same closing remark names 4-bit formats.  E2M1: one sign bit, 2 exponent bits (bias 1), one
+// mantissa bit; the eight magnitudes are 0, 0.5, 1, 1.5, 2, 3, 4, 6 (codes 0..7); there is neither
+// an infinity nor a NaN.  The rule is the one above with M = 1, bias = 1.  Every magnitude at or
+// beyond 6 saturates to 6, infinity included; a NaN has no image in the format and is written as the
+// largest magnitude with its sign bit (a choice of this restatement, not of the paper).
+uint8_t sr_fp4_bits(uint32_t fbits, uint32_t r32) {
+    const int M = 1, bias = 1;
+    const uint32_t max_code = 7u;
+    const uint8_t sign = static_cast<uint8_t>((fbits >> 28) & 0x8u);
+    if (is_nan_bits(fbits)) return static_cast<uint8_t>(sign | max_code);
+    const float a = float_of(fbits & 0x7FFFFFFFu);
+    if (a >= 6.0f) return static_cast<uint8_t>(sign | max_code);
+    if (a == 0.0f) return sign;
+    int E;
+    std::frexp(a, &E);
+    E -= 1;
+    const int Eq = E > 1 - bias ? E : 1 - bias;
+    const double y = std::ldexp(static_cast<double>(a), M - Eq);
+    const double k = std::floor(y);
+    const double f = y - k;
+    const double threshold = std::floor(std::ldexp(f, 32));
+    const uint32_t up = static_cast<double>(r32) < threshold ? 1u : 0u;
+    uint32_t code = static_cast<uint32_t>((Eq + bias - 1) << M) + static_cast<uint32_t>(k) + up;
+    if (code > max_code) code = max_code;
+    return static_cast<uint8_t>(sign | code);
+}
+
+uint8_t oracle_sr_fp4_bits(uint32_t fbits, uint32_t r32) { return sr_fp4_bits(fbits, r32); }
+
+// Array form: two codes per byte, element 2j in bits 0..3 and element 2j+1 in bits 4..7 of byte j
+// (the upper half of the last byte is 0 when n is odd).  Noise: the 32-bit word per element above.
+void oracle_sr_downcast_fp4(const float* src, uint8_t* dst, uint64_t n, uint64_t seed, uint32_t step,
+                            uint32_t tensor_id, uint64_t elem_offset) {
+    const int64_t nbytes = static_cast<int64_t>((n + 1) / 2);
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < nbytes; ++j) {
+        const uint64_t i0 = 2u * static_cast<uint64_t>(j), i1 = i0 + 1;
+        uint8_t b = sr_fp4_bits(bits_of(src[i0]), noise32_for(seed, step, tensor_id, elem_offset + i0));
+        if (i1 < n)
+            b = static_cast<uint8_t>(b | (sr_fp4_bits(bits_of(src[i1]), noise32_for(seed, step, tensor_id, elem_offset + i1)) << 4));
+        dst[j] = b;
+    }
+}
+
+// ---- Eq. 2 in a BF16 accumulation -------------------------------------------------------------
+// Section 3 keeps every tensor in BF16, the accumulated gradient included.  Adding a small term to
+// a BF16 accumulator with nearest rounding loses it whenever it is below half a spacing (the
+// stagnation of Section 2.1); with Q_SR the expected sum is exact.  One accumulation:
+//   t = scale * g          (FP32, one rounding; exact for scale = 1)
+//   s = acc + t            (FP32, one rounding)
+//   acc <- Q_SR(s)  or  Q(s)
+// The noise is rounding slot 3 of the element's group (the counter number 4 * group + 3, which the
+// optimizer step leaves unused), so that accumulation and update draw from disjoint streams even
+// under the same (seed, step, tensor_id).
+uint16_t accumulate_element(uint16_t acc, float g, float scale, uint32_t r16, int stochastic) {
+    const float t = scale * g;
+    const float s = bf16_to_float(acc) + t;
+    return stochastic ? sr_bf16_bits(bits_of(s), r16) : rne_bf16_bits(bits_of(s));
+}
+
+uint16_t oracle_accumulate_element(uint16_t acc, float g, float scale, uint32_t r16, int stochastic) {
+    return accumulate_element(acc, g, scale, r16, stochastic);
+}
+
+void oracle_sr_accumulate(uint16_t* acc, const void* g, int g_is_f32, uint64_t n, float scale, int stochastic,
+                          uint64_t seed, uint32_t step, uint32_t tensor_id, uint64_t elem_offset) {
+    const float* g32 = static_cast<const float*>(g);
+    const uint16_t* g16 = static_cast<const uint16_t*>(g);
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < static_cast<int64_t>(n); ++i) {
+        const float gi = g_is_f32 ? g32[i] : bf16_to_float(g16[i]);
+        const uint32_t r = noise_for_slot(seed, step, tensor_id, elem_offset + static_cast<uint64_t>(i), 3);
+        acc[i] = accumulate_element(acc[i], gi, scale, r, stochastic);
+    }
 }
 
 // Q_SR on an FP32 array; uses rounding slot 0 (the x slot) of the noise.
