@@ -189,7 +189,7 @@ def run_reference(args):
 # CUDA arm
 # ---------------------------------------------------------------------------------------------
 
-EXTRA_CASES = ("shard_fp32_grads", "fp32_master_recipe", "tensor_list", "cast_bf16", "cast_fp8")
+EXTRA_CASES = ("shard_fp32_grads", "fp32_master_recipe", "tensor_list", "cast_bf16", "cast_fp8", "cast_fp4", "accumulate")
 
 
 def time_extras(torch, binding, synth, dev, peak, only=None, elements=0, reps=10, warmup=3):
@@ -217,8 +217,10 @@ def time_extras(torch, binding, synth, dev, peak, only=None, elements=0, reps=10
         _extras_shard(torch, binding, synth, dev, peak, timed, out, want, elements)
     if want("tensor_list"):
         _extras_list(torch, binding, synth, dev, peak, timed, out, compare_flat=only is None)
-    if want("cast_bf16", "cast_fp8"):
+    if want("cast_bf16", "cast_fp8", "cast_fp4"):
         _extras_casts(torch, binding, synth, dev, peak, timed, out, want, elements)
+    if want("accumulate"):
+        _extras_accumulate(torch, binding, synth, dev, peak, timed, out, elements)
     return out
 
 
@@ -314,6 +316,25 @@ def _extras_casts(torch, binding, synth, dev, peak, timed, out, want, elements):
         t_8 = timed(lambda: binding.sr_downcast_f32_fp8(src, dst8, seed=7))
         out["sr_downcast_f32_fp8_e4m3"] = {"elements": nc, "ms": t_8, "params_per_s": nc / t_8 * 1e3,
                                            "gbs": 5 * nc / t_8 / 1e6, "frac": 5 * nc / t_8 / 1e6 / peak}
+    if want("cast_fp4"):
+        dst4 = torch.empty(nc // 2, dtype=torch.uint8, device=dev)
+        t_4 = timed(lambda: binding.sr_downcast_f32_fp4(src, dst4, seed=7))
+        out["sr_downcast_f32_fp4_e2m1"] = {"elements": nc, "ms": t_4, "params_per_s": nc / t_4 * 1e3,
+                                           "gbs": 4.5 * nc / t_4 / 1e6, "frac": 4.5 * nc / t_4 / 1e6 / peak}
+
+
+def _extras_accumulate(torch, binding, synth, dev, peak, timed, out, elements):
+    # BF16 accumulator += BF16 term with stochastic rounding (6 B per element), on the 1/8 shard
+    n = elements or synth.gpt_flat_numel() // 8
+    _, g, acc, _ = synth.adamw_state(n, SEED, dev)
+    step = [0]
+
+    def accumulate():
+        step[0] += 1
+        binding.sr_accumulate_bf16(acc, g, 0.125, SEED, step[0])
+    t_a = timed(accumulate)
+    out["sr_accumulate_bf16"] = {"elements": n, "ms": t_a, "params_per_s": n / t_a * 1e3, "gbs": 6 * n / t_a / 1e6,
+                                 "frac": 6 * n / t_a / 1e6 / peak}
 
 
 def hbm_peak():

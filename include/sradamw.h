@@ -91,6 +91,26 @@ typedef enum { SR_FP8_E4M3 = 0, SR_FP8_E5M2 = 1 } sr_fp8_format;
 sr_status sr_downcast_f32_fp8(const float* src, uint8_t* dst, uint64_t n, sr_fp8_format format, uint64_t seed,
                               uint32_t step, uint32_t tensor_id, uint64_t elem_offset, void* stream);
 
+/* Eq. 2 onto the 4-bit floating-point grid E2M1 (the conclusion names FP8 and FP4): one sign bit, 2
+ * exponent bits with bias 1, one mantissa bit; magnitudes 0, 0.5, 1, 1.5, 2, 3, 4, 6 are codes 0..7,
+ * bit 3 is the sign.  Same rule and same noise as sr_downcast_f32_fp8 with M = 1, bias = 1.  The
+ * format has neither infinity nor NaN: every magnitude at or beyond 6 gives +-6, infinity included,
+ * and a NaN gives the largest magnitude with its sign bit (a choice of this library; the paper is
+ * silent).  src: n FP32 values; dst: (n + 1) / 2 bytes, element 2j in bits 0..3 and element 2j + 1
+ * in bits 4..7 of byte j (the upper half of the last byte is 0 when n is odd). */
+sr_status sr_downcast_f32_fp4(const float* src, uint8_t* dst, uint64_t n, uint64_t seed, uint32_t step,
+                              uint32_t tensor_id, uint64_t elem_offset, void* stream);
+
+/* Eq. 2 (or Eq. 1) in a BF16 accumulation, e.g. of micro-batch gradients (Section 3: every tensor
+ * is BF16): acc[i] <- rounding(acc[i] + scale * g[i]) with the product and the sum each one FP32
+ * operation.  flags = SR_FLAG_SR_P rounds stochastically, flags = 0 to nearest-even; other bits are
+ * rejected.  Noise: rounding slot 3 of the layout above (counter number 4 * (index >> 3) + 3), which
+ * sr_adamw_step never draws, so the same (seed, step, tensor_id) may be shared with the step; the
+ * caller gives every accumulation of one iteration its own `step` value (or seed).  step may be 0.
+ * acc: n BF16 in/out; g: n BF16 or FP32 values per g_dtype, read-only; scale: finite. */
+sr_status sr_accumulate_bf16(uint16_t* acc, const void* g, sr_dtype g_dtype, uint64_t n, float scale, uint32_t flags,
+                             uint64_t seed, uint32_t step, uint32_t tensor_id, uint64_t elem_offset, void* stream);
+
 /* One iteration of Algorithm 1 on a flat buffer of n elements (moment updates, bias-corrected
  * direction with epsilon outside the square root, decoupled weight decay, rounding of x, m, v).
  * p, m, v: BF16 in/out.  g: BF16 or FP32 per g_dtype.  step >= 1 is the 1-based iteration t.

@@ -23,7 +23,7 @@ SR_FLAG_SR_P, SR_FLAG_SR_M, SR_FLAG_SR_V = 1, 2, 4
 SR_FLAGS_DEFAULT = 7
 
 EXPORTS = (
-    "sr_downcast_f32_bf16", "sr_downcast_f32_fp8", "sr_adamw_step", "sr_master_adamw_step", "sr_adamw_step_host", "sr_adamw_step_host_staging_bytes",
+    "sr_downcast_f32_bf16", "sr_downcast_f32_fp8", "sr_downcast_f32_fp4", "sr_accumulate_bf16", "sr_adamw_step", "sr_master_adamw_step", "sr_adamw_step_host", "sr_adamw_step_host_staging_bytes",
     "sr_mt_plan_create", "sr_adamw_multi_tensor",
     "sr_mt_plan_destroy", "sr_mt_plan_total_elements", "grad_sqnorm_workspace_bytes", "grad_sqnorm",
     "grad_sqnorm_static", "grad_sqnorm_static_max_elements",
@@ -78,6 +78,11 @@ def lib() -> ctypes.CDLL:
         L.sr_downcast_f32_bf16.restype = c_int
         L.sr_downcast_f32_fp8.argtypes = [c_void_p, c_void_p, c_uint64, c_int, c_uint64, c_uint32, c_uint32, c_uint64, c_void_p]
         L.sr_downcast_f32_fp8.restype = c_int
+        L.sr_downcast_f32_fp4.argtypes = [c_void_p, c_void_p, c_uint64, c_uint64, c_uint32, c_uint32, c_uint64, c_void_p]
+        L.sr_downcast_f32_fp4.restype = c_int
+        L.sr_accumulate_bf16.argtypes = [c_void_p, c_void_p, c_int, c_uint64, c_float, c_uint32, c_uint64, c_uint32,
+                                         c_uint32, c_uint64, c_void_p]
+        L.sr_accumulate_bf16.restype = c_int
         L.sr_adamw_step.argtypes = [c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_uint64, POINTER(HParams),
                                     c_uint64, c_uint32, c_uint32, c_uint64, c_void_p]
         L.sr_adamw_step.restype = c_int
@@ -164,6 +169,29 @@ def sr_downcast_f32_fp8(src: torch.Tensor, dst: torch.Tensor, seed: int, step: i
     with torch.cuda.device(src.device):
         _check(lib().sr_downcast_f32_fp8(src.data_ptr(), dst.data_ptr(), src.numel(), fmt, seed, step, tensor_id,
                                          elem_offset, _stream(stream)), "sr_downcast_f32_fp8")
+
+
+def sr_downcast_f32_fp4(src: torch.Tensor, dst: torch.Tensor, seed: int, step: int = 0, tensor_id: int = 0,
+                        elem_offset: int = 0, stream=None) -> None:
+    """dst: (n + 1) // 2 bytes (uint8), two E2M1 codes per byte, the even element in the low half."""
+    _want(src, torch.float32, "src"), _want(dst, torch.uint8, "dst")
+    if dst.numel() != (src.numel() + 1) // 2:
+        raise ValueError("size mismatch")
+    with torch.cuda.device(src.device):
+        _check(lib().sr_downcast_f32_fp4(src.data_ptr(), dst.data_ptr(), src.numel(), seed, step, tensor_id, elem_offset,
+                                         _stream(stream)), "sr_downcast_f32_fp4")
+
+
+def sr_accumulate_bf16(acc: torch.Tensor, g: torch.Tensor, scale: float = 1.0, seed: int = 0, step: int = 0,
+                       tensor_id: int = 0, elem_offset: int = 0, stochastic: bool = True, stream=None) -> None:
+    """acc (BF16, in place) <- rounding(acc + scale * g); g is BF16 or FP32."""
+    _want(acc, torch.bfloat16, "acc"), _want(g, g.dtype, "g")
+    if g.numel() != acc.numel():
+        raise ValueError("size mismatch")
+    with torch.cuda.device(acc.device):
+        _check(lib().sr_accumulate_bf16(acc.data_ptr(), g.data_ptr(), _g_dtype(g), acc.numel(), scale,
+                                        SR_FLAG_SR_P if stochastic else 0, seed, step, tensor_id, elem_offset,
+                                        _stream(stream)), "sr_accumulate_bf16")
 
 
 def sr_adamw_step(p: torch.Tensor, g: torch.Tensor, m: torch.Tensor, v: torch.Tensor, hp: HParams, seed: int,

@@ -1,0 +1,102 @@
+// BF16 accumulator with stochastic rounding: acc <- Q_SR(acc + scale * g) (Eq. 2; Section 3 keeps every
+// tensor in BF16, the accumulated gradient included) or the nearest-rounded Q of Eq. 1.
+// FP32 arithmetic in registers, one rounding for the product and one for the sum.  Noise: rounding
+// slot 3 of the group of eight elements (counter number 4 * (index >> 3) + 3), the one the optimizer
+// step leaves unused.  6 bytes per element with BF16 terms (2 + 2 read, 2 written), 8 with FP32 terms.
+
+#include "adamw_body.cuh"
+
+namespace sradamw {
+
+namespace {
+
+constexpr uint32_t kAccumSlot = 3;
+
+template <bool G32>
+__device__ __forceinline__ float term_of(const void* g, uint64_t i) {
+    return G32 ? static_cast<const float*>(g)[i]
+               : __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t*>(g)[i]) << 16);
+}
+
+__device__ __forceinline__ float accumulate(float acc, float g, float scale) {
+    return __fadd_rn(acc, __fmul_rn(scale, g));
+}
+
+// MODE 0: element-wise; 1: 16-byte vectors, per-element noise (offset not a multiple of 8); 2: vectors, grouped
+template <bool G32, bool SR, int MODE>
+__global__ void __launch_bounds__(kBlockThreads)
+k_sr_accumulate(uint16_t* acc, const void* g, uint64_t n, float scale, uint64_t elem_offset, uint32_t tensor_id,
+                uint32_t seed_hi, const __grid_constant__ PhiloxKeys K) {
+    const uint64_t tid = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
+    uint64_t done = 0;
+    if (MODE != 0) {
+        const uint64_t nvec = n >> 3;
+        for (uint64_t vec = tid; vec < nvec; vec += stride) {
+            const uint4 av = ld16(acc, vec);
+            float ge[8];
+            load_grad8<G32>(g, vec, ge);
+            const uint64_t idx0 = elem_offset + (vec << 3);
+            uint4 w = make_uint4(0, 0, 0, 0);
+            if (SR && MODE == 2)
+                w = philox4x32_10(static_cast<uint32_t>(idx0 >> 1) | kAccumSlot, static_cast<uint32_t>(idx0 >> 33), tensor_id,
+                                  seed_hi, K);
+            uint32_t o[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t aw = word_of(av, j);
+                const float s0 = accumulate(bf16_lo(aw), ge[2 * j], scale);
+                const float s1 = accumulate(bf16_hi(aw), ge[2 * j + 1], scale);
+                uint32_t r0, r1;
+                if (!SR || MODE == 2) {
+                    r0 = round_sum_word_nan_safe<SR, false>(s0, word_of(w, j));
+                    r1 = round_sum_word_nan_safe<SR, true>(s1, word_of(w, j));
+                } else {
+                    r0 = round_sum_r16_nan_safe<true>(s0, noise_of_element(idx0 + 2 * j, kAccumSlot, tensor_id, seed_hi, K));
+                    r1 = round_sum_r16_nan_safe<true>(s1, noise_of_element(idx0 + 2 * j + 1, kAccumSlot, tensor_id, seed_hi, K));
+                }
+                o[j] = pack_top_halves(r0, r1);
+            }
+            st16(acc, vec, make_uint4(o[0], o[1], o[2], o[3]));
+        }
+        done = nvec << 3;
+    }
+    for (uint64_t i = done + tid; i < n; i += stride) {
+        const float s = accumulate(__uint_as_float(static_cast<uint32_t>(acc[i]) << 16), term_of<G32>(g, i), scale);
+        const uint32_t r = SR ? noise_of_element(elem_offset + i, kAccumSlot, tensor_id, seed_hi, K) : 0u;
+        acc[i] = static_cast<uint16_t>(round_sum_r16_nan_safe<SR>(s, r) >> 16);
+    }
+}
+
+template <bool G32, bool SR, int MODE>
+cudaError_t launch_accum_mode(uint16_t* acc, const void* g, uint64_t n, float scale, uint64_t elem_offset,
+                              uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev,
+                              cudaStream_t stream) {
+    auto k = k_sr_accumulate<G32, SR, MODE>;
+    const uint64_t items = MODE == 0 ? n : (n >> 3) + 8;
+    k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(acc, g, n, scale, elem_offset, tensor_id, seed_hi, K);
+    return cudaGetLastError();
+}
+
+template <bool G32, bool SR>
+cudaError_t launch_accum_t(uint16_t* acc, const void* g, uint64_t n, float scale, uint64_t elem_offset, uint32_t tensor_id,
+                           uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev, cudaStream_t stream) {
+    if (!(aligned16(acc) && aligned16(g)))
+        return launch_accum_mode<G32, SR, 0>(acc, g, n, scale, elem_offset, tensor_id, seed_hi, K, dev, stream);
+    if (SR && (elem_offset & 7u) != 0)
+        return launch_accum_mode<G32, SR, 1>(acc, g, n, scale, elem_offset, tensor_id, seed_hi, K, dev, stream);
+    return launch_accum_mode<G32, SR, 2>(acc, g, n, scale, elem_offset, tensor_id, seed_hi, K, dev, stream);
+}
+
+}  // namespace
+
+cudaError_t launch_accumulate(uint16_t* acc, const void* g, bool g_f32, uint64_t n, float scale, bool stochastic,
+                              uint64_t elem_offset, uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K,
+                              const DeviceInfo& dev, cudaStream_t stream) {
+#define SR_ACC(G, S) launch_accum_t<G, S>(acc, g, n, scale, elem_offset, tensor_id, seed_hi, K, dev, stream)
+    if (g_f32) return stochastic ? SR_ACC(true, true) : SR_ACC(true, false);
+    return stochastic ? SR_ACC(false, true) : SR_ACC(false, false);
+#undef SR_ACC
+}
+
+}  // namespace sradamw

@@ -137,6 +137,33 @@ sr_status sr_downcast_f32_fp8(const float* src, uint8_t* dst, uint64_t n, sr_fp8
     return e == cudaSuccess ? SR_OK : cuda_fail(e);
 }
 
+sr_status sr_downcast_f32_fp4(const float* src, uint8_t* dst, uint64_t n, uint64_t seed, uint32_t step,
+                              uint32_t tensor_id, uint64_t elem_offset, void* stream) {
+    if (n == 0) return SR_OK;
+    if (src == nullptr || dst == nullptr) return SR_ERR_INVALID_ARG;
+    DeviceInfo dev;
+    sr_status st = current_device(&dev);
+    if (st != SR_OK) return st;
+    const cudaError_t e = launch_downcast_fp4(src, dst, n, elem_offset, tensor_id, static_cast<uint32_t>(seed >> 32),
+                                              make_keys(seed, step), dev, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SR_OK : cuda_fail(e);
+}
+
+sr_status sr_accumulate_bf16(uint16_t* acc, const void* g, sr_dtype g_dtype, uint64_t n, float scale, uint32_t flags,
+                             uint64_t seed, uint32_t step, uint32_t tensor_id, uint64_t elem_offset, void* stream) {
+    if (g_dtype != SR_DT_BF16 && g_dtype != SR_DT_F32) return SR_ERR_INVALID_ARG;
+    if ((flags & ~static_cast<uint32_t>(SR_FLAG_SR_P)) != 0 || !std::isfinite(scale)) return SR_ERR_INVALID_ARG;
+    if (n == 0) return SR_OK;
+    if (acc == nullptr || g == nullptr) return SR_ERR_INVALID_ARG;
+    DeviceInfo dev;
+    sr_status st = current_device(&dev);
+    if (st != SR_OK) return st;
+    const cudaError_t e = launch_accumulate(acc, g, g_dtype == SR_DT_F32, n, scale, (flags & SR_FLAG_SR_P) != 0, elem_offset,
+                                            tensor_id, static_cast<uint32_t>(seed >> 32), make_keys(seed, step), dev,
+                                            static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SR_OK : cuda_fail(e);
+}
+
 sr_status sr_adamw_step(uint16_t* p, const void* g, sr_dtype g_dtype, uint16_t* m, uint16_t* v, uint64_t n,
                         const sr_adamw_hparams* hp, uint64_t seed, uint32_t step, uint32_t tensor_id,
                         uint64_t elem_offset, void* stream) {

@@ -1,6 +1,7 @@
-// Stochastic-rounding cast FP32 -> FP8 (E4M3 / E5M2): Eq. 2 on the 8-bit grids, the extension the
-// paper's conclusion names.  5 bytes per element (4 read, 1 written).  32 noise bits per element,
-// one Philox call per four consecutive elements (counter number = index >> 2, word = index & 3).
+// Stochastic-rounding casts FP32 -> FP8 (E4M3 / E5M2) and FP32 -> FP4 (E2M1): Eq. 2 on the 8-bit and
+// 4-bit grids, the extension the paper's conclusion names.  5 bytes per element (4 read, 1 written)
+// for FP8, 4.5 for FP4 (two codes per byte).  32 noise bits per element, one Philox call per four
+// consecutive elements (counter number = index >> 2, word = index & 3).
 
 #include "adamw_body.cuh"
 
@@ -8,13 +9,15 @@ namespace sradamw {
 
 namespace {
 
-template <bool E5M2>
-struct Fp8 {
-    static constexpr int M = E5M2 ? 2 : 3;
-    static constexpr int kBias = E5M2 ? 15 : 7;
-    static constexpr uint32_t kMaxCode = E5M2 ? 0x7Bu : 0x7Eu;
-    static constexpr uint32_t kMaxBits = E5M2 ? 0x47600000u : 0x43E00000u;   // 57344.0f, 448.0f
-    static constexpr uint32_t kInfCode = E5M2 ? 0x7Cu : 0x7Eu;               // E4M3 has no infinity
+// FMT 0: E4M3, 1: E5M2, 2: E2M1
+constexpr int kE4M3 = 0, kE5M2 = 1, kE2M1 = 2;
+
+template <int FMT>
+struct Small {
+    static constexpr int M = FMT == kE5M2 ? 2 : FMT == kE4M3 ? 3 : 1;
+    static constexpr int kBias = FMT == kE5M2 ? 15 : FMT == kE4M3 ? 7 : 1;
+    static constexpr uint32_t kMaxCode = FMT == kE5M2 ? 0x7Bu : FMT == kE4M3 ? 0x7Eu : 0x7u;   // 57344, 448, 6
+    static constexpr uint32_t kInfCode = 0x7Cu;                              // E5M2 only: the others have no infinity
     static constexpr uint32_t kMinBiasedExp = 127 + 1 - kBias;               // FP32 exponent field of the smallest normal level
 };
 
@@ -24,10 +27,11 @@ struct Fp8 {
 // (mant * 2^32) >> D holds k in its high word and floor(f * 2^32) in its low word; both are zero once
 // D >= 56, which also covers zero and the FP32 subnormals (their exponent field is 0, so D is far
 // beyond 56 whatever their significand).  The code of level k' is ((Eq + bias - 1) << M) + k' for
-// subnormal and normal levels alike; the clamp saturates every finite |x| beyond the largest level.
-template <bool E5M2>
+// subnormal and normal levels alike; the clamp saturates every finite |x| beyond the largest level
+// (and, for E2M1, infinity and NaN as well: their exponent field puts the code far beyond the clamp).
+template <int FMT>
 __device__ __forceinline__ uint32_t sr_fp8_magnitude(uint32_t abits, uint32_t r) {
-    using F = Fp8<E5M2>;
+    using F = Small<FMT>;
     const uint32_t e = abits >> 23;                                    // biased FP32 exponent
     const uint32_t mant = (abits & 0x7FFFFFu) | 0x800000u;
     const uint32_t eq = e < F::kMinBiasedExp ? F::kMinBiasedExp : e;   // Eq + 127
@@ -38,15 +42,27 @@ __device__ __forceinline__ uint32_t sr_fp8_magnitude(uint32_t abits, uint32_t r)
     const uint32_t threshold = dropped > 32u ? __funnelshift_rc(mant, 0u, dropped - 32u) : low;
     uint32_t code = ((eq - 127u + F::kBias - 1u) << F::M) + k + (r < threshold ? 1u : 0u);
     code = code > F::kMaxCode ? F::kMaxCode : code;
-    if (E5M2) code = abits == 0x7F800000u ? F::kInfCode : code;
+    if (FMT == kE2M1) return code;
+    if (FMT == kE5M2) code = abits == 0x7F800000u ? F::kInfCode : code;
     return abits > 0x7F800000u ? 0x7Fu : code;                         // NaN -> 0x7F (its sign is dropped below)
 }
 
-template <bool E5M2>
+template <int FMT>
 __device__ __forceinline__ uint32_t sr_fp8_code(uint32_t fbits, uint32_t r) {
     const uint32_t abits = fbits & 0x7FFFFFFFu;
     const uint32_t sign = abits > 0x7F800000u ? 0u : ((fbits >> 24) & 0x80u);
-    return sign | sr_fp8_magnitude<E5M2>(abits, r);
+    return sign | sr_fp8_magnitude<FMT>(abits, r);
+}
+
+// E2M1: sign in bit 3 (kept for NaN too), magnitude code in bits 0..2
+__device__ __forceinline__ uint32_t sr_fp4_code(uint32_t fbits, uint32_t r) {
+    return ((fbits >> 28) & 0x8u) | sr_fp8_magnitude<kE2M1>(fbits & 0x7FFFFFFFu, r);
+}
+
+// four values -> four 4-bit codes in bits 0..15 (element j in bits 4j..4j+3)
+__device__ __forceinline__ uint32_t cast4_fp4(const uint4 x, const uint4 w) {
+    const uint32_t n0 = sr_fp4_code(x.x, w.x), n1 = sr_fp4_code(x.y, w.y), n2 = sr_fp4_code(x.z, w.z), n3 = sr_fp4_code(x.w, w.w);
+    return (n1 * 16u + n0) + (n3 * 16u + n2) * 256u;
 }
 
 __device__ __forceinline__ uint32_t noise32_of_element(uint64_t idx, uint32_t c2, uint32_t c3, const PhiloxKeys& K) {
@@ -57,11 +73,11 @@ __device__ __forceinline__ uint32_t noise32_of_element(uint64_t idx, uint32_t c2
 }
 
 // four values -> four bytes; the four sign bits are gathered with two byte permutes
-template <bool E5M2>
+template <int FMT>
 __device__ __forceinline__ uint32_t cast4(const uint4 x, const uint4 w) {
     const uint32_t ax = x.x & 0x7FFFFFFFu, ay = x.y & 0x7FFFFFFFu, az = x.z & 0x7FFFFFFFu, aw = x.w & 0x7FFFFFFFu;
-    const uint32_t m0 = sr_fp8_magnitude<E5M2>(ax, w.x), m1 = sr_fp8_magnitude<E5M2>(ay, w.y);
-    const uint32_t m2 = sr_fp8_magnitude<E5M2>(az, w.z), m3 = sr_fp8_magnitude<E5M2>(aw, w.w);
+    const uint32_t m0 = sr_fp8_magnitude<FMT>(ax, w.x), m1 = sr_fp8_magnitude<FMT>(ay, w.y);
+    const uint32_t m2 = sr_fp8_magnitude<FMT>(az, w.z), m3 = sr_fp8_magnitude<FMT>(aw, w.w);
     const uint32_t mags = __byte_perm(__byte_perm(m0, m1, 0x0040), __byte_perm(m2, m3, 0x0040), 0x5410);
     const uint32_t tops = __byte_perm(__byte_perm(x.x, x.y, 0x0073), __byte_perm(x.z, x.w, 0x0073), 0x5410);
     // a NaN code (0x7F) keeps no sign: mask the sign bit where the magnitude byte is 0x7F with all of bits 0..6 set
@@ -71,7 +87,7 @@ __device__ __forceinline__ uint32_t cast4(const uint4 x, const uint4 w) {
 
 // VEC: 16 elements per thread-iteration (4 x 16-byte loads, 1 x 16-byte store); needs both buffers
 // 16-byte aligned and elem_offset a multiple of 4 (whole noise groups).
-template <bool E5M2, bool VEC>
+template <int FMT, bool VEC>
 __global__ void __launch_bounds__(kBlockThreads)
 k_sr_downcast_fp8(const float* __restrict__ src, uint8_t* __restrict__ dst, uint64_t n, uint64_t elem_offset,
                   uint32_t tensor_id, uint32_t seed_hi, const __grid_constant__ PhiloxKeys K) {
@@ -85,22 +101,57 @@ k_sr_downcast_fp8(const float* __restrict__ src, uint8_t* __restrict__ dst, uint
             const uint64_t number = (elem_offset + (vec << 4)) >> 2;
             const uint32_t c0 = static_cast<uint32_t>(number), c1 = static_cast<uint32_t>(number >> 32);
             uint4 o;
-            o.x = cast4<E5M2>(a, philox4x32_10(c0, c1, tensor_id, seed_hi, K));
-            o.y = cast4<E5M2>(b, philox4x32_10(c0 + 1, c1, tensor_id, seed_hi, K));
-            o.z = cast4<E5M2>(c, philox4x32_10(c0 + 2, c1, tensor_id, seed_hi, K));
-            o.w = cast4<E5M2>(d, philox4x32_10(c0 + 3, c1, tensor_id, seed_hi, K));
+            o.x = cast4<FMT>(a, philox4x32_10(c0, c1, tensor_id, seed_hi, K));
+            o.y = cast4<FMT>(b, philox4x32_10(c0 + 1, c1, tensor_id, seed_hi, K));
+            o.z = cast4<FMT>(c, philox4x32_10(c0 + 2, c1, tensor_id, seed_hi, K));
+            o.w = cast4<FMT>(d, philox4x32_10(c0 + 3, c1, tensor_id, seed_hi, K));
             st16(dst, vec, o);
         }
         done = nvec << 4;
     }
     for (uint64_t i = done + tid; i < n; i += stride)
-        dst[i] = static_cast<uint8_t>(sr_fp8_code<E5M2>(__float_as_uint(src[i]), noise32_of_element(elem_offset + i, tensor_id, seed_hi, K)));
+        dst[i] = static_cast<uint8_t>(sr_fp8_code<FMT>(__float_as_uint(src[i]), noise32_of_element(elem_offset + i, tensor_id, seed_hi, K)));
 }
 
-template <bool E5M2, bool VEC>
+// E2M1, two codes per byte (element 2j in bits 0..3 of byte j).  VEC: 16 elements per
+// thread-iteration (4 x 16-byte loads, one 8-byte store); needs src 16-byte and dst 8-byte aligned
+// and elem_offset a multiple of 16.  The rest (and everything without VEC) goes byte by byte, one
+// thread per output byte.
+template <bool VEC>
+__global__ void __launch_bounds__(kBlockThreads)
+k_sr_downcast_fp4(const float* __restrict__ src, uint8_t* __restrict__ dst, uint64_t n, uint64_t elem_offset,
+                  uint32_t tensor_id, uint32_t seed_hi, const __grid_constant__ PhiloxKeys K) {
+    const uint64_t tid = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
+    uint64_t done = 0;
+    if (VEC) {
+        const uint64_t nvec = n >> 4;
+        for (uint64_t vec = tid; vec < nvec; vec += stride) {
+            const uint4 a = ld16(src, 4 * vec), b = ld16(src, 4 * vec + 1), c = ld16(src, 4 * vec + 2), d = ld16(src, 4 * vec + 3);
+            const uint64_t number = (elem_offset + (vec << 4)) >> 2;
+            const uint32_t c0 = static_cast<uint32_t>(number), c1 = static_cast<uint32_t>(number >> 32);
+            const uint32_t lo = cast4_fp4(a, philox4x32_10(c0, c1, tensor_id, seed_hi, K)) |
+                                (cast4_fp4(b, philox4x32_10(c0 + 1, c1, tensor_id, seed_hi, K)) << 16);
+            const uint32_t hi = cast4_fp4(c, philox4x32_10(c0 + 2, c1, tensor_id, seed_hi, K)) |
+                                (cast4_fp4(d, philox4x32_10(c0 + 3, c1, tensor_id, seed_hi, K)) << 16);
+            __stcs(reinterpret_cast<uint2*>(dst) + vec, make_uint2(lo, hi));
+        }
+        done = nvec << 4;
+    }
+    const uint64_t nbytes = (n + 1) >> 1;
+    for (uint64_t j = (done >> 1) + tid; j < nbytes; j += stride) {
+        const uint64_t i0 = 2 * j, i1 = i0 + 1;
+        uint32_t byte = sr_fp4_code(__float_as_uint(src[i0]), noise32_of_element(elem_offset + i0, tensor_id, seed_hi, K));
+        if (i1 < n)
+            byte |= sr_fp4_code(__float_as_uint(src[i1]), noise32_of_element(elem_offset + i1, tensor_id, seed_hi, K)) << 4;
+        dst[j] = static_cast<uint8_t>(byte);
+    }
+}
+
+template <int FMT, bool VEC>
 cudaError_t launch_fp8_t(const float* src, uint8_t* dst, uint64_t n, uint64_t elem_offset, uint32_t tensor_id,
                          uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev, cudaStream_t stream) {
-    auto k = k_sr_downcast_fp8<E5M2, VEC>;
+    auto k = k_sr_downcast_fp8<FMT, VEC>;
     const uint64_t items = VEC ? (n >> 4) + 16 : n;
     k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(src, dst, n, elem_offset, tensor_id, seed_hi, K);
     return cudaGetLastError();
@@ -113,10 +164,24 @@ cudaError_t launch_downcast_fp8(const float* src, uint8_t* dst, uint64_t n, bool
                                 cudaStream_t stream) {
     // the low word of the group number must not wrap inside a 16-element vector: offset multiple of 16
     const bool vec = aligned16(src) && aligned16(dst) && (elem_offset & 15u) == 0;
-    if (e5m2) return vec ? launch_fp8_t<true, true>(src, dst, n, elem_offset, tensor_id, seed_hi, K, dev, stream)
-                         : launch_fp8_t<true, false>(src, dst, n, elem_offset, tensor_id, seed_hi, K, dev, stream);
-    return vec ? launch_fp8_t<false, true>(src, dst, n, elem_offset, tensor_id, seed_hi, K, dev, stream)
-               : launch_fp8_t<false, false>(src, dst, n, elem_offset, tensor_id, seed_hi, K, dev, stream);
+    if (e5m2) return vec ? launch_fp8_t<kE5M2, true>(src, dst, n, elem_offset, tensor_id, seed_hi, K, dev, stream)
+                         : launch_fp8_t<kE5M2, false>(src, dst, n, elem_offset, tensor_id, seed_hi, K, dev, stream);
+    return vec ? launch_fp8_t<kE4M3, true>(src, dst, n, elem_offset, tensor_id, seed_hi, K, dev, stream)
+               : launch_fp8_t<kE4M3, false>(src, dst, n, elem_offset, tensor_id, seed_hi, K, dev, stream);
+}
+
+cudaError_t launch_downcast_fp4(const float* src, uint8_t* dst, uint64_t n, uint64_t elem_offset, uint32_t tensor_id,
+                                uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev, cudaStream_t stream) {
+    const bool vec = aligned16(src) && (reinterpret_cast<uintptr_t>(dst) & 7u) == 0 && (elem_offset & 15u) == 0;
+    const uint64_t items = (vec ? (n >> 4) + 16 : (n + 1) >> 1);
+    if (vec) {
+        auto k = k_sr_downcast_fp4<true>;
+        k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(src, dst, n, elem_offset, tensor_id, seed_hi, K);
+    } else {
+        auto k = k_sr_downcast_fp4<false>;
+        k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(src, dst, n, elem_offset, tensor_id, seed_hi, K);
+    }
+    return cudaGetLastError();
 }
 
 }  // namespace sradamw

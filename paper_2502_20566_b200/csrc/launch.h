@@ -78,6 +78,13 @@ cudaError_t launch_downcast_fp8(const float* src, uint8_t* dst, uint64_t n, bool
                                 uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev,
                                 cudaStream_t stream);
 
+cudaError_t launch_downcast_fp4(const float* src, uint8_t* dst, uint64_t n, uint64_t elem_offset, uint32_t tensor_id,
+                                uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev, cudaStream_t stream);
+
+cudaError_t launch_accumulate(uint16_t* acc, const void* g, bool g_f32, uint64_t n, float scale, bool stochastic,
+                              uint64_t elem_offset, uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K,
+                              const DeviceInfo& dev, cudaStream_t stream);
+
 cudaError_t launch_master_adamw(float* p, uint16_t* p16, const void* g, bool g_f32, float* m, float* v, uint64_t n,
                                 const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream);
 

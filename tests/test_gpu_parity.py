@@ -667,3 +667,117 @@ def test_fp8_cast_is_unbiased_over_seeds(env):
         assert torch.all((vals.abs() == lo) | (vals.abs() == lo + delta))      # the two neighbouring levels only
         sigma = delta * torch.sqrt(f * (1 - f) / seeds)
         assert torch.all((vals.mean(dim=0) - x.double()).abs() <= 6 * sigma + 1e-300)
+
+
+# ---------------------------------------------------------------------------------------------
+# FP4 (E2M1) stochastic-rounding cast
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n,offset,shift", [(0, 0, 0), (1, 0, 0), (3, 0, 0), (1 << 22, 0, 0), ((1 << 20) + 13, 16 * 77, 0),
+                                            (70001, 5, 0), (70002, 32, 4), (70001, 48, 3), (5000, (1 << 34) - 64, 0)])
+def test_fp4_cast_bit_exact(env, n, offset, shift):
+    """shift moves the source by `shift` floats and the destination by `shift` bytes (unaligned buffers)."""
+    oracle, binding, synth, dev = env
+    src = synth.downcast_mix(n + shift, 23, dev)[shift:]
+    if n > 1000:                                   # most of the mix lies outside the E2M1 range: add in-range values
+        k = 3 * n // 4
+        scale = torch.pow(10.0, torch.rand(k, device=dev, generator=torch.Generator(device=dev).manual_seed(4)) * 5 - 4)
+        src[:k] = torch.randn(k, device=dev, generator=torch.Generator(device=dev).manual_seed(3)) * scale
+    nbytes = (n + 1) // 2
+    dst = torch.full((nbytes + shift + 16,), 0xEE, dtype=torch.uint8, device=dev)
+    out = dst[shift:shift + nbytes]
+    binding.sr_downcast_f32_fp4(src, out, seed=(9 << 32) | 5, step=2, tensor_id=7, elem_offset=offset)
+    torch.cuda.synchronize()
+    want = oracle.sr_downcast_fp4(src.cpu().numpy().copy(), (9 << 32) | 5, 2, 7, offset)
+    got = out.cpu().numpy()
+    assert int(np.count_nonzero(got != want)) == 0
+    assert bool((dst[shift + nbytes:] == 0xEE).all()) and bool((dst[:shift] == 0xEE).all())   # nothing written outside
+    if n > 1000:
+        codes = np.concatenate([got & 0xF, got >> 4])
+        assert len(np.unique(codes)) == 16         # every code of the grid occurs
+
+
+def test_fp4_cast_is_unbiased_over_seeds(env):
+    """Mean over 2048 seeds of 4096 values inside (-6, 6): within 6 sigma of x, sigma^2 = Delta^2 f (1 - f) / seeds."""
+    _, binding, _, dev = env
+    k, seeds = 4096, 2048
+    gen = torch.Generator(device=dev).manual_seed(12)
+    x = (torch.rand(k, device=dev, generator=gen) * 2 - 1) * 5.9 * torch.pow(2.0, -torch.rand(k, device=dev, generator=gen) * 6)
+    outs = torch.empty((seeds, k // 2), dtype=torch.uint8, device=dev)
+    for s in range(seeds):
+        binding.sr_downcast_f32_fp4(x, outs[s], seed=s)
+    torch.cuda.synchronize()
+    table = torch.tensor([0, .5, 1, 1.5, 2, 3, 4, 6, -0.0, -.5, -1, -1.5, -2, -3, -4, -6], dtype=torch.float64, device=dev)
+    codes = torch.stack([outs & 0xF, outs >> 4], dim=2).reshape(seeds, k).long()
+    vals = table[codes]
+    a = x.double().abs()
+    eq = torch.clamp(torch.floor(torch.log2(a)), min=0)                       # binade that sets the spacing (bias 1)
+    delta = torch.exp2(eq - 1)
+    lo = torch.floor(a / delta) * delta
+    f = (a - lo) / delta
+    assert torch.all((vals.abs() == lo) | (vals.abs() == lo + delta))
+    sigma = delta * torch.sqrt(f * (1 - f) / seeds)
+    assert torch.all((vals.mean(dim=0) - x.double()).abs() <= 6 * sigma + 1e-300)
+
+
+# ---------------------------------------------------------------------------------------------
+# BF16 accumulation with stochastic rounding
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("g_dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("stochastic", [True, False])
+@pytest.mark.parametrize("n,offset,shift", [(0, 0, 0), (5, 0, 0), (1 << 22, 0, 0), ((1 << 20) + 11, 8 * 123, 0), (70001, 5, 0),
+                                            (70001, 64, 1), (4096, (1 << 36) - 1024, 0)])
+def test_accumulate_bit_exact(env, g_dtype, stochastic, n, offset, shift):
+    oracle, binding, synth, dev = env
+    p, g, m, v = synth.adamw_state(n + shift, 57, dev, g_dtype=g_dtype, outlier_fraction=0.01)
+    acc, g = m[shift:], g[shift:]                   # a BF16 accumulator of gradient-like magnitude
+    if n > 100:
+        acc[:8] = torch.tensor([0.0, -0.0, float("inf"), float("-inf"), float("nan"), 3.3895e38, 1e-40, 1.0], device=dev).bfloat16()
+        g[:8] = torch.tensor([-0.0, 0.0, 1.0, float("inf"), 1.0, 3e38, 1e-40, -1.0], device=dev).to(g_dtype)
+    want = bits(acc)
+    gh = host_g(g)
+    for micro in range(3):
+        binding.sr_accumulate_bf16(acc, g, 0.25, seed=(3 << 32) | 77, step=10 + micro, tensor_id=5, elem_offset=offset,
+                                   stochastic=stochastic)
+        oracle.sr_accumulate(want, gh, 0.25, (3 << 32) | 77, 10 + micro, 5, offset, stochastic)
+    torch.cuda.synchronize()
+    assert mismatches(bits(acc), want) == 0
+    if shift:
+        assert mismatches(bits(m[:shift]), bits(synth.adamw_state(n + shift, 57, dev, g_dtype=g_dtype, outlier_fraction=0.01)[2][:shift])) == 0
+
+
+def test_accumulate_stagnation_and_mean(env):
+    """Section 2.1 on the device: terms of a quarter spacing never move a nearest-rounded accumulator; under
+    stochastic rounding the mean over many accumulators follows the exact sum."""
+    _, binding, _, dev = env
+    n, steps, u = 1 << 16, 256, 2.0 ** -9
+    g = torch.full((n,), u, dtype=torch.float32, device=dev)
+    near = torch.ones(n, dtype=torch.bfloat16, device=dev)
+    sr = torch.ones(n, dtype=torch.bfloat16, device=dev)
+    for t in range(1, steps + 1):
+        binding.sr_accumulate_bf16(near, g, 1.0, seed=5, step=t, stochastic=False)
+        binding.sr_accumulate_bf16(sr, g, 1.0, seed=5, step=t, stochastic=True)
+    torch.cuda.synchronize()
+    assert bool((near == 1.0).all())
+    vals = sr.double()
+    sigma = (steps * (2.0 ** -7) ** 2 / 4) ** 0.5
+    assert abs(float(vals.mean()) - (1.0 + steps * u)) < 6 * sigma / n ** 0.5
+    assert float(vals.std()) > 0.2 * sigma
+
+
+def test_accumulate_noise_is_disjoint_from_the_step(env):
+    """The accumulation draws rounding slot 3, the step slots 0..2: with the same (seed, step, tensor_id) the
+    up/down decisions of the two calls on identical fractions are not the same."""
+    oracle, binding, _, dev = env
+    n = 1 << 16
+    x = torch.full((n,), 1.0 + 2.0 ** -9, dtype=torch.float32, device=dev)    # fraction 1/4 of a BF16 spacing
+    cast = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    binding.sr_downcast_f32_bf16(x, cast, seed=8, step=4, tensor_id=1)       # slot 0
+    acc = torch.ones(n, dtype=torch.bfloat16, device=dev)
+    binding.sr_accumulate_bf16(acc, torch.full((n,), 2.0 ** -9, dtype=torch.float32, device=dev), 1.0, seed=8, step=4, tensor_id=1)
+    torch.cuda.synchronize()
+    up_cast, up_acc = (cast > 1.0), (acc > 1.0)
+    assert abs(float(up_cast.float().mean()) - 0.25) < 0.02 and abs(float(up_acc.float().mean()) - 0.25) < 0.02
+    both = float((up_cast & up_acc).float().mean())
+    assert abs(both - 0.0625) < 0.01                                           # independent: P(both) = 1/16
