@@ -413,6 +413,47 @@ def test_clipped_shard_full_size(env):
     assert _clipped_shard(env, n, 3) == (0, 0, 0)
 
 
+def test_clipped_sequence_in_a_cuda_graph(env):
+    """accumulate -> norm -> clip factor -> step captured once on a stream and replayed: no call allocates,
+    synchronises or reads back, so the whole sequence is capturable; every replay matches the oracle."""
+    oracle, binding, synth, dev = env
+    n = (1 << 21) + 24
+    p, g, m, v = synth.adamw_state(n, 23, dev, g_dtype=torch.float32, outlier_fraction=0.01)
+    acc = torch.zeros(n, dtype=torch.bfloat16, device=dev)
+    ws = torch.empty(max(1, binding.grad_sqnorm_workspace_bytes(n) // 8), dtype=torch.float64, device=dev)
+    S = torch.zeros(1, dtype=torch.float64, device=dev)
+    gs = torch.zeros(1, dtype=torch.float32, device=dev)
+    hp = binding.hparams(**HP, grad_scale_dev=gs)
+    pb, gb, mb, vb, ab = bits(p), host_g(g), bits(m), bits(v), bits(acc)
+
+    def sequence():
+        binding.sr_accumulate_bf16(acc, g, 0.5, seed=1234, step=7, tensor_id=2)
+        binding.grad_sqnorm(acc, S, ws)
+        binding.sr_clip_scale(S, 1.0, 1.0, gs)
+        binding.sr_adamw_step(p, acc, m, v, hp, 1234, 7, 2, 0)
+
+    binding.lib()                                   # library and device info are set up before the capture
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        sequence()                                  # warm-up outside the capture (replayed on the oracle as well)
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        sequence()
+    replays = 3
+    for _ in range(replays):
+        graph.replay()
+    torch.cuda.synchronize()
+    for _ in range(1 + replays):
+        oracle.sr_accumulate(ab, gb, 0.5, 1234, 7, 2, 0, True)
+        S_o = oracle.sqnorm(ab)
+        oracle.adamw_step(pb, ab, mb, vb, oracle.hparams(**HP), 1234, 7, 2, 0, oracle.clip_scale(S_o, 1.0, 1.0))
+    assert float(S.item()).hex() == S_o.hex()
+    assert mismatches(bits(acc), ab) == 0
+    assert (mismatches(bits(p), pb), mismatches(bits(m), mb), mismatches(bits(v), vb)) == (0, 0, 0)
+
+
 # ---------------------------------------------------------------------------------------------
 # tensor list
 # ---------------------------------------------------------------------------------------------
