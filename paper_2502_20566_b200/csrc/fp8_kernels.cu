@@ -17,34 +17,35 @@ struct Small {
     static constexpr int M = FMT == kE5M2 ? 2 : FMT == kE4M3 ? 3 : 1;
     static constexpr int kBias = FMT == kE5M2 ? 15 : FMT == kE4M3 ? 7 : 1;
     static constexpr uint32_t kMaxCode = FMT == kE5M2 ? 0x7Bu : FMT == kE4M3 ? 0x7Eu : 0x7u;   // 57344, 448, 6
+    static constexpr uint32_t kMaxBits = FMT == kE5M2 ? 0x47600000u : FMT == kE4M3 ? 0x43E00000u : 0x40C00000u;   // as FP32
     static constexpr uint32_t kInfCode = 0x7Cu;                              // E5M2 only: the others have no infinity
     static constexpr uint32_t kMinBiasedExp = 127 + 1 - kBias;               // FP32 exponent field of the smallest normal level
 };
 
 // The magnitude code of one value (sign handled by the caller).  a = |x| lies in the binade
 // Eq = max(E, 1 - bias); y = a / 2^(Eq - M) = k + f; move to level k + 1 iff r < floor(f * 2^32).
-// In integers: with the 24-bit significand `mant` of a and D = (23 - M) + (Eq - E) dropped bits,
-// (mant * 2^32) >> D holds k in its high word and floor(f * 2^32) in its low word; both are zero once
-// D >= 56, which also covers zero and the FP32 subnormals (their exponent field is 0, so D is far
-// beyond 56 whatever their significand).  The code of level k' is ((Eq + bias - 1) << M) + k' for
-// subnormal and normal levels alike; the clamp saturates every finite |x| beyond the largest level
-// (and, for E2M1, infinity and NaN as well: their exponent field puts the code far beyond the clamp).
+// Evaluated with exact FP32 operations, which keeps most of the work off the integer pipe that
+// bounds this kernel: y = a * 2^(M - Eq) is a scaling by a power of two (exact, subnormal a
+// included; y < 2^(M+1)); adding 2^23 with rounding toward zero leaves k in the low bits of the sum;
+// f = y - k is exact; f * 2^32 < 2^32 is exact and its truncation to an integer is the threshold.
+// The code of level k' is ((Eq + bias - 1) << M) + k' for subnormal and normal levels alike.
+// Magnitudes at or beyond the largest level (infinity and NaN included, whose y is meaningless)
+// are replaced at the end.
 template <int FMT>
 __device__ __forceinline__ uint32_t sr_fp8_magnitude(uint32_t abits, uint32_t r) {
     using F = Small<FMT>;
-    const uint32_t e = abits >> 23;                                    // biased FP32 exponent
-    const uint32_t mant = (abits & 0x7FFFFFu) | 0x800000u;
-    const uint32_t eq = e < F::kMinBiasedExp ? F::kMinBiasedExp : e;   // Eq + 127
-    const uint32_t dropped = (23u - F::M) + (eq - e);                  // 20 or 21 in the normal range
-    // (mant : 0) >> dropped with clamped funnel shifts (a shift of 32 or more yields what is left)
-    const uint32_t k = __funnelshift_rc(mant, 0u, dropped);
-    const uint32_t low = __funnelshift_rc(0u, mant, dropped);
-    const uint32_t threshold = dropped > 32u ? __funnelshift_rc(mant, 0u, dropped - 32u) : low;
-    uint32_t code = ((eq - 127u + F::kBias - 1u) << F::M) + k + (r < threshold ? 1u : 0u);
-    code = code > F::kMaxCode ? F::kMaxCode : code;
+    const uint32_t e = abits >> 23;                                            // biased FP32 exponent
+    const uint32_t eqb = e < F::kMinBiasedExp ? F::kMinBiasedExp : e;          // Eq + 127
+    const float scale = __uint_as_float(((254u + F::M) << 23) - (eqb << 23));  // 2^(M - Eq)
+    const float y = __fmul_rn(__uint_as_float(abits), scale);
+    const float t = __fadd_rz(y, 8388608.0f);                                  // 2^23 + k
+    const float f = __fsub_rn(y, __fsub_rn(t, 8388608.0f));
+    const uint32_t threshold = __float2uint_rz(__fmul_rn(f, 4294967296.0f));
+    uint32_t code = (eqb << F::M) + __float_as_uint(t) - (0x4B000000u + (F::kMinBiasedExp << F::M)) + (r < threshold ? 1u : 0u);
+    code = abits >= F::kMaxBits ? F::kMaxCode : code;
     if (FMT == kE2M1) return code;
     if (FMT == kE5M2) code = abits == 0x7F800000u ? F::kInfCode : code;
-    return abits > 0x7F800000u ? 0x7Fu : code;                         // NaN -> 0x7F (its sign is dropped below)
+    return abits > 0x7F800000u ? 0x7Fu : code;                                 // NaN -> 0x7F (its sign is dropped below)
 }
 
 template <int FMT>
