@@ -138,7 +138,8 @@ sr_status sr_master_adamw_step(float* p, uint16_t* p_bf16, const void* g, sr_dty
  * sr_adamw_step_host_staging_bytes(g_dtype, chunk_elems) bytes, chunk_elems a non-zero multiple of
  * 8; larger chunks amortise copy latency (2^24 elements is a reasonable choice).
  * grad_scale_dev, if set, stays a device pointer.  The first call on a device creates the
- * library's second stream and two events (kept until the process ends). */
+ * library's second stream and two events (kept until the process ends); calls from several host
+ * threads are serialised while they enqueue. */
 size_t sr_adamw_step_host_staging_bytes(sr_dtype g_dtype, uint64_t chunk_elems);
 sr_status sr_adamw_step_host(uint16_t* p_host, const void* g_host, sr_dtype g_dtype, uint16_t* m_host,
                              uint16_t* v_host, uint64_t n, const sr_adamw_hparams* hp, uint64_t seed, uint32_t step,
@@ -151,7 +152,10 @@ sr_status sr_adamw_step_host(uint16_t* p_host, const void* g_host, sr_dtype g_dt
  * pointers and element counts; they may be freed after the call.  Tensor i uses
  * tensor_id = tensor_id_base + i and element indices starting at 0.  One hparams set serves the list.
  * The plan stays valid while the tensors it names stay allocated; destroy it with
- * sr_mt_plan_destroy (which synchronises nothing: do not destroy while a step using it is in flight). */
+ * sr_mt_plan_destroy (which synchronises nothing: do not destroy while a step using it is in flight).
+ * A plan belongs to the device that was current when it was created: sr_adamw_multi_tensor returns
+ * SR_ERR_INVALID_ARG under another current device.  Creation returns SR_ERR_WORKSPACE when host or
+ * device memory for the tables cannot be had. */
 typedef struct sr_mt_plan sr_mt_plan;
 sr_status sr_mt_plan_create(sr_mt_plan** out, uint32_t num_tensors, uint16_t* const* p, const void* const* g,
                             uint16_t* const* m, uint16_t* const* v, const uint64_t* numel, sr_dtype g_dtype,

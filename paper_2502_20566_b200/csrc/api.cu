@@ -1,8 +1,10 @@
 // C-ABI layer of libsradamw.so: argument checks, per-iteration scalars (Algorithm 1, the m-hat and
 // v-hat steps), Philox round keys, multi-tensor plans; all device work is in the kernel files.
 
+#include <atomic>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -22,19 +24,20 @@ sr_status cuda_fail(cudaError_t e) {
 
 constexpr int kMaxDevices = 64;
 struct DeviceSlot {
-    bool known = false;
+    std::atomic<bool> known{false};
     DeviceInfo info{};
 };
 DeviceSlot g_devices[kMaxDevices];
 
-// Properties of the current device, queried once per device.  Racing first calls write the same values.
+// Properties of the current device, queried once per device.  Racing first calls write the same
+// values; the flag is published after them.
 sr_status current_device(DeviceInfo* out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail(e);
     if (dev < 0 || dev >= kMaxDevices) return SR_ERR_UNSUPPORTED_DEVICE;
     DeviceSlot& slot = g_devices[dev];
-    if (!slot.known) {
+    if (!slot.known.load(std::memory_order_acquire)) {
         int sm = 0, major = 0;
         e = cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return cuda_fail(e);
@@ -42,7 +45,7 @@ sr_status current_device(DeviceInfo* out) {
         if (e != cudaSuccess) return cuda_fail(e);
         slot.info.sm_count = sm;
         slot.info.cc_major = major;
-        slot.known = true;
+        slot.known.store(true, std::memory_order_release);
     }
     if (slot.info.cc_major != 10) return SR_ERR_UNSUPPORTED_DEVICE;
     *out = slot.info;
@@ -99,6 +102,10 @@ sr_status make_scalars(const sr_adamw_hparams* hp, uint32_t step, StepScalars* S
 }
 
 }  // namespace
+
+namespace sradamw {
+int note_cuda_error(cudaError_t e) { return static_cast<int>(cuda_fail(e)); }
+}  // namespace sradamw
 
 struct sr_mt_plan {
     MtWork* d_work = nullptr;
@@ -206,6 +213,7 @@ struct HostPipe {
     cudaEvent_t fork = nullptr, join = nullptr;
 };
 HostPipe g_pipes[kMaxDevices];
+std::mutex g_pipe_mutex;   // the side stream and its two events are shared by all calls on a device
 
 size_t slot_bytes(bool g_f32, uint64_t chunk) {
     // p, m, v (2 bytes each) and g, each region rounded up to 256 bytes
@@ -238,6 +246,7 @@ sr_status sr_adamw_step_host(uint16_t* p_host, const void* g_host, sr_dtype g_dt
     if (st != SR_OK) return st;
     int dev_id = 0;
     cudaGetDevice(&dev_id);
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);   // enqueueing only; nothing below waits for the GPU
     HostPipe& pipe = g_pipes[dev_id];
     cudaError_t e;
     if (!pipe.ready) {
@@ -298,6 +307,7 @@ sr_status sr_mt_plan_create(sr_mt_plan** out, uint32_t num_tensors, uint16_t* co
     const size_t gsz = g_dtype == SR_DT_F32 ? 4 : 2;
     std::vector<MtWork> chunks;
     uint64_t total = 0;
+    try {
     for (uint32_t i = 0; i < num_tensors; ++i) {
         if (numel[i] != 0 && (p[i] == nullptr || g[i] == nullptr || m[i] == nullptr || v[i] == nullptr))
             return SR_ERR_INVALID_ARG;
@@ -314,9 +324,12 @@ sr_status sr_mt_plan_create(sr_mt_plan** out, uint32_t num_tensors, uint16_t* co
         }
         total += numel[i];
     }
+    } catch (const std::bad_alloc&) {   // no exception crosses the C ABI
+        return SR_ERR_WORKSPACE;
+    }
 
     sr_mt_plan* plan = new (std::nothrow) sr_mt_plan;
-    if (plan == nullptr) return SR_ERR_INVALID_ARG;
+    if (plan == nullptr) return SR_ERR_WORKSPACE;
     plan->num_tensors = num_tensors;
     plan->num_chunks = static_cast<uint32_t>(chunks.size());
     plan->total_elements = total;
@@ -350,6 +363,9 @@ sr_status sr_adamw_multi_tensor(const sr_mt_plan* plan, const sr_adamw_hparams* 
     DeviceInfo dev;
     st = current_device(&dev);
     if (st != SR_OK) return st;
+    int current = -1;
+    cudaGetDevice(&current);
+    if (current != plan->device) return SR_ERR_INVALID_ARG;   // the work table lives on the plan's device
     const cudaError_t e =
         launch_adamw_mt(plan->d_work, plan->num_chunks, plan->g_f32, tensor_id_base,
                         static_cast<uint32_t>(seed >> 32), hp->flags, make_keys(seed, step), S, dev,

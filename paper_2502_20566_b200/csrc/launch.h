@@ -78,6 +78,9 @@ cudaError_t launch_downcast_fp8(const float* src, uint8_t* dst, uint64_t n, bool
                                 uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev,
                                 cudaStream_t stream);
 
+// records e for sr_last_cuda_error() of the calling thread and returns the value of SR_ERR_CUDA
+int note_cuda_error(cudaError_t e);
+
 cudaError_t launch_downcast_fp4(const float* src, uint8_t* dst, uint64_t n, uint64_t elem_offset, uint32_t tensor_id,
                                 uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev, cudaStream_t stream);
 
