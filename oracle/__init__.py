@@ -18,6 +18,7 @@ _SRC = os.path.join(_HERE, "sradamw_oracle.cpp")
 _LIB = os.path.join(_HERE, "libsradamw_oracle.so")
 
 SR_P, SR_M, SR_V = 1, 2, 4
+EPS_INSIDE = 8
 SR_ALL = SR_P | SR_M | SR_V
 
 
@@ -42,6 +43,8 @@ class Scalars(ctypes.Structure):
         ("rsqrt_bc2", c_float),
         ("eps", c_float),
         ("lr_wd", c_float),
+        ("inv_bc2", c_float),
+        ("eps_inside", c_uint32),
     ]
 
 

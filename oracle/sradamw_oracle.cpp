@@ -40,8 +40,10 @@
 // the element function against correctly rounded exact rational arithmetic; the step-1 closed
 // form; a library AdamW as a loose bound; the summation tree against exact integer arithmetic.
 // Not pinned by the paper (its Algorithm 1 is ambiguous there; "parity unpinned" for that choice
-// alone): where epsilon sits relative to the square root.  This file uses the AdamW convention of
-// the optimizer the paper cites, sqrt(v/(1-beta2^t)) + epsilon.
+// alone): where epsilon sits relative to the square root.  The default is the AdamW convention of
+// the optimizer the paper cites, sqrt(v/(1-beta2^t)) + epsilon; flag bit 3 selects the other reading,
+// sqrt(v/(1-beta2^t) + epsilon), the form of the paper's analysis.  Both are pinned arithmetically
+// (exact rational intermediates, closed forms); which one the paper's experiments ran is not.
 
 #include <cmath>
 #include <cstdint>
@@ -173,7 +175,8 @@ struct oracle_hparams {
     float beta2;
     float eps;
     float weight_decay;  // lambda
-    uint32_t flags;      // bit0/1/2: stochastic rounding on x / m / v (else nearest-even)
+    uint32_t flags;      // bit0/1/2: stochastic rounding on x / m / v (else nearest-even);
+                         // bit3: epsilon under the square root (see oracle_adamw_element)
 };
 
 // Scalars that are the same for every element of one iteration.
@@ -186,6 +189,8 @@ struct oracle_scalars {
     float rsqrt_bc2;        // 1 / sqrt(1 - beta2^t)            (the v-hat step)
     float eps;
     float lr_wd;            // alpha_t * lambda
+    float inv_bc2;          // 1 / (1 - beta2^t)                (the v-hat step without its root)
+    uint32_t eps_inside;    // 1: the direction divides by sqrt(v-hat + eps) instead of sqrt(v-hat) + eps
 };
 
 // The FP32 intermediates of one element, in the order they are produced.
@@ -196,8 +201,8 @@ struct oracle_trace {
     float b1;     // (1-beta2) * g
     float b2;     // b1 * g
     float v_new;  // beta2*v + b2                    (moment update for v)
-    float s;      // sqrt(v_new)
-    float den;    // s * rsqrt_bc2 + eps
+    float s;      // sqrt(v_new)                     [epsilon inside: v_new * inv_bc2 + eps]
+    float den;    // s * rsqrt_bc2 + eps             [epsilon inside: sqrt(s)]
     float u;      // m_new / den
     float w;      // lr_wd * x
     float q;      // step_size*u + w
@@ -244,11 +249,18 @@ int oracle_adamw_scalars(const oracle_hparams* hp, uint32_t step, oracle_scalars
     out->rsqrt_bc2 = static_cast<float>(1.0 / std::sqrt(bc2));
     out->eps = hp->eps;
     out->lr_wd = static_cast<float>(lr * wd);
+    out->inv_bc2 = static_cast<float>(1.0 / bc2);
+    out->eps_inside = (hp->flags >> 3) & 1u;
     return 0;
 }
 
 // One element of Algorithm 1 in FP32.  Each line is one correctly rounded operation; fmaf is a
 // single rounding of a*b+c.
+// Where epsilon sits: Algorithm 1 as printed takes a square root in the v-hat step and again divides
+// by sqrt(v-hat + eps).  Two readings are implemented.  Default: the AdamW of the optimizer the paper
+// cites, sqrt(v/(1-beta2^t)) + eps.  With eps_inside: the form of the paper's analysis (appendix:
+// x - alpha_t m / sqrt(eps + v)) with the bias correction of the v-hat step kept,
+// sqrt(v/(1-beta2^t) + eps), i.e. the printed update step with the extra root of the v-hat step dropped.
 void oracle_adamw_element(float x, float g_in, float m, float v, float gscale,
                           const oracle_scalars* sc, oracle_trace* t) {
     t->g = gscale * g_in;
@@ -257,8 +269,13 @@ void oracle_adamw_element(float x, float g_in, float m, float v, float gscale,
     t->b1 = sc->one_minus_beta2 * t->g;
     t->b2 = t->b1 * t->g;
     t->v_new = fmaf(sc->beta2, v, t->b2);
-    t->s = sqrtf(t->v_new);
-    t->den = fmaf(t->s, sc->rsqrt_bc2, sc->eps);
+    if (sc->eps_inside) {
+        t->s = fmaf(t->v_new, sc->inv_bc2, sc->eps);
+        t->den = sqrtf(t->s);
+    } else {
+        t->s = sqrtf(t->v_new);
+        t->den = fmaf(t->s, sc->rsqrt_bc2, sc->eps);
+    }
     t->u = t->m_new / t->den;
     t->w = sc->lr_wd * x;
     t->q = fmaf(sc->step_size, t->u, t->w);

@@ -113,8 +113,12 @@ def _check_trace(x, g, m, v, gscale, sc, t):
     assert t.b1 == round_to_f32(F(sc.one_minus_beta2) * F(t.g))
     assert t.b2 == round_to_f32(F(t.b1) * F(t.g))
     assert t.v_new == round_to_f32(F(sc.beta2) * F(v) + F(t.b2))
-    assert _is_correct_sqrt(t.s, t.v_new)
-    assert t.den == round_to_f32(F(t.s) * F(sc.rsqrt_bc2) + F(sc.eps))
+    if sc.eps_inside:
+        assert t.s == round_to_f32(F(t.v_new) * F(sc.inv_bc2) + F(sc.eps))
+        assert _is_correct_sqrt(t.den, t.s)
+    else:
+        assert _is_correct_sqrt(t.s, t.v_new)
+        assert t.den == round_to_f32(F(t.s) * F(sc.rsqrt_bc2) + F(sc.eps))
     assert t.u == round_to_f32(F(t.m_new) / F(t.den))
     assert t.w == round_to_f32(F(sc.lr_wd) * F(x))
     assert t.q == round_to_f32(F(sc.step_size) * F(t.u) + F(t.w))
@@ -167,6 +171,83 @@ def test_first_step_from_zero_state_closed_form():
         assert t.x_new == pytest.approx(want, rel=2e-6, abs=1e-9)
         # the bias-corrected direction is g / (|g| + eps): magnitude just under 1, sign of g
         assert sc.step_size * t.u == pytest.approx(HP["lr"] * g / (abs(g) + HP["eps"]), rel=1e-6)
+
+
+# ---------------------------------------------------------------------------------------------
+# the other reading of the update step: epsilon under the square root
+# ---------------------------------------------------------------------------------------------
+
+def test_eps_inside_scalar_and_exact_intermediates():
+    rng = np.random.default_rng(31)
+    for eps in (1e-8, 1e-6, 1e-3):
+        hp = oracle.hparams(lr=6e-4, beta1=0.9, beta2=0.95, eps=eps, weight_decay=0.1, flags=oracle.SR_ALL | oracle.EPS_INSIDE)
+        for step in (1, 10, 1000):
+            sc = oracle.adamw_scalars(hp, step)
+            assert sc.eps_inside == 1
+            b2 = frac_of_float(f32(0.95))
+            exact = 1 / (1 - b2 ** step)
+            assert abs(frac_of_float(sc.inv_bc2) - exact) <= exact * Fraction(1, 1 << 23)      # one FP32 rounding of 1/(1-beta2^t)
+            for _ in range(100):
+                x = float(torch.tensor(rng.normal(0, 0.02)).to(torch.bfloat16))
+                g = f32(rng.normal(0, 1.0) * 10.0 ** rng.uniform(-8, 0))
+                m = float(torch.tensor(rng.normal(0, 1e-4)).to(torch.bfloat16))
+                v = float(torch.tensor(10.0 ** rng.uniform(-20, -2)).to(torch.bfloat16))
+                t = oracle.adamw_element(x, g, m, v, 1.0, sc)
+                _check_trace(x, g, m, v, 1.0, sc, t)
+    assert oracle.adamw_scalars(oracle.hparams(**HP), 5).eps_inside == 0
+
+
+def test_eps_inside_first_step_closed_form_and_difference_from_default():
+    """t = 1, m = v = 0: v-hat = g^2, so the direction is g / sqrt(g^2 + eps); for |g| << sqrt(eps) that is
+    g / sqrt(eps), whereas the default reading gives g / (|g| + eps): the two readings are told apart."""
+    eps = 1e-6
+    kw = dict(lr=6e-4, beta1=0.9, beta2=0.95, eps=eps, weight_decay=0.1)
+    inside = oracle.adamw_scalars(oracle.hparams(**kw, flags=oracle.SR_ALL | oracle.EPS_INSIDE), 1)
+    outside = oracle.adamw_scalars(oracle.hparams(**kw), 1)
+    rng = np.random.default_rng(32)
+    for _ in range(200):
+        x = float(torch.tensor(rng.normal(0, 0.02)).to(torch.bfloat16))
+        g = float(torch.tensor(rng.normal(0, 1e-3)).to(torch.bfloat16))
+        t = oracle.adamw_element(x, g, 0.0, 0.0, 1.0, inside)
+        want = x - kw["lr"] * (g / math.sqrt(g * g + eps) + kw["weight_decay"] * x)
+        assert t.x_new == pytest.approx(want, rel=2e-6, abs=1e-9)
+    g = f32(1e-5)                                                   # |g| = 0.01 sqrt(eps)
+    ti = oracle.adamw_element(0.0, g, 0.0, 0.0, 1.0, inside)
+    to = oracle.adamw_element(0.0, g, 0.0, 0.0, 1.0, outside)
+    assert inside.step_size * ti.u == pytest.approx(kw["lr"] * g / math.sqrt(eps), rel=1e-3)
+    assert outside.step_size * to.u == pytest.approx(kw["lr"] * g / (g + eps), rel=1e-5)
+    assert abs(to.u) > 50 * abs(ti.u)
+
+
+def test_eps_inside_with_zero_eps_agrees_with_the_default_to_rounding():
+    kw = dict(lr=6e-4, beta1=0.9, beta2=0.95, eps=0.0, weight_decay=0.0)
+    rng = np.random.default_rng(33)
+    for step in (1, 7, 300):
+        a = oracle.adamw_scalars(oracle.hparams(**kw, flags=oracle.SR_ALL | oracle.EPS_INSIDE), step)
+        b = oracle.adamw_scalars(oracle.hparams(**kw), step)
+        for _ in range(100):
+            g, m, v = f32(rng.normal(0, 1e-3)), f32(rng.normal(0, 1e-4)), f32(rng.normal(0, 1e-3) ** 2)
+            ta, tb = oracle.adamw_element(0.1, g, m, v, 1.0, a), oracle.adamw_element(0.1, g, m, v, 1.0, b)
+            assert ta.den == pytest.approx(tb.den, rel=4e-7) and ta.m_new == tb.m_new and ta.v_new == tb.v_new
+
+
+def test_eps_inside_array_step_uses_the_flag():
+    n = 4096
+    p, g, m, v = synth.adamw_state(n, 12, "cpu")
+    kw = dict(lr=6e-4, beta1=0.9, beta2=0.95, eps=1e-4, weight_decay=0.1)
+    outs = []
+    for flags in (oracle.SR_ALL, oracle.SR_ALL | oracle.EPS_INSIDE):
+        pb, gb, mb, vb = (synth.bits16(t).copy() for t in (p, g, m, v))
+        hp = oracle.hparams(**kw, flags=flags)
+        oracle.adamw_step(pb, gb, mb, vb, hp, seed=3, step=4)
+        sc = oracle.adamw_scalars(hp, 4)
+        for i in range(0, n, 97):
+            t = oracle.adamw_element(float(p[i]), float(g[i]), float(m[i]), float(v[i]), 1.0, sc)
+            r = oracle.noise(3, 4, 0, i)
+            assert pb[i] == oracle.sr_bf16_bits(f32_bits(t.x_new), r[0])
+        outs.append((pb, mb, vb))
+    assert not np.array_equal(outs[0][0], outs[1][0])               # x differs between the readings
+    assert np.array_equal(outs[0][1], outs[1][1]) and np.array_equal(outs[0][2], outs[1][2])   # m, v do not
 
 
 def test_zero_gradient_only_decays():
