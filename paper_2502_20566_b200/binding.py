@@ -21,6 +21,7 @@ SR_OK, SR_ERR_INVALID_ARG, SR_ERR_UNSUPPORTED_DEVICE, SR_ERR_WORKSPACE, SR_ERR_C
 SR_DT_BF16, SR_DT_F32 = 0, 1
 SR_FLAG_SR_P, SR_FLAG_SR_M, SR_FLAG_SR_V = 1, 2, 4
 SR_FLAGS_DEFAULT = 7
+SR_FLAG_EPS_INSIDE = 8
 
 EXPORTS = (
     "sr_downcast_f32_bf16", "sr_downcast_f32_fp8", "sr_downcast_f32_fp4", "sr_accumulate_bf16", "sr_adamw_step", "sr_master_adamw_step", "sr_adamw_step_host", "sr_adamw_step_host_staging_bytes",

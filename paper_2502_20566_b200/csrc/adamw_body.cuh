@@ -211,9 +211,9 @@ unsigned grid_for(Kernel kernel, uint64_t work_items, const DeviceInfo& dev, int
 }
 
 // The branch-free path needs den = sqrt(v1) * rsqrt_bc2 + eps to stay inside the range its
-// division was validated for.
+// division was validated for, and implements the default placement of epsilon only.
 inline bool fast_path_allowed(const StepScalars& S) {
-    return S.rsqrt_bc2 >= 1.0f && S.rsqrt_bc2 <= 1024.0f && S.eps >= 0.0f && S.eps <= 1.0f;
+    return !S.eps_inside && S.rsqrt_bc2 >= 1.0f && S.rsqrt_bc2 <= 1024.0f && S.eps >= 0.0f && S.eps <= 1.0f;
 }
 inline bool needs_scale(const StepScalars& S) { return S.gscale_dev != nullptr || S.gscale != 1.0f; }
 

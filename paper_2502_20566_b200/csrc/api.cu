@@ -84,7 +84,7 @@ sr_status make_scalars(const sr_adamw_hparams* hp, uint32_t step, StepScalars* S
     if (!(hp->beta1 >= 0.0f && hp->beta1 < 1.0f) || !(hp->beta2 >= 0.0f && hp->beta2 < 1.0f)) return SR_ERR_INVALID_ARG;
     if (!finite_f(hp->eps) || hp->eps < 0.0f || !finite_f(hp->weight_decay)) return SR_ERR_INVALID_ARG;
     if (hp->grad_scale_dev == nullptr && !finite_f(hp->grad_scale)) return SR_ERR_INVALID_ARG;
-    if (hp->flags & ~7u) return SR_ERR_INVALID_ARG;
+    if (hp->flags & ~(7u | SR_FLAG_EPS_INSIDE)) return SR_ERR_INVALID_ARG;
     const double b1 = hp->beta1, b2 = hp->beta2, lr = hp->lr, wd = hp->weight_decay;
     const double bc1 = 1.0 - power_u32(b1, step);
     const double bc2 = 1.0 - power_u32(b2, step);
@@ -98,6 +98,18 @@ sr_status make_scalars(const sr_adamw_hparams* hp, uint32_t step, StepScalars* S
     S->lr_wd = static_cast<float>(lr * wd);
     S->gscale = hp->grad_scale;
     S->gscale_dev = hp->grad_scale_dev;
+    S->eps_inside = (hp->flags & SR_FLAG_EPS_INSIDE) ? 1u : 0u;
+    if (S->eps_inside) {
+        S->pre_mul = static_cast<float>(1.0 / bc2);
+        S->pre_add = hp->eps;
+        S->post_mul = 1.0f;
+        S->post_add = 0.0f;
+    } else {
+        S->pre_mul = 1.0f;
+        S->pre_add = 0.0f;
+        S->post_mul = S->rsqrt_bc2;
+        S->post_add = hp->eps;
+    }
     return SR_OK;
 }
 

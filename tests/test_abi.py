@@ -65,7 +65,7 @@ def test_argument_errors_come_before_device_work(lib):
     assert call(bad, 1) == b.SR_ERR_INVALID_ARG
     bad = b.hparams(float("nan"), 0.9, 0.95, 1e-8, 0.1)
     assert call(bad, 1) == b.SR_ERR_INVALID_ARG
-    bad = b.hparams(6e-4, 0.9, 0.95, 1e-8, 0.1, flags=8)
+    bad = b.hparams(6e-4, 0.9, 0.95, 1e-8, 0.1, flags=16)
     assert call(bad, 1) == b.SR_ERR_INVALID_ARG
     bad = b.hparams(6e-4, 0.9, 0.95, 1e-8, 0.1)
     bad.struct_size = 44

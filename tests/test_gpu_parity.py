@@ -106,6 +106,54 @@ def test_flat_step_rounding_modes(env, flags, g_dtype):
     assert run_both(env, p, g, m, v, HP, seed=3, step=10, gscale=0.125, flags=flags) == (0, 0, 0)
 
 
+@pytest.mark.parametrize("eps", [1e-8, 1e-4])
+@pytest.mark.parametrize("flags", [15, 9, 8])
+@pytest.mark.parametrize("g_dtype,n,offset", [(torch.bfloat16, (1 << 20) + 5, 0), (torch.float32, 50001, 24), (torch.bfloat16, 4099, 3)])
+def test_flat_step_eps_inside(env, eps, flags, g_dtype, n, offset):
+    """The other reading of the update step (epsilon under the square root, flag bit 3), with every rounding
+    choice it is combined with here: bit-exact, and different from the default reading."""
+    oracle, binding, synth, dev = env
+    kw = dict(HP, eps=eps)
+    p, g, m, v = synth.adamw_state(n, 14, dev, g_dtype=g_dtype)
+    if n > 10000:                                   # special values take the same route as everything else
+        mix = synth.downcast_mix(64, 5, dev)
+        p[:64], m[64:128], v[128:192] = mix.bfloat16(), mix.bfloat16(), mix.abs().bfloat16()
+    q = p.clone()
+    assert run_both(env, p, g, m, v, kw, seed=21, step=10, elem_offset=offset, gscale=0.5, flags=flags) == (0, 0, 0)
+    if eps > 1e-6 and n > 10000:
+        p2, g2, m2, v2 = synth.adamw_state(n, 14, dev, g_dtype=g_dtype)
+        binding.sr_adamw_step(p2, g2, m2, v2, binding.hparams(**kw, grad_scale=0.5, flags=flags & 7), 21, 10, 0, offset)
+        torch.cuda.synchronize()
+        assert mismatches(bits(p2)[192:], bits(p)[192:]) > n // 4
+
+
+def test_eps_inside_list_and_master_recipe(env):
+    oracle, binding, synth, dev = env
+    kw = dict(HP, eps=1e-5)
+    sizes = [5, 8192, 8193, 30000, 77, 2 * 8192 + 7]
+    T = [synth.adamw_state(n, 700 + i, dev) for i, n in enumerate(sizes)]
+    P, G, M, V = ([t[k] for t in T] for k in range(4))
+    plan = binding.sr_mt_plan_create(P, G, M, V)
+    host = [[bits(t) for t in P], [host_g(t) for t in G], [bits(t) for t in M], [bits(t) for t in V]]
+    binding.sr_adamw_multi_tensor(plan, binding.hparams(**kw, flags=15), 4, 2, tensor_id_base=50)
+    torch.cuda.synchronize()
+    for i in range(len(sizes)):
+        oracle.adamw_step(host[0][i], host[1][i], host[2][i], host[3][i], oracle.hparams(**kw, flags=15), 4, 2, 50 + i)
+        assert mismatches(bits(P[i]), host[0][i]) + mismatches(bits(M[i]), host[2][i]) + mismatches(bits(V[i]), host[3][i]) == 0
+    plan.destroy()
+    n = 40003
+    p0, g, m0, v0 = synth.adamw_state(n, 41, dev, g_dtype=torch.float32)
+    p, m, v = p0.float(), m0.float(), v0.float()
+    p16 = torch.zeros(n, dtype=torch.bfloat16, device=dev)
+    ph, mh, vh = (t.cpu().numpy().copy() for t in (p, m, v))
+    want16 = oracle.master_adamw_step(ph, host_g(g), mh, vh, oracle.hparams(**kw, flags=15), 3)
+    binding.sr_master_adamw_step(p, p16, g, m, v, binding.hparams(**kw, flags=15), 3)
+    torch.cuda.synchronize()
+    for dev_t, host_t in ((p, ph), (m, mh), (v, vh)):
+        assert np.array_equal(dev_t.cpu().numpy().view(np.uint32), host_t.view(np.uint32))
+    assert mismatches(bits(p16), want16) == 0
+
+
 def test_flat_step_special_values(env):
     """NaN, infinities, zeros, subnormals and huge values in every input."""
     _, _, synth, dev = env
