@@ -7,6 +7,8 @@ namespace sradamw {
 
 // MODE 0: element-wise (any alignment, any offset)
 //      1: 16-byte vectors, reference arithmetic, per-element noise (elem_offset not a multiple of 8)
+//      4: 16-byte vectors, reference arithmetic, one Philox call per (vector, slot): elem_offset a
+//         multiple of 8 but scalars outside what the branch-free arithmetic covers
 // Persistent grid: thread t takes vectors t, t + T, t + 2T, ... (T = threads in the grid).
 template <bool G32, uint32_t FLAGS, int MODE>
 __global__ void __launch_bounds__(kBlockThreads, kMinBlocksPerSM)
@@ -23,7 +25,7 @@ k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n
     }
     const uint64_t nvec = n >> 3;
     for (uint64_t vec = tid; vec < nvec; vec += stride)
-        step_vec8_reference<G32, FLAGS, false>(p, g, m, v, vec, elem_offset + (vec << 3), tensor_id, seed_hi, gscale, K, S);
+        step_vec8_reference<G32, FLAGS, MODE == 4>(p, g, m, v, vec, elem_offset + (vec << 3), tensor_id, seed_hi, gscale, K, S);
     const uint64_t done = nvec << 3;
     if (tid < n - done)
         step_scalar<G32, FLAGS>(p, g, m, v, done + tid, elem_offset + done + tid, tensor_id, seed_hi, gscale, K, S);
@@ -107,7 +109,7 @@ cudaError_t launch_flat_mode(uint16_t* p, const void* g, uint16_t* m, uint16_t* 
                              uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K, const StepScalars& S,
                              const DeviceInfo& dev, cudaStream_t stream) {
     const uint64_t items = MODE == 0 ? n : (n >> 3) + 8;   // + 8: enough threads for the ragged tail
-    if (MODE >= 2) {
+    if (MODE == 2 || MODE == 3) {
         constexpr bool kStaged = G32 ? (SR_STAGE_F32 != 0) : (SR_STAGE_BF16 != 0);
         const uint32_t c1 = static_cast<uint32_t>(elem_offset >> 33);
         if (kStaged && n >= kLongLaunchElems) {
@@ -119,7 +121,7 @@ cudaError_t launch_flat_mode(uint16_t* p, const void* g, uint16_t* m, uint16_t* 
             k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
         }
     } else {
-        auto k = k_sr_adamw_flat<G32, FLAGS, (MODE < 2 ? MODE : 0)>;
+        auto k = k_sr_adamw_flat<G32, FLAGS, (MODE < 2 || MODE == 4 ? MODE : 0)>;
         k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset, tensor_id, seed_hi, K, S);
     }
     return cudaGetLastError();
@@ -145,8 +147,10 @@ cudaError_t launch_flat_flags(uint16_t* p, const void* g, uint16_t* m, uint16_t*
         cudaError_t e;
         if (!vec)
             e = launch_flat_mode<G32, FLAGS, 0>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream);
-        else if ((idx & 7u) != 0 || !fast_path_allowed(S))
+        else if ((idx & 7u) != 0)
             e = launch_flat_mode<G32, FLAGS, 1>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream);
+        else if (!fast_path_allowed(S))
+            e = launch_flat_mode<G32, FLAGS, 4>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream);
         else if (needs_scale(S))
             e = launch_flat_mode<G32, FLAGS, 3>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream);
         else
