@@ -1,0 +1,120 @@
+"""``torch.optim`` front end of the fused step: Algorithm 1 (AdamW on BF16 parameters with stochastically
+rounded updates and a random state shared by all replicas) for a model whose parameters are BF16 CUDA tensors.
+
+The class only marshals arguments: every parameter group becomes one tensor-list plan and one
+``sr_adamw_multi_tensor`` launch per step.  Moments are BF16 (6 bytes of optimizer-side state per parameter
+instead of the 14 of an FP32-master recipe).  The noise is a pure function of (seed, step, tensor id, element
+index), so there is no generator state to fork, restore or checkpoint: replicas that hold the same seed stay
+bit-identical, and ``state_dict`` / ``load_state_dict`` resume a run bit-exactly.
+"""
+
+from __future__ import annotations
+
+from typing import Iterable, Optional
+
+import torch
+
+from . import binding
+
+
+class SRAdamW(torch.optim.Optimizer):
+    """AdamW with BF16 parameters, gradients and moments and stochastic rounding (Algorithm 1).
+
+    params: BF16 CUDA parameters (or parameter groups); gradients may be BF16 or FP32, one type per group.
+    sr_flags: which of x, m, v are rounded stochastically (``binding.SR_FLAG_SR_P | _M | _V``); 1 is the
+        paper's update-only SR, 0 plain nearest rounding.
+    eps_inside: the other reading of the update step, epsilon under the square root.
+    seed: the shared random state; give every data-parallel replica the same value.
+    ``step(grad_scale=...)`` multiplies the gradients by a host scalar, ``step(grad_scale_dev=t)`` by a device
+    scalar (e.g. the output of ``sr_clip_scale``), without an extra pass over them.
+    """
+
+    def __init__(self, params: Iterable, lr: float = 1e-3, betas=(0.9, 0.999), eps: float = 1e-8,
+                 weight_decay: float = 1e-2, seed: int = 0, sr_flags: int = binding.SR_FLAGS_DEFAULT,
+                 eps_inside: bool = False):
+        if lr < 0 or not 0 <= betas[0] < 1 or not 0 <= betas[1] < 1 or eps < 0:
+            raise ValueError("invalid hyper-parameter")
+        if sr_flags & ~7:
+            raise ValueError("sr_flags: bits 0..2 only")
+        defaults = dict(lr=lr, betas=tuple(betas), eps=eps, weight_decay=weight_decay)
+        super().__init__(params, defaults)
+        self.seed = int(seed)
+        self.flags = int(sr_flags) | (binding.SR_FLAG_EPS_INSIDE if eps_inside else 0)
+        self._steps = 0
+        self._plans = {}          # group index -> (key of data pointers, plan)
+        binding.lib()             # fail here, not in the first step, when the CUDA library is missing
+        for group in self.param_groups:
+            for p in group["params"]:
+                if not p.is_cuda or p.dtype != torch.bfloat16 or not p.is_contiguous():
+                    raise TypeError("SRAdamW needs contiguous BF16 CUDA parameters")
+
+    # the moments are created on first use so that load_state_dict can supply them instead
+    def _moments(self, p: torch.Tensor):
+        st = self.state[p]
+        if "exp_avg" not in st:
+            st["exp_avg"] = torch.zeros_like(p, memory_format=torch.contiguous_format)
+            st["exp_avg_sq"] = torch.zeros_like(p, memory_format=torch.contiguous_format)
+        return st["exp_avg"], st["exp_avg_sq"]
+
+    def _plan(self, gi: int, group) -> Optional[binding.MtPlan]:
+        P, G, M, V = [], [], [], []
+        g_dtype = None
+        for p in group["params"]:
+            if p.grad is not None:
+                if p.grad.is_sparse:
+                    raise RuntimeError("SRAdamW does not support sparse gradients")
+                g_dtype = g_dtype or p.grad.dtype
+        if g_dtype is None:
+            return None
+        empty = None
+        for p in group["params"]:
+            g = p.grad
+            if g is None:
+                # keeps the tensor ids of the others unchanged: an entry of zero elements
+                if empty is None:
+                    empty = (torch.empty(0, dtype=torch.bfloat16, device=p.device), torch.empty(0, dtype=g_dtype, device=p.device))
+                P.append(empty[0]); G.append(empty[1]); M.append(empty[0]); V.append(empty[0])
+                continue
+            m, v = self._moments(p)
+            P.append(p.data); G.append(g if g.is_contiguous() else g.contiguous()); M.append(m); V.append(v)
+        key = tuple(t.data_ptr() for ts in (P, G, M, V) for t in ts) + tuple(t.numel() for t in P)
+        cached = self._plans.get(gi)
+        if cached is None or cached[0] != key:
+            if cached is not None:
+                cached[1].destroy()
+            cached = (key, binding.sr_mt_plan_create(P, G, M, V))
+            self._plans[gi] = cached
+        return cached[1]
+
+    @torch.no_grad()
+    def step(self, closure=None, grad_scale: float = 1.0, grad_scale_dev: Optional[torch.Tensor] = None):
+        loss = None
+        if closure is not None:
+            with torch.enable_grad():
+                loss = closure()
+        self._steps += 1
+        base = 0
+        for gi, group in enumerate(self.param_groups):
+            plan = self._plan(gi, group)
+            if plan is not None:
+                hp = binding.hparams(lr=group["lr"], beta1=group["betas"][0], beta2=group["betas"][1], eps=group["eps"],
+                                     weight_decay=group["weight_decay"], grad_scale=grad_scale,
+                                     grad_scale_dev=grad_scale_dev, flags=self.flags)
+                binding.sr_adamw_multi_tensor(plan, hp, self.seed, self._steps, tensor_id_base=base)
+            base += len(group["params"])
+        return loss
+
+    # ---- checkpointing: seed and step count are the whole random state -------------------------
+    def state_dict(self):
+        d = super().state_dict()
+        d["sr"] = {"seed": self.seed, "steps": self._steps, "flags": self.flags}
+        return d
+
+    def load_state_dict(self, state_dict):
+        sr = state_dict.get("sr")
+        super().load_state_dict({k: v for k, v in state_dict.items() if k != "sr"})
+        if sr is not None:
+            self.seed, self._steps, self.flags = int(sr["seed"]), int(sr["steps"]), int(sr["flags"])
+        for cached in self._plans.values():
+            cached[1].destroy()
+        self._plans = {}

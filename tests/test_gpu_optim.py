@@ -1,0 +1,118 @@
+"""The torch.optim front end on a GPU: bit-exact against the oracle, the paper's qualitative claim on a
+synthetic regression (BF16 + stochastic rounding follows FP32 AdamW where BF16 + nearest rounding stagnates,
+Section 2.1), and bit-exact resume from a checkpoint."""
+
+import copy
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    import oracle
+    from paper_2502_20566_b200 import binding, optim, synth
+    binding.lib()
+    return oracle, binding, optim, synth, torch.device("cuda", 0)
+
+
+def bits(t):
+    return t.detach().view(torch.int16).cpu().numpy().view(np.uint16).copy()
+
+
+def test_optimizer_step_is_the_oracle_step(env):
+    oracle, binding, optim, synth, dev = env
+    sizes = [(300, 70), (70,), (8192,), (1,), (129, 64)]
+    gen = torch.Generator(device=dev).manual_seed(1)
+    params = [torch.nn.Parameter((torch.randn(s, device=dev, generator=gen) * 0.05).bfloat16()) for s in sizes]
+    groups = [dict(params=params[:3], weight_decay=0.1), dict(params=params[3:], weight_decay=0.0, lr=3e-4)]
+    opt = optim.SRAdamW(groups, lr=6e-4, betas=(0.9, 0.95), eps=1e-8, seed=(5 << 32) | 9)
+    host = [dict(p=bits(p).reshape(-1), m=np.zeros(p.numel(), np.uint16), v=np.zeros(p.numel(), np.uint16)) for p in params]
+    for step in (1, 2, 3):
+        for i, p in enumerate(params):
+            p.grad = None if (step == 2 and i == 1) else (torch.randn(p.shape, device=dev, generator=gen) * 1e-3).bfloat16()
+        opt.step(grad_scale=0.5)
+        torch.cuda.synchronize()
+        for i, p in enumerate(params):
+            if p.grad is None:
+                continue
+            kw = dict(lr=6e-4 if i < 3 else 3e-4, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1 if i < 3 else 0.0)
+            h = host[i]
+            oracle.adamw_step(h["p"], bits(p.grad).reshape(-1), h["m"], h["v"], oracle.hparams(**kw), (5 << 32) | 9, step, i, 0, 0.5)
+            assert np.array_equal(bits(p).reshape(-1), h["p"])
+            assert np.array_equal(bits(opt.state[p]["exp_avg"]).reshape(-1), h["m"])
+            assert np.array_equal(bits(opt.state[p]["exp_avg_sq"]).reshape(-1), h["v"])
+
+
+def _regression(dev):
+    gen = torch.Generator(device=dev).manual_seed(7)
+    d, n = 256, 2048
+    X = torch.randn(n, d, device=dev, generator=gen)
+    w_star = torch.randn(d, device=dev, generator=gen)
+    w_star = torch.where(w_star.abs() < 0.5, w_star.sign() * 0.5 - w_star, w_star)      # |w*| >= 0.5: coarse BF16 spacing
+    y = X @ w_star
+    w0 = (w_star + 0.05 * torch.randn(d, device=dev, generator=gen)).bfloat16().float()
+    return X, y, w_star, w0
+
+
+def _train(make_opt, w0, X, y, dtype, steps=400):
+    w = torch.nn.Parameter(w0.to(dtype).clone())
+    opt = make_opt([w])
+    for _ in range(steps):
+        r = X @ w.detach().float() - y
+        w.grad = (X.t() @ r / X.shape[0]).to(dtype)
+        opt.step()
+    return w.detach().float()
+
+
+def test_sr_follows_fp32_where_nearest_rounding_stagnates(env):
+    """Updates of about lr = 5e-4 per step are far below half a BF16 spacing (2^-9 .. 2^-8 for these weights):
+    nearest rounding discards them, stochastic rounding applies them in expectation."""
+    _, binding, optim, _, dev = env
+    X, y, w_star, w0 = _regression(dev)
+    kw = dict(lr=5e-4, betas=(0.9, 0.95), eps=1e-8, weight_decay=0.0)
+    err = lambda w: float((w - w_star).norm())
+    e0 = err(w0)
+    e_fp32 = err(_train(lambda ps: torch.optim.AdamW(ps, **kw), w0, X, y, torch.float32))
+    e_sr = err(_train(lambda ps: optim.SRAdamW(ps, seed=3, **kw), w0, X, y, torch.bfloat16))
+    e_near = err(_train(lambda ps: optim.SRAdamW(ps, seed=3, sr_flags=0, **kw), w0, X, y, torch.bfloat16))
+    assert e_fp32 < 0.2 * e0
+    assert e_sr < 0.35 * e0                      # SR gets most of the way (its floor is the BF16 spacing)
+    assert e_near > 0.8 * e0                     # nearest rounding hardly moves
+    assert e_sr < 0.4 * e_near
+
+
+def test_resume_from_checkpoint_is_bit_exact(env):
+    _, binding, optim, _, dev = env
+    gen = torch.Generator(device=dev).manual_seed(11)
+    shapes = [(64, 33), (33,), (4097,)]
+    init = [(torch.randn(s, device=dev, generator=gen) * 0.05).bfloat16() for s in shapes]
+    grads = [[(torch.randn(s, device=dev, generator=gen) * 1e-3).bfloat16() for s in shapes] for _ in range(6)]
+
+    def run(params, opt, steps):
+        for t in steps:
+            for p, g in zip(params, grads[t]):
+                p.grad = g.clone()
+            opt.step()
+
+    a = [torch.nn.Parameter(t.clone()) for t in init]
+    opt_a = optim.SRAdamW(a, lr=1e-3, betas=(0.9, 0.95), seed=42)
+    run(a, opt_a, range(6))
+    b = [torch.nn.Parameter(t.clone()) for t in init]
+    opt_b = optim.SRAdamW(b, lr=1e-3, betas=(0.9, 0.95), seed=42)
+    run(b, opt_b, range(3))
+    saved = copy.deepcopy(opt_b.state_dict())
+    weights = [p.detach().clone() for p in b]
+    c = [torch.nn.Parameter(t.clone()) for t in weights]
+    opt_c = optim.SRAdamW(c, lr=1e-3, betas=(0.9, 0.95), seed=0)          # the seed comes from the checkpoint
+    opt_c.load_state_dict(saved)
+    run(c, opt_c, range(3, 6))
+    torch.cuda.synchronize()
+    for pa, pc in zip(a, c):
+        assert np.array_equal(bits(pa), bits(pc))
+        assert np.array_equal(bits(opt_a.state[pa]["exp_avg_sq"]), bits(opt_c.state[pc]["exp_avg_sq"]))
