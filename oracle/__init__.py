@@ -266,6 +266,22 @@ def sqnorm(g) -> float:
     return float(lib().oracle_sqnorm(_ptr(_check(g, np.uint16)), 0, g.size))
 
 
+def sqnorm_list(grads) -> float:
+    """Sum of squares over a list of gradient arrays: one block sum per chunk of 8192 consecutive entries of
+    each array (arrays in list order, the block rule applied inside the chunk), then the array of block sums
+    reduced by the tree.  Composed from the two routines above."""
+    partials = []
+    for g in grads:
+        flat = np.ascontiguousarray(g).reshape(-1)
+        for start in range(0, flat.size, 8192):
+            partials.append(sqnorm(np.ascontiguousarray(flat[start:start + 8192])))
+    if not partials:
+        return 0.0
+    if len(partials) == 1:
+        return partials[0]
+    return tree_sum(np.array(partials, dtype=np.float64))
+
+
 def tree_sum(terms) -> float:
     _check(terms, np.float64)
     return float(lib().oracle_tree_sum(_ptr(terms), terms.size))

@@ -471,3 +471,20 @@ def test_clip_scale_closed_forms():
     S = 7.3e4
     gs = oracle.clip_scale(S, 0.25, 2.0)
     assert gs * math.sqrt(S) == pytest.approx(2.0, rel=1e-6)
+
+
+def test_list_norm_reduces_to_the_flat_norm_and_is_exact_on_integers():
+    """Pins for the list form of the squared norm: one tensor gives the flat routine's bits; tensors whose
+    lengths are multiples of 8192 give the bits of their concatenation; integer data give the exact sum."""
+    rng = np.random.default_rng(40)
+    a = rng.normal(0, 1e-3, 3 * 8192).astype(np.float32)
+    b = rng.normal(0, 1.0, 8192).astype(np.float32)
+    c = rng.normal(0, 1e-2, 20000).astype(np.float32)
+    assert oracle.sqnorm_list([c]).hex() == oracle.sqnorm(c).hex()
+    assert oracle.sqnorm_list([a, b, c]).hex() == oracle.sqnorm(np.concatenate([a, b, c])).hex()
+    ints = [rng.integers(-50, 50, n).astype(np.float32) for n in (5, 8192, 8193, 1, 0, 30000)]
+    assert oracle.sqnorm_list(ints) == float(sum(int((x.astype(np.int64) ** 2).sum()) for x in ints))
+    assert oracle.sqnorm_list([]) == 0.0 and oracle.sqnorm_list([np.zeros(0, np.float32)]) == 0.0
+    bf = [(x.view(np.uint32) >> 16).astype(np.uint16) for x in (a, c)]
+    want = sum(float(v) ** 2 for x in bf for v in (x.astype(np.uint32) << 16).view(np.float32).astype(np.float64))
+    assert oracle.sqnorm_list(bf) == pytest.approx(want, rel=1e-12)
