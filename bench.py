@@ -292,6 +292,23 @@ def _extras_list(torch, binding, synth, dev, peak, timed, out, compare_flat):
     ne = plan.total_elements
     out["tensor_list_gpt2_350m"] = {"tensors": len(specs), "elements": ne, "ms": t_mt, "params_per_s": ne / t_mt * 1e3,
                                     "gbs": 14 * ne / t_mt / 1e6, "frac": 14 * ne / t_mt / 1e6 / peak}
+    # global-norm clipping of the whole list on the device: list norm -> clip factor -> step (16 B per element)
+    ws = torch.empty(max(1, binding.grad_sqnorm_multi_tensor_workspace_bytes(plan) // 8), dtype=torch.float64, device=dev)
+    S = torch.zeros(1, dtype=torch.float64, device=dev)
+    gs = torch.zeros(1, dtype=torch.float32, device=dev)
+    hp_clip = binding.hparams(**HP, grad_scale_dev=gs)
+    t_norm = timed(lambda: binding.grad_sqnorm_multi_tensor(plan, S, ws))
+
+    def clipped():
+        step[0] += 1
+        binding.grad_sqnorm_multi_tensor(plan, S, ws)
+        binding.sr_clip_scale(S, 1.0, 1.0, gs)
+        binding.sr_adamw_multi_tensor(plan, hp_clip, SEED, step[0])
+    t_clip = timed(clipped)
+    out["tensor_list_gpt2_350m"]["grad_sqnorm_multi_tensor"] = {"ms": t_norm, "gbs": 2 * ne / t_norm / 1e6,
+                                                                "frac": 2 * ne / t_norm / 1e6 / peak}
+    out["tensor_list_gpt2_350m"]["norm_clip_step"] = {"ms": t_clip, "params_per_s": ne / t_clip * 1e3,
+                                                      "gbs": 16 * ne / t_clip / 1e6, "frac": 16 * ne / t_clip / 1e6 / peak}
     plan.destroy()
     del P, G, M, V
     if not compare_flat:

@@ -184,6 +184,20 @@ size_t grad_sqnorm_workspace_bytes(uint64_t n);
 sr_status grad_sqnorm(const void* g, sr_dtype g_dtype, uint64_t n, double* out_dev, void* workspace,
                       size_t workspace_bytes, void* stream);
 
+/* The same sum over the gradients of a tensor list (global-norm clipping of a whole model; not part
+ * of the paper either).  The first pass takes one block sum per chunk of the plan: tensor by tensor
+ * in list order, every tensor cut into chunks of 8192 consecutive entries (the last one ragged), the
+ * block rule above applied inside each chunk with positions counted from the chunk's start.  The
+ * array of block sums, in that order, is then reduced by the later passes of grad_sqnorm.  For a
+ * list of one tensor the result equals grad_sqnorm's, bit for bit; so it does for a list whose
+ * tensors all have lengths that are multiples of 8192, against grad_sqnorm of their concatenation.
+ * out_dev: one double on the device.  workspace: device memory of at least
+ * grad_sqnorm_multi_tensor_workspace_bytes(plan) bytes, 8-byte aligned (may be NULL when that is 0).
+ * Reads the gradient pointers the plan was created with; call under the plan's device. */
+size_t grad_sqnorm_multi_tensor_workspace_bytes(const sr_mt_plan* plan);
+sr_status grad_sqnorm_multi_tensor(const sr_mt_plan* plan, double* out_dev, void* workspace, size_t workspace_bytes,
+                                   void* stream);
+
 /* grad_sqnorm for callers that cannot allocate.  (The paper has no counterpart; neither has the
  * rest of the norm/clipping code.)  Some users of this library run where cudaMalloc is not an
  * option: inside a process whose device memory is owned and fully handed out by someone else's

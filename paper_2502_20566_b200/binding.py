@@ -27,7 +27,7 @@ EXPORTS = (
     "sr_downcast_f32_bf16", "sr_downcast_f32_fp8", "sr_downcast_f32_fp4", "sr_accumulate_bf16", "sr_adamw_step", "sr_master_adamw_step", "sr_adamw_step_host", "sr_adamw_step_host_staging_bytes",
     "sr_mt_plan_create", "sr_adamw_multi_tensor",
     "sr_mt_plan_destroy", "sr_mt_plan_total_elements", "grad_sqnorm_workspace_bytes", "grad_sqnorm",
-    "grad_sqnorm_static", "grad_sqnorm_static_max_elements",
+    "grad_sqnorm_static", "grad_sqnorm_static_max_elements", "grad_sqnorm_multi_tensor", "grad_sqnorm_multi_tensor_workspace_bytes",
     "sr_clip_scale", "sr_status_string", "sr_last_cuda_error", "sr_abi_version",
 )
 
@@ -104,6 +104,10 @@ def lib() -> ctypes.CDLL:
         L.sr_mt_plan_destroy.restype = c_int
         L.sr_mt_plan_total_elements.argtypes = [c_void_p]
         L.sr_mt_plan_total_elements.restype = c_uint64
+        L.grad_sqnorm_multi_tensor_workspace_bytes.argtypes = [c_void_p]
+        L.grad_sqnorm_multi_tensor_workspace_bytes.restype = c_size_t
+        L.grad_sqnorm_multi_tensor.argtypes = [c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.grad_sqnorm_multi_tensor.restype = c_int
         L.grad_sqnorm_workspace_bytes.argtypes = [c_uint64]
         L.grad_sqnorm_workspace_bytes.restype = c_size_t
         L.grad_sqnorm.argtypes = [c_void_p, c_int, c_uint64, c_void_p, c_void_p, c_size_t, c_void_p]
@@ -315,6 +319,19 @@ def grad_sqnorm(g: torch.Tensor, out: torch.Tensor, workspace: Optional[torch.Te
     with torch.cuda.device(g.device):
         _check(lib().grad_sqnorm(g.data_ptr(), _g_dtype(g), g.numel(), out.data_ptr(), ws_ptr, ws_bytes,
                                  _stream(stream)), "grad_sqnorm")
+
+
+def grad_sqnorm_multi_tensor_workspace_bytes(plan: MtPlan) -> int:
+    return int(lib().grad_sqnorm_multi_tensor_workspace_bytes(plan._handle))
+
+
+def grad_sqnorm_multi_tensor(plan: MtPlan, out: torch.Tensor, workspace: Optional[torch.Tensor], stream=None) -> None:
+    """Sum of squares over all gradients of the plan's list; out: one float64 on the device."""
+    _want(out, torch.float64, "out")
+    ws_ptr, ws_bytes = (workspace.data_ptr(), workspace.numel() * workspace.element_size()) if workspace is not None else (None, 0)
+    with torch.cuda.device(plan.device):
+        _check(lib().grad_sqnorm_multi_tensor(plan._handle, out.data_ptr(), ws_ptr, ws_bytes, _stream(stream)),
+               "grad_sqnorm_multi_tensor")
 
 
 def grad_sqnorm_static_max_elements() -> int:

@@ -413,6 +413,27 @@ sr_status grad_sqnorm(const void* g, sr_dtype g_dtype, uint64_t n, double* out_d
     return e == cudaSuccess ? SR_OK : cuda_fail(e);
 }
 
+size_t grad_sqnorm_multi_tensor_workspace_bytes(const sr_mt_plan* plan) {
+    return plan ? static_cast<size_t>(sqnorm_mt_scratch_doubles(plan->num_chunks) * sizeof(double)) : 0;
+}
+
+sr_status grad_sqnorm_multi_tensor(const sr_mt_plan* plan, double* out_dev, void* workspace, size_t workspace_bytes,
+                                   void* stream) {
+    if (plan == nullptr || out_dev == nullptr) return SR_ERR_INVALID_ARG;
+    const size_t need = grad_sqnorm_multi_tensor_workspace_bytes(plan);
+    if (need != 0 && (workspace == nullptr || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 7u)))
+        return SR_ERR_WORKSPACE;
+    DeviceInfo dev;
+    sr_status st = current_device(&dev);
+    if (st != SR_OK) return st;
+    int current = -1;
+    cudaGetDevice(&current);
+    if (current != plan->device) return SR_ERR_INVALID_ARG;
+    const cudaError_t e = launch_sqnorm_mt(plan->d_work, plan->num_chunks, plan->g_f32, out_dev,
+                                           static_cast<double*>(workspace), dev, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SR_OK : cuda_fail(e);
+}
+
 sr_status sr_clip_scale(const double* sqnorm_dev, float accum_scale, float max_norm, float* gscale_out_dev,
                         void* stream) {
     if (sqnorm_dev == nullptr || gscale_out_dev == nullptr) return SR_ERR_INVALID_ARG;

@@ -93,6 +93,9 @@ cudaError_t launch_master_adamw(float* p, uint16_t* p16, const void* g, bool g_f
 
 // Squared norm: number of doubles of scratch needed, and the launcher.
 uint64_t sqnorm_scratch_doubles(uint64_t n);
+uint64_t sqnorm_mt_scratch_doubles(uint64_t num_chunks);
+cudaError_t launch_sqnorm_mt(const MtWork* work, uint32_t num_chunks, bool g_f32, double* out, double* scratch,
+                             const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_sqnorm(const void* g, bool g_f32, uint64_t n, double* out, double* scratch,
                           const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_clip_scale(const double* sqnorm, float accum_scale, float max_norm, float* out,

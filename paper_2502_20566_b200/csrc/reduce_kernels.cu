@@ -93,6 +93,59 @@ k_sqnorm_pass1(const void* __restrict__ g, uint64_t n, uint64_t num_blocks, bool
     }
 }
 
+// First pass over a tensor list: out[c] = tree-block sum of squares of work-table entry c (a chunk of
+// at most 8192 consecutive gradient entries of one tensor, positions counted from the chunk's start).
+template <bool G32>
+__global__ void __launch_bounds__(kTreeThreads)
+k_sqnorm_mt_pass1(const MtWork* __restrict__ work, uint32_t num_chunks, double* __restrict__ out) {
+    __shared__ double warp_sums[8];
+    const uint32_t j = threadIdx.x;
+    for (uint32_t c = blockIdx.x; c < num_chunks; c += gridDim.x) {
+        const void* g = work[c].g;
+        const uint32_t len = work[c].len;
+        double acc = 0.0;
+        if (len == kTreeBlock && (reinterpret_cast<uintptr_t>(g) & 15u) == 0) {
+            if (G32) {
+                const float4* src = reinterpret_cast<const float4*>(g) + j;
+                float4 q[8];
+#pragma unroll
+                for (int r = 0; r < 8; ++r) q[r] = __ldcs(src + r * 256);
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    acc = add_square(acc, q[r].x);
+                    acc = add_square(acc, q[r].y);
+                    acc = add_square(acc, q[r].z);
+                    acc = add_square(acc, q[r].w);
+                }
+            } else {
+                const uint2* src = reinterpret_cast<const uint2*>(g) + j;
+                uint2 q[8];
+#pragma unroll
+                for (int r = 0; r < 8; ++r) q[r] = __ldcs(src + r * 256);
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    acc = add_square(acc, bf16_lo(q[r].x));
+                    acc = add_square(acc, bf16_hi(q[r].x));
+                    acc = add_square(acc, bf16_lo(q[r].y));
+                    acc = add_square(acc, bf16_hi(q[r].y));
+                }
+            }
+        } else {
+            for (int r = 0; r < 8; ++r)
+                for (int k = 0; k < 4; ++k) {
+                    const uint32_t e = static_cast<uint32_t>(r) * 1024u + 4u * j + k;
+                    if (e < len) {
+                        const float gi = G32 ? static_cast<const float*>(g)[e]
+                                             : __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t*>(g)[e]) << 16);
+                        acc = add_square(acc, gi);
+                    }
+                }
+        }
+        const double total = fold_block(acc, warp_sums);
+        if (j == 0) out[c] = total;
+    }
+}
+
 // Later passes: the same rule on an array of doubles (no squaring).
 __global__ void __launch_bounds__(kTreeThreads)
 k_tree_pass(const double* __restrict__ in, uint64_t count, uint64_t num_blocks, double* __restrict__ out) {
@@ -134,6 +187,45 @@ uint64_t sqnorm_scratch_doubles(uint64_t n) {
         count = blocks_of(count);
     }
     return total;
+}
+
+// Scratch of the list norm: one double per chunk plus every later level (nothing for 0 or 1 chunks).
+uint64_t sqnorm_mt_scratch_doubles(uint64_t num_chunks) {
+    uint64_t total = 0;
+    uint64_t count = num_chunks;
+    while (count > 1) {
+        total += count;
+        count = blocks_of(count);
+    }
+    return total;
+}
+
+cudaError_t launch_sqnorm_mt(const MtWork* work, uint32_t num_chunks, bool g_f32, double* out, double* scratch,
+                             const DeviceInfo& dev, cudaStream_t stream) {
+    if (num_chunks == 0) return cudaMemsetAsync(out, 0, sizeof(double), stream);
+    uint64_t count = num_chunks;
+    double* level_out = count == 1 ? out : scratch;
+    const uint64_t cap = static_cast<uint64_t>(dev.sm_count) * 8u;
+    {
+        const unsigned grid = static_cast<unsigned>(count < cap ? count : cap);
+        if (g_f32)
+            k_sqnorm_mt_pass1<true><<<grid, kTreeThreads, 0, stream>>>(work, num_chunks, level_out);
+        else
+            k_sqnorm_mt_pass1<false><<<grid, kTreeThreads, 0, stream>>>(work, num_chunks, level_out);
+        cudaError_t err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+    }
+    while (count > 1) {
+        const uint64_t next = blocks_of(count);
+        const double* level_in = level_out;
+        level_out = next == 1 ? out : level_out + count;
+        const unsigned grid = static_cast<unsigned>(next < cap ? next : cap);
+        k_tree_pass<<<grid, kTreeThreads, 0, stream>>>(level_in, count, next, level_out);
+        cudaError_t err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+        count = next;
+    }
+    return cudaSuccess;
 }
 
 cudaError_t launch_sqnorm(const void* g, bool g_f32, uint64_t n, double* out, double* scratch,

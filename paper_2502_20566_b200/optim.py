@@ -25,13 +25,16 @@ class SRAdamW(torch.optim.Optimizer):
         paper's update-only SR, 0 plain nearest rounding.
     eps_inside: the other reading of the update step, epsilon under the square root.
     seed: the shared random state; give every data-parallel replica the same value.
-    ``step(grad_scale=...)`` multiplies the gradients by a host scalar, ``step(grad_scale_dev=t)`` by a device
-    scalar (e.g. the output of ``sr_clip_scale``), without an extra pass over them.
+    max_norm: clip the global gradient norm (over all groups) to this value; the norm, the clipping factor and
+        the step all stay on the device (``grad_sqnorm_multi_tensor`` -> ``sr_clip_scale`` -> step).
+    ``step(grad_scale=...)`` multiplies the gradients by a host scalar (with clipping: the factor the norm is
+    taken under, e.g. 1 / accumulation steps), ``step(grad_scale_dev=t)`` by a device scalar, without an extra
+    pass over them.
     """
 
     def __init__(self, params: Iterable, lr: float = 1e-3, betas=(0.9, 0.999), eps: float = 1e-8,
                  weight_decay: float = 1e-2, seed: int = 0, sr_flags: int = binding.SR_FLAGS_DEFAULT,
-                 eps_inside: bool = False):
+                 eps_inside: bool = False, max_norm: Optional[float] = None):
         if lr < 0 or not 0 <= betas[0] < 1 or not 0 <= betas[1] < 1 or eps < 0:
             raise ValueError("invalid hyper-parameter")
         if sr_flags & ~7:
@@ -40,8 +43,10 @@ class SRAdamW(torch.optim.Optimizer):
         super().__init__(params, defaults)
         self.seed = int(seed)
         self.flags = int(sr_flags) | (binding.SR_FLAG_EPS_INSIDE if eps_inside else 0)
+        self.max_norm = max_norm
         self._steps = 0
-        self._plans = {}          # group index -> (key of data pointers, plan)
+        self._plans = {}          # group index (or "all" for the norm) -> (key of data pointers, plan)
+        self._clip = None         # device scalars and workspace of the clipped step
         binding.lib()             # fail here, not in the first step, when the CUDA library is missing
         for group in self.param_groups:
             for p in group["params"]:
@@ -56,7 +61,7 @@ class SRAdamW(torch.optim.Optimizer):
             st["exp_avg_sq"] = torch.zeros_like(p, memory_format=torch.contiguous_format)
         return st["exp_avg"], st["exp_avg_sq"]
 
-    def _plan(self, gi: int, group) -> Optional[binding.MtPlan]:
+    def _plan(self, gi, group) -> Optional[binding.MtPlan]:
         P, G, M, V = [], [], [], []
         g_dtype = None
         for p in group["params"]:
@@ -93,6 +98,10 @@ class SRAdamW(torch.optim.Optimizer):
             with torch.enable_grad():
                 loss = closure()
         self._steps += 1
+        if self.max_norm is not None:
+            if grad_scale_dev is not None:
+                raise ValueError("max_norm computes the device scale itself")
+            grad_scale_dev, grad_scale = self._clip_scale(grad_scale), 1.0
         base = 0
         for gi, group in enumerate(self.param_groups):
             plan = self._plan(gi, group)
@@ -103,6 +112,22 @@ class SRAdamW(torch.optim.Optimizer):
                 binding.sr_adamw_multi_tensor(plan, hp, self.seed, self._steps, tensor_id_base=base)
             base += len(group["params"])
         return loss
+
+    def _clip_scale(self, accum_scale: float) -> Optional[torch.Tensor]:
+        """Device scalar accum_scale * min(1, max_norm / (accum_scale * ||g|| + 1e-6)) over every gradient."""
+        everything = dict(params=[p for group in self.param_groups for p in group["params"]])
+        plan = self._plan("all", everything)
+        if plan is None:
+            return None
+        need = binding.grad_sqnorm_multi_tensor_workspace_bytes(plan)
+        if self._clip is None or self._clip[2].numel() * 8 < need:
+            dev = plan.device
+            self._clip = (torch.zeros(1, dtype=torch.float64, device=dev), torch.zeros(1, dtype=torch.float32, device=dev),
+                          torch.empty(max(1, need // 8), dtype=torch.float64, device=dev))
+        S, gs, ws = self._clip
+        binding.grad_sqnorm_multi_tensor(plan, S, ws)
+        binding.sr_clip_scale(S, accum_scale, self.max_norm, gs)
+        return gs
 
     # ---- checkpointing: seed and step count are the whole random state -------------------------
     def state_dict(self):

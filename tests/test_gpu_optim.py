@@ -116,3 +116,64 @@ def test_resume_from_checkpoint_is_bit_exact(env):
     for pa, pc in zip(a, c):
         assert np.array_equal(bits(pa), bits(pc))
         assert np.array_equal(bits(opt_a.state[pa]["exp_avg_sq"]), bits(opt_c.state[pc]["exp_avg_sq"]))
+
+
+@pytest.mark.parametrize("g_dtype", [torch.float32, torch.bfloat16])
+def test_list_norm_bit_exact(env, g_dtype):
+    """grad_sqnorm_multi_tensor against the oracle on lists with ragged, empty, tiny and unaligned tensors; a
+    list of one tensor equals grad_sqnorm."""
+    oracle, binding, _, synth, dev = env
+    rng = np.random.default_rng(3)
+    sizes = [1, 5, 8192, 8193, 0, 3 * 8192, 70001, 17, 2 * 8192 + 9] + [int(x) for x in rng.integers(1, 40000, 60)]
+    P, G, M, V = [], [], [], []
+    for i, n in enumerate(sizes):
+        shift = 1 if i % 7 == 2 else 0
+        p, g, m, v = synth.adamw_state(n + shift, 300 + i, dev, g_dtype=g_dtype, outlier_fraction=0.01)
+        P.append(p[shift:]); G.append(g[shift:]); M.append(m[shift:]); V.append(v[shift:])
+    plan = binding.sr_mt_plan_create(P, G, M, V)
+    ws = torch.empty(max(1, binding.grad_sqnorm_multi_tensor_workspace_bytes(plan) // 8), dtype=torch.float64, device=dev)
+    S = torch.zeros(1, dtype=torch.float64, device=dev)
+    host = [g.cpu().numpy().copy() if g_dtype == torch.float32 else bits(g) for g in G]
+    for _ in range(2):
+        binding.grad_sqnorm_multi_tensor(plan, S, ws)
+        torch.cuda.synchronize()
+        assert float(S.item()).hex() == oracle.sqnorm_list(host).hex()
+    plan.destroy()
+    one = binding.sr_mt_plan_create(P[6:7], G[6:7], M[6:7], V[6:7])
+    ws1 = torch.empty(max(1, binding.grad_sqnorm_multi_tensor_workspace_bytes(one) // 8), dtype=torch.float64, device=dev)
+    S1, S2 = torch.zeros(1, dtype=torch.float64, device=dev), torch.zeros(1, dtype=torch.float64, device=dev)
+    binding.grad_sqnorm_multi_tensor(one, S1, ws1)
+    ws2 = torch.empty(max(1, binding.grad_sqnorm_workspace_bytes(sizes[6]) // 8), dtype=torch.float64, device=dev)
+    binding.grad_sqnorm(G[6], S2, ws2)
+    torch.cuda.synchronize()
+    assert float(S1.item()).hex() == float(S2.item()).hex()
+    one.destroy()
+    empty = binding.sr_mt_plan_create([], [], [], [])
+    binding.grad_sqnorm_multi_tensor(empty, S, None)
+    torch.cuda.synchronize()
+    assert float(S.item()) == 0.0
+
+
+def test_clipped_optimizer_step_is_the_oracle_sequence(env):
+    oracle, binding, optim, synth, dev = env
+    gen = torch.Generator(device=dev).manual_seed(21)
+    shapes = [(500, 40), (40,), (9000,), (3,)]
+    params = [torch.nn.Parameter((torch.randn(s, device=dev, generator=gen) * 0.05).bfloat16()) for s in shapes]
+    groups = [dict(params=params[:2], weight_decay=0.1), dict(params=params[2:], weight_decay=0.0)]
+    opt = optim.SRAdamW(groups, lr=6e-4, betas=(0.9, 0.95), seed=77, max_norm=0.5)
+    host = [dict(p=bits(p).reshape(-1), m=np.zeros(p.numel(), np.uint16), v=np.zeros(p.numel(), np.uint16)) for p in params]
+    for step in (1, 2):
+        for p in params:
+            p.grad = (torch.randn(p.shape, device=dev, generator=gen) * (0.02 if step == 1 else 1e-4)).bfloat16()   # clipped, then not
+        opt.step(grad_scale=0.25)
+        torch.cuda.synchronize()
+        gh = [bits(p.grad).reshape(-1) for p in params]
+        S = oracle.sqnorm_list(gh)
+        gscale = oracle.clip_scale(S, 0.25, 0.5)
+        assert (gscale < 0.25) == (step == 1)
+        for i, p in enumerate(params):
+            kw = dict(lr=6e-4, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1 if i < 2 else 0.0)
+            h = host[i]
+            oracle.adamw_step(h["p"], gh[i], h["m"], h["v"], oracle.hparams(**kw), 77, step, i, 0, gscale)
+            assert np.array_equal(bits(p).reshape(-1), h["p"])
+            assert np.array_equal(bits(opt.state[p]["exp_avg"]).reshape(-1), h["m"])
