@@ -100,9 +100,23 @@ __global__ void __launch_bounds__(kTreeThreads)
 k_sqnorm_mt_pass1(const MtWork* __restrict__ work, uint32_t num_chunks, double* __restrict__ out) {
     __shared__ double warp_sums[8];
     const uint32_t j = threadIdx.x;
-    for (uint32_t c = blockIdx.x; c < num_chunks; c += gridDim.x) {
-        const void* g = work[c].g;
-        const uint32_t len = work[c].len;
+    // the entry after the current one is fetched before the current chunk's data, so that its latency
+    // is not paid between chunks
+    uint64_t c = blockIdx.x;
+    const void* g = nullptr;
+    uint32_t len = 0;
+    if (c < num_chunks) {
+        g = work[c].g;
+        len = work[c].len;
+    }
+    for (; c < num_chunks; c += gridDim.x) {
+        const uint64_t cn = c + gridDim.x;
+        const void* g_next = nullptr;
+        uint32_t len_next = 0;
+        if (cn < num_chunks) {
+            g_next = work[cn].g;
+            len_next = work[cn].len;
+        }
         double acc = 0.0;
         if (len == kTreeBlock && (reinterpret_cast<uintptr_t>(g) & 15u) == 0) {
             if (G32) {
@@ -143,6 +157,8 @@ k_sqnorm_mt_pass1(const MtWork* __restrict__ work, uint32_t num_chunks, double* 
         }
         const double total = fold_block(acc, warp_sums);
         if (j == 0) out[c] = total;
+        g = g_next;
+        len = len_next;
     }
 }
 
