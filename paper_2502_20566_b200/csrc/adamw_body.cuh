@@ -19,6 +19,27 @@ __device__ __forceinline__ void st16(void* base, uint64_t vec, uint4 val) {
     __stcs(reinterpret_cast<uint4*>(base) + vec, val);
 }
 
+// 32-byte accesses (the 256-bit vector loads/stores of sm_100): eight consecutive 32-bit words per
+// thread.  A warp then touches each 32-byte sector of its 1 KB once, where two 16-byte accesses at a
+// 32-byte stride touch every sector twice.  The address (base + 32 * vec) must be 32-byte aligned.
+struct Words8 {
+    uint32_t w[8];
+};
+__device__ __forceinline__ Words8 ld32(const void* base, uint64_t vec) {
+    Words8 r;
+    asm volatile("ld.global.cs.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]), "=r"(r.w[4]), "=r"(r.w[5]), "=r"(r.w[6]), "=r"(r.w[7])
+                 : "l"(static_cast<const char*>(base) + 32 * vec));
+    return r;
+}
+__device__ __forceinline__ void st32(void* base, uint64_t vec, const Words8& r) {
+    asm volatile("st.global.cs.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"
+                 :
+                 : "r"(r.w[0]), "r"(r.w[1]), "r"(r.w[2]), "r"(r.w[3]), "r"(r.w[4]), "r"(r.w[5]), "r"(r.w[6]), "r"(r.w[7]),
+                   "l"(static_cast<char*>(base) + 32 * vec)
+                 : "memory");
+}
+
 // ---- asynchronous global -> shared copies (16 bytes, L2 only) ---------------------------------
 // Used to keep a thread's NEXT vector in flight while it computes the current one without
 // spending registers on it.  Each thread copies into and reads from its own shared-memory slots,
@@ -50,9 +71,16 @@ __device__ __forceinline__ void unpack_grad8(const uint4 g0, const uint4 g1, flo
 }
 
 // the eight gradient values of a vector as FP32
+// wide (FP32 gradients only): the gradient buffer is 32-byte aligned, one 32-byte load.  Used by the
+// FP32-master kernel; in the SR step kernels it measured 1.8 % slower than the two 16-byte loads
+// (same GPU, 832M elements), so they do not ask for it.
 template <bool G32>
-__device__ __forceinline__ void load_grad8(const void* g, uint64_t vec, float (&ge)[8]) {
-    if (G32) {
+__device__ __forceinline__ void load_grad8(const void* g, uint64_t vec, float (&ge)[8], bool wide = false) {
+    if (G32 && wide) {
+        const Words8 r = ld32(g, vec);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) ge[e] = __uint_as_float(r.w[e]);
+    } else if (G32) {
         const uint4 g0 = ld16(g, 2 * vec);
         const uint4 g1 = ld16(g, 2 * vec + 1);
         ge[0] = __uint_as_float(g0.x); ge[1] = __uint_as_float(g0.y);

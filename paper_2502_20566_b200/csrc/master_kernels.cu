@@ -42,7 +42,9 @@ __device__ __forceinline__ void master_scalar(float* p, uint16_t* p16, const voi
 // Eight consecutive elements per thread-iteration: 6 x 16-byte loads for x, m, v, one or two for g;
 // 6 x 16-byte stores and one for the BF16 copy.  FAST: branch-free arithmetic inside the validated
 // operand range with the reference arithmetic as fallback for the vector, as in the SR kernels.
-template <bool G32, bool FAST, bool SCALE>
+// WIDE: x, m, v (and FP32 g) are 32-byte aligned and move with one 32-byte access per thread and
+// array (measured on B200: 84 % -> 94 % of the copy peak on 832M elements).
+template <bool G32, bool FAST, bool SCALE, bool WIDE>
 __global__ void __launch_bounds__(kBlockThreads, 4)
 k_master_adamw(float* p, uint16_t* p16, const void* g, float* m, float* v, uint64_t n, bool vec_ok,
                const __grid_constant__ StepScalars S) {
@@ -55,14 +57,31 @@ k_master_adamw(float* p, uint16_t* p16, const void* g, float* m, float* v, uint6
     }
     const uint64_t nvec = n >> 3;
     for (uint64_t vec = tid; vec < nvec; vec += stride) {
-        const float4 pa = ldf4(p, 2 * vec), pb = ldf4(p, 2 * vec + 1);
-        const float4 ma = ldf4(m, 2 * vec), mb = ldf4(m, 2 * vec + 1);
-        const float4 va = ldf4(v, 2 * vec), vb = ldf4(v, 2 * vec + 1);
-        float ge[8];
-        load_grad8<G32>(g, vec, ge);
-        const float x[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
-        const float mm[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
-        const float vv[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+        float x[8], mm[8], vv[8], ge[8];
+        if (WIDE) {
+            const Words8 pw = ld32(p, vec), mw = ld32(m, vec), vw = ld32(v, vec);
+            load_grad8<G32>(g, vec, ge, true);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                x[e] = __uint_as_float(pw.w[e]);
+                mm[e] = __uint_as_float(mw.w[e]);
+                vv[e] = __uint_as_float(vw.w[e]);
+            }
+        } else {
+            const float4 pa = ldf4(p, 2 * vec), pb = ldf4(p, 2 * vec + 1);
+            const float4 ma = ldf4(m, 2 * vec), mb = ldf4(m, 2 * vec + 1);
+            const float4 va = ldf4(v, 2 * vec), vb = ldf4(v, 2 * vec + 1);
+            load_grad8<G32>(g, vec, ge);
+            const float xs[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
+            const float ms[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
+            const float vs[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                x[e] = xs[e];
+                mm[e] = ms[e];
+                vv[e] = vs[e];
+            }
+        }
         ElementOut r[8];
         bool redo = !FAST;
         if (FAST) {
@@ -80,12 +99,25 @@ k_master_adamw(float* p, uint16_t* p16, const void* g, float* m, float* v, uint6
 #pragma unroll
             for (int e = 0; e < 8; ++e) r[e] = adamw_element(x[e], ge[e], mm[e], vv[e], gscale, S);
         }
-        stf4(p, 2 * vec, r[0].x, r[1].x, r[2].x, r[3].x);
-        stf4(p, 2 * vec + 1, r[4].x, r[5].x, r[6].x, r[7].x);
-        stf4(m, 2 * vec, r[0].m, r[1].m, r[2].m, r[3].m);
-        stf4(m, 2 * vec + 1, r[4].m, r[5].m, r[6].m, r[7].m);
-        stf4(v, 2 * vec, r[0].v, r[1].v, r[2].v, r[3].v);
-        stf4(v, 2 * vec + 1, r[4].v, r[5].v, r[6].v, r[7].v);
+        if (WIDE) {
+            Words8 xo, mo, vo;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                xo.w[e] = __float_as_uint(r[e].x);
+                mo.w[e] = __float_as_uint(r[e].m);
+                vo.w[e] = __float_as_uint(r[e].v);
+            }
+            st32(p, vec, xo);
+            st32(m, vec, mo);
+            st32(v, vec, vo);
+        } else {
+            stf4(p, 2 * vec, r[0].x, r[1].x, r[2].x, r[3].x);
+            stf4(p, 2 * vec + 1, r[4].x, r[5].x, r[6].x, r[7].x);
+            stf4(m, 2 * vec, r[0].m, r[1].m, r[2].m, r[3].m);
+            stf4(m, 2 * vec + 1, r[4].m, r[5].m, r[6].m, r[7].m);
+            stf4(v, 2 * vec, r[0].v, r[1].v, r[2].v, r[3].v);
+            stf4(v, 2 * vec + 1, r[4].v, r[5].v, r[6].v, r[7].v);
+        }
         st16(p16, vec, make_uint4(rne_pair(r[0].x, r[1].x), rne_pair(r[2].x, r[3].x), rne_pair(r[4].x, r[5].x),
                                   rne_pair(r[6].x, r[7].x)));
     }
@@ -93,13 +125,22 @@ k_master_adamw(float* p, uint16_t* p16, const void* g, float* m, float* v, uint6
     if (tid < n - done) master_scalar<G32>(p, p16, g, m, v, done + tid, gscale, S);
 }
 
-template <bool G32, bool FAST, bool SCALE>
-cudaError_t launch_master_t(float* p, uint16_t* p16, const void* g, float* m, float* v, uint64_t n, bool vec_ok,
+template <bool G32, bool FAST, bool SCALE, bool WIDE>
+cudaError_t launch_master_w(float* p, uint16_t* p16, const void* g, float* m, float* v, uint64_t n, bool vec_ok,
                             const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream) {
-    auto k = k_master_adamw<G32, FAST, SCALE>;
+    auto k = k_master_adamw<G32, FAST, SCALE, WIDE>;
     const uint64_t items = vec_ok ? (n >> 3) + 8 : n;
     k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, p16, g, m, v, n, vec_ok, S);
     return cudaGetLastError();
+}
+
+template <bool G32, bool FAST, bool SCALE>
+cudaError_t launch_master_t(float* p, uint16_t* p16, const void* g, float* m, float* v, uint64_t n, bool vec_ok,
+                            const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream) {
+    auto aligned32 = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 31u) == 0; };
+    const bool wide = vec_ok && aligned32(p) && aligned32(m) && aligned32(v) && (!G32 || aligned32(g));
+    return wide ? launch_master_w<G32, FAST, SCALE, true>(p, p16, g, m, v, n, vec_ok, S, dev, stream)
+                : launch_master_w<G32, FAST, SCALE, false>(p, p16, g, m, v, n, vec_ok, S, dev, stream);
 }
 
 }  // namespace

@@ -154,6 +154,28 @@ def test_eps_inside_list_and_master_recipe(env):
     assert mismatches(bits(p16), want16) == 0
 
 
+@pytest.mark.parametrize("shift", [0, 4, 12])
+def test_fp32_gradient_alignments(env, shift):
+    """FP32 gradient buffers at 32-byte and at 16-byte-only alignment (shift counts 4-byte steps: 4 and 12 leave
+    16-byte alignment only), flat and list."""
+    oracle, binding, synth, dev = env
+    n = 200003
+    p, g, m, v = synth.adamw_state(n + 32, 77, dev, g_dtype=torch.float32)
+    g = g[shift:shift + n]
+    p, m, v = (t[:n] for t in (p, m, v))
+    assert g.data_ptr() % 16 == 0 and (g.data_ptr() % 32 == 0) == (shift % 8 == 0)
+    assert run_both(env, p, g, m, v, HP, seed=8, step=3, gscale=0.25) == (0, 0, 0)
+    P, G, M, V = [p[:70000], p[70000:]], [g[:70000], g[70000:]], [m[:70000], m[70000:]], [v[:70000], v[70000:]]
+    plan = binding.sr_mt_plan_create(P, G, M, V)
+    host = [[bits(t) for t in P], [host_g(t) for t in G], [bits(t) for t in M], [bits(t) for t in V]]
+    binding.sr_adamw_multi_tensor(plan, binding.hparams(**HP), 8, 4, tensor_id_base=3)
+    torch.cuda.synchronize()
+    for i in range(2):
+        oracle.adamw_step(host[0][i], host[1][i], host[2][i], host[3][i], oracle.hparams(**HP), 8, 4, 3 + i)
+        assert mismatches(bits(P[i]), host[0][i]) + mismatches(bits(M[i]), host[2][i]) + mismatches(bits(V[i]), host[3][i]) == 0
+    plan.destroy()
+
+
 def test_flat_step_special_values(env):
     """NaN, infinities, zeros, subnormals and huge values in every input."""
     _, _, synth, dev = env
@@ -648,18 +670,21 @@ def test_host_resident_step_equals_oracle(env, g_dtype):
 # FP32-master comparison recipe
 # ---------------------------------------------------------------------------------------------
 
-@pytest.mark.parametrize("n,shift", [(0, 0), (5, 0), (8 * 4096 + 3, 0), ((1 << 22) + 11, 0), (9001, 1)])
+@pytest.mark.parametrize("n,shift", [(0, 0), (5, 0), (8 * 4096 + 3, 0), ((1 << 22) + 11, 0), (9001, 1), (70003, 4)])
 @pytest.mark.parametrize("g_dtype,gscale", [(torch.bfloat16, 1.0), (torch.float32, 0.125)])
 def test_master_recipe_bit_exact(env, n, shift, g_dtype, gscale):
     """FP32 master weights and moments + nearest-rounded BF16 copy (the paper's mixed-precision
-    comparison): two consecutive steps, every FP32 word and every BF16 pattern equal to the oracle's."""
+    comparison): two consecutive steps, every FP32 word and every BF16 pattern equal to the oracle's.
+    shift moves every buffer by 4 * shift bytes: 1 = unaligned (element-wise path), 4 = 16-byte but not
+    32-byte aligned (16-byte accesses), 0 = 32-byte accesses."""
     oracle, binding, synth, dev = env
-    p0, g, m0, v0 = synth.adamw_state(n + shift, 31 + n, dev, g_dtype=g_dtype)
-    p, m, v = (t.float()[shift:] for t in (p0, m0, v0))
-    g = g[shift:]
+    s16 = 2 * shift                                  # BF16 buffers: twice the elements for the same bytes
+    p0, g, m0, v0 = synth.adamw_state(n + 2 * shift, 31 + n, dev, g_dtype=g_dtype)
+    p, m, v = (t.float()[shift:shift + n] for t in (p0, m0, v0))
+    g = g[shift:shift + n] if g_dtype == torch.float32 else g[s16:s16 + n]
     if n > 100:
         p[7], m[11], v[13], v[17] = float("nan"), float("inf"), 0.0, 1e-30      # vectors that leave the fast range
-    p16 = torch.zeros(n + shift, dtype=torch.bfloat16, device=dev)[shift:]
+    p16 = torch.zeros(n + s16, dtype=torch.bfloat16, device=dev)[s16:]
     ph, mh, vh = (t.cpu().numpy().copy() for t in (p, m, v))
     gh = host_g(g)
     hp_kw = dict(HP)
