@@ -22,7 +22,7 @@ __device__ __forceinline__ float accumulate(float acc, float g, float scale) {
     return __fadd_rn(acc, __fmul_rn(scale, g));
 }
 
-// MODE 0: element-wise; 1: 16-byte vectors, per-element noise (offset not a multiple of 8); 2: vectors, grouped
+// MODE 0: element-wise; 1: 16-byte vectors straddling two noise groups (offset not a multiple of 8); 2: vectors, grouped
 template <bool G32, bool SR, int MODE>
 __global__ void __launch_bounds__(kBlockThreads)
 k_sr_accumulate(uint16_t* acc, const void* g, uint64_t n, float scale, uint64_t elem_offset, uint32_t tensor_id,
@@ -41,21 +41,16 @@ k_sr_accumulate(uint16_t* acc, const void* g, uint64_t n, float scale, uint64_t 
             if (SR && MODE == 2)
                 w = philox4x32_10(static_cast<uint32_t>(idx0 >> 1) | kAccumSlot, static_cast<uint32_t>(idx0 >> 33), tensor_id,
                                   seed_hi, K);
+            else if (SR)
+                w = straddling_noise(idx0, kAccumSlot, tensor_id, seed_hi, K);
             uint32_t o[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const uint32_t aw = word_of(av, j);
                 const float s0 = accumulate(bf16_lo(aw), ge[2 * j], scale);
                 const float s1 = accumulate(bf16_hi(aw), ge[2 * j + 1], scale);
-                uint32_t r0, r1;
-                if (!SR || MODE == 2) {
-                    r0 = round_sum_word_nan_safe<SR, false>(s0, word_of(w, j));
-                    r1 = round_sum_word_nan_safe<SR, true>(s1, word_of(w, j));
-                } else {
-                    r0 = round_sum_r16_nan_safe<true>(s0, noise_of_element(idx0 + 2 * j, kAccumSlot, tensor_id, seed_hi, K));
-                    r1 = round_sum_r16_nan_safe<true>(s1, noise_of_element(idx0 + 2 * j + 1, kAccumSlot, tensor_id, seed_hi, K));
-                }
-                o[j] = pack_top_halves(r0, r1);
+                o[j] = pack_top_halves(round_sum_word_nan_safe<SR, false>(s0, word_of(w, j)),
+                                       round_sum_word_nan_safe<SR, true>(s1, word_of(w, j)));
             }
             st16(acc, vec, make_uint4(o[0], o[1], o[2], o[3]));
         }

@@ -98,11 +98,30 @@ __device__ __forceinline__ void load_grad8(const void* g, uint64_t vec, float (&
 
 __device__ __forceinline__ uint32_t word_of(const uint4& w, int j) { return j == 0 ? w.x : j == 1 ? w.y : j == 2 ? w.z : w.w; }
 
+// Noise words of one slot for a vector whose first element sits at position r = idx0 & 7 of its
+// noise group: the vector takes the last 8 - r halfwords of group A = idx0 >> 3 and the first r of
+// group A + 1, i.e. 128 bits starting at bit 16 r of the 256-bit string (call A : call A + 1).
+// r is the same for every vector of a launch, so the word shifts below are uniform selects.
+__device__ __forceinline__ uint4 straddling_noise(uint64_t idx0, uint32_t slot, uint32_t c2, uint32_t c3, const PhiloxKeys& K) {
+    const uint64_t num_a = ((idx0 >> 3) << 2) | slot, num_b = num_a + 4;
+    const uint4 a = philox4x32_10(static_cast<uint32_t>(num_a), static_cast<uint32_t>(num_a >> 32), c2, c3, K);
+    const uint4 b = philox4x32_10(static_cast<uint32_t>(num_b), static_cast<uint32_t>(num_b >> 32), c2, c3, K);
+    const uint32_t r = static_cast<uint32_t>(idx0) & 7u;
+    const bool by2 = (r & 4u) != 0, by1 = (r & 2u) != 0;
+    // words r>>1 .. (r>>1)+4 of (a.x a.y a.z a.w b.x b.y b.z b.w)
+    const uint32_t x0 = by2 ? a.z : a.x, x1 = by2 ? a.w : a.y, x2 = by2 ? b.x : a.z, x3 = by2 ? b.y : a.w;
+    const uint32_t x4 = by2 ? b.z : b.x, x5 = by2 ? b.w : b.y;
+    const uint32_t y0 = by1 ? x1 : x0, y1 = by1 ? x2 : x1, y2 = by1 ? x3 : x2, y3 = by1 ? x4 : x3, y4 = by1 ? x5 : x4;
+    const uint32_t sh = (r & 1u) * 16u;
+    return make_uint4(__funnelshift_r(y0, y1, sh), __funnelshift_r(y1, y2, sh), __funnelshift_r(y2, y3, sh),
+                      __funnelshift_r(y3, y4, sh));
+}
+
 // ---- reference vector: IEEE square root / division, NaN rule -------------------------------
 // GROUPED = true needs idx0 (global index of the vector's first element) to be a multiple of 8: the
-// vector is then exactly one noise group and three Philox calls serve it.  GROUPED = false draws
-// every element's noise on its own and is valid for any idx0.  Kept out of line: the fast kernels
-// call it only for the rare vector that leaves the fast range.
+// vector is then exactly one noise group and three Philox calls serve it.  GROUPED = false is valid
+// for any idx0: the vector straddles two groups and takes six calls.  Kept out of line: the fast
+// kernels call it only for the rare vector that leaves the fast range.
 template <bool G32, uint32_t FLAGS, bool GROUPED>
 __device__ __noinline__ void step_vec8_reference(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t vec,
                                                  uint64_t idx0, uint32_t c2, uint32_t c3, float gscale,
@@ -116,6 +135,10 @@ __device__ __noinline__ void step_vec8_reference(uint16_t* p, const void* g, uin
         if (FLAGS & 1u) wx = philox4x32_10(c0, c1, c2, c3, K);
         if (FLAGS & 2u) wm = philox4x32_10(c0 + 1, c1, c2, c3, K);
         if (FLAGS & 4u) wv = philox4x32_10(c0 + 2, c1, c2, c3, K);
+    } else {
+        if (FLAGS & 1u) wx = straddling_noise(idx0, 0, c2, c3, K);
+        if (FLAGS & 2u) wm = straddling_noise(idx0, 1, c2, c3, K);
+        if (FLAGS & 4u) wv = straddling_noise(idx0, 2, c2, c3, K);
     }
     uint32_t po[4], mo[4], vo[4];
 #pragma unroll
@@ -123,19 +146,9 @@ __device__ __noinline__ void step_vec8_reference(uint16_t* p, const void* g, uin
         const uint32_t pw = word_of(pv, j), mw = word_of(mv, j), vw = word_of(vv, j);
         const ElementOut r0 = adamw_element(bf16_lo(pw), ge[2 * j], bf16_lo(mw), bf16_lo(vw), gscale, S);
         const ElementOut r1 = adamw_element(bf16_hi(pw), ge[2 * j + 1], bf16_hi(mw), bf16_hi(vw), gscale, S);
-        uint32_t x0, x1, m0, m1, v0, v1;   // 16-bit noise per element and slot
-        if (GROUPED) {
-            const uint32_t ax = word_of(wx, j), am = word_of(wm, j), av = word_of(wv, j);
-            x0 = ax & 0xFFFFu; x1 = ax >> 16; m0 = am & 0xFFFFu; m1 = am >> 16; v0 = av & 0xFFFFu; v1 = av >> 16;
-        } else {
-            const uint64_t i0 = idx0 + 2 * j, i1 = i0 + 1;
-            x0 = (FLAGS & 1u) ? noise_of_element(i0, 0, c2, c3, K) : 0u;
-            x1 = (FLAGS & 1u) ? noise_of_element(i1, 0, c2, c3, K) : 0u;
-            m0 = (FLAGS & 2u) ? noise_of_element(i0, 1, c2, c3, K) : 0u;
-            m1 = (FLAGS & 2u) ? noise_of_element(i1, 1, c2, c3, K) : 0u;
-            v0 = (FLAGS & 4u) ? noise_of_element(i0, 2, c2, c3, K) : 0u;
-            v1 = (FLAGS & 4u) ? noise_of_element(i1, 2, c2, c3, K) : 0u;
-        }
+        // 16-bit noise per element and slot: the pair's word holds the even element's in its low half
+        const uint32_t ax = word_of(wx, j), am = word_of(wm, j), av = word_of(wv, j);
+        const uint32_t x0 = ax & 0xFFFFu, x1 = ax >> 16, m0 = am & 0xFFFFu, m1 = am >> 16, v0 = av & 0xFFFFu, v1 = av >> 16;
         po[j] = pack_top_halves(round_sum_r16_nan_safe<(FLAGS & 1u) != 0>(r0.x, x0),
                                 round_sum_r16_nan_safe<(FLAGS & 1u) != 0>(r1.x, x1));
         mo[j] = pack_top_halves(round_sum_r16_nan_safe<(FLAGS & 2u) != 0>(r0.m, m0),

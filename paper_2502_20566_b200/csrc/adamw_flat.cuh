@@ -6,7 +6,8 @@
 namespace sradamw {
 
 // MODE 0: element-wise (any alignment, any offset)
-//      1: 16-byte vectors, reference arithmetic, per-element noise (elem_offset not a multiple of 8)
+//      1: 16-byte vectors, reference arithmetic, elem_offset not a multiple of 8: every vector straddles two
+//         noise groups (six Philox calls per vector)
 //      4: 16-byte vectors, reference arithmetic, one Philox call per (vector, slot): elem_offset a
 //         multiple of 8 but scalars outside what the branch-free arithmetic covers
 // Persistent grid: thread t takes vectors t, t + T, t + 2T, ... (T = threads in the grid).

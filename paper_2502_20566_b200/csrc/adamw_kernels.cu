@@ -28,7 +28,7 @@ __device__ __forceinline__ uint32_t cast_pair(uint32_t b_even, uint32_t b_odd, u
     return pack_top_halves(s0, s1);
 }
 
-// MODE 0: element-wise; 1: vectors, per-element noise (offset not a multiple of 8); 2: vectors, grouped
+// MODE 0: element-wise; 1: vectors straddling two noise groups (offset not a multiple of 8); 2: vectors, grouped
 template <int MODE>
 __global__ void __launch_bounds__(kBlockThreads)
 k_sr_downcast(const float* __restrict__ src, uint16_t* __restrict__ dst, uint64_t n, uint64_t elem_offset,
@@ -42,23 +42,15 @@ k_sr_downcast(const float* __restrict__ src, uint16_t* __restrict__ dst, uint64_
             const uint4 a = ld16(src, 2 * vec);
             const uint4 b = ld16(src, 2 * vec + 1);
             const uint64_t idx0 = elem_offset + (vec << 3);
+            // MODE 1: the vector straddles two noise groups (two Philox calls); MODE 2: it is one group
+            const uint4 w = MODE == 2 ? philox4x32_10(static_cast<uint32_t>(idx0 >> 1), static_cast<uint32_t>(idx0 >> 33),
+                                                      tensor_id, seed_hi, K)
+                                      : straddling_noise(idx0, 0, tensor_id, seed_hi, K);
             uint4 o;
-            if (MODE == 2) {
-                const uint4 w = philox4x32_10(static_cast<uint32_t>(idx0 >> 1), static_cast<uint32_t>(idx0 >> 33),
-                                              tensor_id, seed_hi, K);
-                o.x = cast_pair(a.x, a.y, w.x);
-                o.y = cast_pair(a.z, a.w, w.y);
-                o.z = cast_pair(b.x, b.y, w.z);
-                o.w = cast_pair(b.z, b.w, w.w);
-            } else {
-                const uint32_t in[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-                uint32_t s[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e)
-                    s[e] = round_sum_r16_nan_safe<true>(__uint_as_float(in[e]), noise_of_element(idx0 + e, 0, tensor_id, seed_hi, K));
-                o = make_uint4(pack_top_halves(s[0], s[1]), pack_top_halves(s[2], s[3]), pack_top_halves(s[4], s[5]),
-                               pack_top_halves(s[6], s[7]));
-            }
+            o.x = cast_pair(a.x, a.y, w.x);
+            o.y = cast_pair(a.z, a.w, w.y);
+            o.z = cast_pair(b.x, b.y, w.z);
+            o.w = cast_pair(b.z, b.w, w.w);
             st16(dst, vec, o);
         }
         done = nvec << 3;

@@ -176,6 +176,30 @@ def test_fp32_gradient_alignments(env, shift):
     plan.destroy()
 
 
+@pytest.mark.parametrize("r", [1, 2, 3, 4, 5, 6, 7])
+def test_offsets_that_split_noise_groups(env, r):
+    """elem_offset = r mod 8 with aligned buffers: every 16-byte vector takes its noise from two groups.  Step, cast
+    and accumulation, across a multiple of 2^33 in index space (where the high counter word changes)."""
+    oracle, binding, synth, dev = env
+    n = 40000 + r
+    offset = (1 << 36) - 20000 + r - 8
+    assert offset % 8 == r
+    for g_dtype, flags in ((torch.bfloat16, 7), (torch.float32, 5)):
+        p, g, m, v = synth.adamw_state(n, 60 + r, dev, g_dtype=g_dtype)
+        assert run_both(env, p, g, m, v, HP, seed=(7 << 32) | 3, step=12, tensor_id=9, elem_offset=offset, flags=flags) == (0, 0, 0)
+    src = synth.downcast_mix(n, 61, dev)
+    dst = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    binding.sr_downcast_f32_bf16(src, dst, seed=(7 << 32) | 3, step=1, tensor_id=2, elem_offset=offset)
+    torch.cuda.synchronize()
+    assert mismatches(bits(dst), oracle.sr_downcast(src.cpu().numpy().copy(), (7 << 32) | 3, 1, 2, offset)) == 0
+    _, g, acc, _ = synth.adamw_state(n, 62, dev)
+    want = bits(acc)
+    binding.sr_accumulate_bf16(acc, g, 0.5, seed=5, step=2, tensor_id=1, elem_offset=offset)
+    oracle.sr_accumulate(want, bits(g), 0.5, 5, 2, 1, offset, True)
+    torch.cuda.synchronize()
+    assert mismatches(bits(acc), want) == 0
+
+
 def test_flat_step_special_values(env):
     """NaN, infinities, zeros, subnormals and huge values in every input."""
     _, _, synth, dev = env
