@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0       # used only when MEASURED_PEAKS.json is absent
 # 2^30-element case (profiles/k_sr_adamw_flat_fast__long_launch_shape__2pow30.md: 5.794371 TB/s x 2.584544 ms);
 # the traffic of a streaming kernel grows in proportion to the element count, so the full-size figure is
 # this times n.  Set to None whenever the kernel changes until a new capture exists.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = 5.714450e12 * 2.620672e-3 / (1 << 30)
+NCU_TRAFFIC_BYTES_PER_ELEMENT = 5.780220e12 * 2.591168e-3 / (1 << 30)
 
 
 def parse_args():

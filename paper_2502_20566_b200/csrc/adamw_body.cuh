@@ -9,6 +9,10 @@
 
 #include "launch.h"
 
+#ifndef SR_PACKED_F32X2
+#define SR_PACKED_F32X2 1
+#endif
+
 namespace sradamw {
 
 // ---- 16-byte streaming accesses ------------------------------------------------------------
@@ -181,8 +185,14 @@ __device__ __forceinline__ void step_vec8_fast_loaded(uint16_t* p, const void* g
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const uint32_t pw = word_of(pv, j), mw = word_of(mv, j), vw = word_of(vv, j);
+#if SR_PACKED_F32X2
+        ElementOut r0, r1;
+        adamw_pair_in_range<SCALE>(bf16_lo(pw), bf16_hi(pw), ge[2 * j], ge[2 * j + 1], bf16_lo(mw), bf16_hi(mw), bf16_lo(vw),
+                                   bf16_hi(vw), gscale, S, r0, r1);
+#else
         const ElementOut r0 = adamw_element_in_range<SCALE>(bf16_lo(pw), ge[2 * j], bf16_lo(mw), bf16_lo(vw), gscale, S);
         const ElementOut r1 = adamw_element_in_range<SCALE>(bf16_hi(pw), ge[2 * j + 1], bf16_hi(mw), bf16_hi(vw), gscale, S);
+#endif
         track.add(r0, r1);
         po[j] = pack_top_halves(round_sum_word<(FLAGS & 1u) != 0, false>(r0.x, word_of(wx, j)),
                                 round_sum_word<(FLAGS & 1u) != 0, true>(r1.x, word_of(wx, j)));
