@@ -670,6 +670,45 @@ def test_flat_6p7b_every_element(env):
     assert nchunks == 100
 
 
+@pytest.mark.parametrize("flags,gscale,offset", [(7, 1.0, 0), (5, 0.25, (1 << 33) - (1 << 29))])
+def test_long_launch_tiles_with_ragged_tail_and_special_values(env, flags, gscale, offset):
+    """A launch long enough for the long-launch shape (2^30 elements) plus a ragged tail, with NaN / infinity /
+    zero / tiny values sprinkled in (vectors that fall back to the reference arithmetic), a gradient scale,
+    nearest rounding on m, and an offset that makes the buffer cross a multiple of 2^33 in index space.  Every
+    element is compared."""
+    oracle, binding, synth, dev = env
+    n = (1 << 30) + 3 * 4096 + 1237
+    guard = 64
+    roles = (synth.ROLE_P, synth.ROLE_G, synth.ROLE_M, synth.ROLE_V)
+    bufs = [torch.empty(n + guard, dtype=torch.bfloat16, device=dev) for _ in range(4)]
+    for t, role in zip(bufs, roles):
+        synth.fill_state(t[:n], role, 77)
+        t[n:] = 1.5
+    p, g, m, v = (t[:n] for t in bufs)
+    special = torch.tensor([float("nan"), float("inf"), -float("inf"), 0.0, -0.0, 1e-30, 3e38, 1e-40], device=dev).bfloat16()
+    for k, t in enumerate((p, g, m, v)):
+        pos = torch.arange(8, device=dev) * 977 + 13 + 131071 * k
+        t[pos] = special.abs() if k == 3 else special
+        t[pos + (1 << 29)] = special.abs() if k == 3 else special
+    before = [bits(t[c * synth.CHUNK:(c + 1) * synth.CHUNK]) for c in (0, 8) for t in (p, g, m, v)]
+    binding.sr_adamw_step(p, g, m, v, binding.hparams(**HP, grad_scale=gscale, flags=flags), 4321, 17, 5, offset)
+    torch.cuda.synchronize()
+    for t in bufs:
+        assert torch.all(t[n:] == 1.5)
+    hp_o = oracle.hparams(**HP, flags=flags)
+    nchunks = (n + synth.CHUNK - 1) // synth.CHUNK
+    for c in range(nchunks):
+        start = c * synth.CHUNK
+        length = min(synth.CHUNK, n - start)
+        if c in (0, 8):                               # the chunks that hold the special values
+            pre = [a.copy() for a in before[(0 if c == 0 else 4):(4 if c == 0 else 8)]]
+        else:
+            pre = [bits(synth.state_chunk(role, 77, c, length, dev)) for role in roles]
+        oracle.adamw_step(*pre, hp_o, 4321, 17, 5, offset + start, gscale)
+        bad = sum(mismatches(bits(t[start:start + length]), pre[k]) for k, t in ((0, p), (2, m), (3, v)))
+        assert bad == 0, f"chunk {c}"
+
+
 # ---------------------------------------------------------------------------------------------
 # host-resident state
 # ---------------------------------------------------------------------------------------------
