@@ -27,12 +27,13 @@ constexpr uint32_t kMtChunkElems = 8192;   // multiple of 8; never crosses a mul
 // 2..6 stages on the real kernels).  Every kernel's arithmetic needs about 96 registers; tighter
 // budgets cost more in instruction scheduling than they gain in occupancy.
 //  - kernels that load straight into registers: 128 threads, >= 5 blocks/SM (640 threads/SM);
-//  - the staged flat kernel has two shapes.  Long launches (>= 2^30 elements, tens of milliseconds,
+//  - the staged flat kernel has two shapes.  Long launches (>= 2^29 elements, milliseconds and more,
 //    which run into the board's power cap): 256 threads, 2 blocks/SM, 3 vectors per thread in
 //    flight or in use (48 KB of shared memory per block) -- with the memory latency covered by the
 //    staging, fewer resident warps ran faster under the cap (90% vs 86% of the copy peak at 6.7B).
-//    Shorter launches, which finish before the cap bites: 128 x 5 with 2 stages (93% vs 87% at
-//    355M elements);
+//    Shorter launches, which finish before the cap bites: 128 x 5 with 2 stages.  Same GPU, short vs
+//    long shape: 2^26 elements 0.155 vs 0.159 ms, 2^28 0.623 vs 0.641, 355M 0.827 vs 0.817-0.842,
+//    832M 1.95-2.05 vs 1.93-1.95: the long shape takes over between 2^28 and 2^30;
 //  - the staged multi-tensor kernel keeps 128 x 5 with 2 stages.
 #ifndef SR_BLOCK_THREADS
 #define SR_BLOCK_THREADS 128
@@ -56,7 +57,7 @@ constexpr int kFlatStagedMinBlocks = SR_FLAT_STAGED_MIN_BLOCKS;
 constexpr int kFlatStages = SR_FLAT_STAGES;
 constexpr int kMtStages = 2;
 constexpr int kShortStages = 2;
-constexpr uint64_t kLongLaunchElems = static_cast<uint64_t>(1) << 30;
+constexpr uint64_t kLongLaunchElems = static_cast<uint64_t>(1) << 29;
 
 struct DeviceInfo {
     int sm_count;
