@@ -48,6 +48,48 @@ __device__ __forceinline__ uint32_t sr_fp8_magnitude(uint32_t abits, uint32_t r)
     return abits > 0x7F800000u ? 0x7Fu : code;                                 // NaN -> 0x7F (its sign is dropped below)
 }
 
+// The same for two values at once with the packed FP32 instructions of sm_100 (each lane is the scalar
+// operation, rounding mode included): half the floating-point instructions.
+__device__ __forceinline__ uint64_t add_rz2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+template <int FMT>
+__device__ __forceinline__ uint32_t finish_code(uint32_t abits, uint32_t eqb, float t, float fscaled, uint32_t r) {
+    using F = Small<FMT>;
+    const uint32_t threshold = __float2uint_rz(fscaled);
+    uint32_t code = (eqb << F::M) + __float_as_uint(t) - (0x4B000000u + (F::kMinBiasedExp << F::M)) + (r < threshold ? 1u : 0u);
+    code = abits >= F::kMaxBits ? F::kMaxCode : code;
+    if (FMT == kE2M1) return code;
+    if (FMT == kE5M2) code = abits == 0x7F800000u ? F::kInfCode : code;
+    return abits > 0x7F800000u ? 0x7Fu : code;
+}
+
+template <int FMT>
+__device__ __forceinline__ void sr_fp8_magnitude2(uint32_t a0, uint32_t a1, uint32_t r0, uint32_t r1, uint32_t& c0, uint32_t& c1) {
+    using F = Small<FMT>;
+    const uint32_t e0 = a0 >> 23, e1 = a1 >> 23;
+    const uint32_t q0 = e0 < F::kMinBiasedExp ? F::kMinBiasedExp : e0, q1 = e1 < F::kMinBiasedExp ? F::kMinBiasedExp : e1;
+    const float s0 = __uint_as_float(((254u + F::M) << 23) - (q0 << 23)), s1 = __uint_as_float(((254u + F::M) << 23) - (q1 << 23));
+    const uint64_t y = mul2(pack2(__uint_as_float(a0), __uint_as_float(a1)), pack2(s0, s1));
+    const uint64_t magic = dup2(8388608.0f);
+    const uint64_t t = add_rz2(y, magic);
+    const uint64_t f = sub2(y, sub2(t, magic));
+    const uint64_t fs = mul2(f, dup2(4294967296.0f));
+    float t0, t1, f0, f1;
+    unpack2(t, t0, t1);
+    unpack2(fs, f0, f1);
+    c0 = finish_code<FMT>(a0, q0, t0, f0, r0);
+    c1 = finish_code<FMT>(a1, q1, t1, f1, r1);
+}
+
 template <int FMT>
 __device__ __forceinline__ uint32_t sr_fp8_code(uint32_t fbits, uint32_t r) {
     const uint32_t abits = fbits & 0x7FFFFFFFu;
@@ -62,7 +104,13 @@ __device__ __forceinline__ uint32_t sr_fp4_code(uint32_t fbits, uint32_t r) {
 
 // four values -> four 4-bit codes in bits 0..15 (element j in bits 4j..4j+3)
 __device__ __forceinline__ uint32_t cast4_fp4(const uint4 x, const uint4 w) {
-    const uint32_t n0 = sr_fp4_code(x.x, w.x), n1 = sr_fp4_code(x.y, w.y), n2 = sr_fp4_code(x.z, w.z), n3 = sr_fp4_code(x.w, w.w);
+    uint32_t n0, n1, n2, n3;
+    sr_fp8_magnitude2<kE2M1>(x.x & 0x7FFFFFFFu, x.y & 0x7FFFFFFFu, w.x, w.y, n0, n1);
+    sr_fp8_magnitude2<kE2M1>(x.z & 0x7FFFFFFFu, x.w & 0x7FFFFFFFu, w.z, w.w, n2, n3);
+    n0 |= (x.x >> 28) & 0x8u;
+    n1 |= (x.y >> 28) & 0x8u;
+    n2 |= (x.z >> 28) & 0x8u;
+    n3 |= (x.w >> 28) & 0x8u;
     return (n1 * 16u + n0) + (n3 * 16u + n2) * 256u;
 }
 
@@ -77,8 +125,9 @@ __device__ __forceinline__ uint32_t noise32_of_element(uint64_t idx, uint32_t c2
 template <int FMT>
 __device__ __forceinline__ uint32_t cast4(const uint4 x, const uint4 w) {
     const uint32_t ax = x.x & 0x7FFFFFFFu, ay = x.y & 0x7FFFFFFFu, az = x.z & 0x7FFFFFFFu, aw = x.w & 0x7FFFFFFFu;
-    const uint32_t m0 = sr_fp8_magnitude<FMT>(ax, w.x), m1 = sr_fp8_magnitude<FMT>(ay, w.y);
-    const uint32_t m2 = sr_fp8_magnitude<FMT>(az, w.z), m3 = sr_fp8_magnitude<FMT>(aw, w.w);
+    uint32_t m0, m1, m2, m3;
+    sr_fp8_magnitude2<FMT>(ax, ay, w.x, w.y, m0, m1);
+    sr_fp8_magnitude2<FMT>(az, aw, w.z, w.w, m2, m3);
     const uint32_t mags = __byte_perm(__byte_perm(m0, m1, 0x0040), __byte_perm(m2, m3, 0x0040), 0x5410);
     const uint32_t tops = __byte_perm(__byte_perm(x.x, x.y, 0x0073), __byte_perm(x.z, x.w, 0x0073), 0x5410);
     // a NaN code (0x7F) keeps no sign: mask the sign bit where the magnitude byte is 0x7F with all of bits 0..6 set
