@@ -3,6 +3,12 @@
 
 #include "adamw_body.cuh"
 
+// Direct-load shape (FP32 gradients): the next vector's loads are issued before the current vector is
+// computed.  Measured on B200, 832M elements, same GPU: 2.26 -> 2.15 ms.
+#ifndef SR_DIRECT_PREFETCH
+#define SR_DIRECT_PREFETCH 1
+#endif
+
 namespace sradamw {
 
 // MODE 0: element-wise (any alignment, any offset)
@@ -87,8 +93,36 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
         }
         async_copy_wait<0>();
     } else {
+#if SR_DIRECT_PREFETCH
+        // the next vector's loads are issued before the current one is computed (register double buffer)
+        uint4 pv = make_uint4(0, 0, 0, 0), mv = pv, vv = pv, g0 = pv, g1 = pv;
+        auto load = [&](uint64_t vec, uint4& a, uint4& b, uint4& c, uint4& d0, uint4& d1) {
+            if (vec < nvec) {
+                a = ld16(p, vec);
+                b = ld16(m, vec);
+                c = ld16(v, vec);
+                if (G32) {
+                    d0 = ld16(g, 2 * vec);
+                    d1 = ld16(g, 2 * vec + 1);
+                } else {
+                    d0 = ld16(g, vec);
+                }
+            }
+        };
+        load(tid, pv, mv, vv, g0, g1);
+        for (uint64_t vec = tid; vec < nvec; vec += stride) {
+            uint4 pn = pv, mn = mv, vn = vv, gn0 = g0, gn1 = g1;
+            load(vec + stride, pn, mn, vn, gn0, gn1);
+            float ge[8];
+            unpack_grad8<G32>(g0, g1, ge);
+            step_vec8_fast_loaded<G32, FLAGS, SCALE>(p, g, m, v, vec, elem_offset + (vec << 3), pv, mv, vv, ge, c1, tensor_id, seed_hi,
+                                                     gscale, K, S);
+            pv = pn; mv = mn; vv = vn; g0 = gn0; g1 = gn1;
+        }
+#else
         for (uint64_t vec = tid; vec < nvec; vec += stride)
             step_vec8_fast<G32, FLAGS, SCALE>(p, g, m, v, vec, elem_offset + (vec << 3), c1, tensor_id, seed_hi, gscale, K, S);
+#endif
     }
     const uint64_t done = nvec << 3;
     if (tid < n - done)
