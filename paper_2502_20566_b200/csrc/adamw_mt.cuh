@@ -83,7 +83,37 @@ k_sr_adamw_mt(const MtWork* __restrict__ work, uint32_t num_chunks, uint32_t ten
         const uint32_t nvec = cur.nvec(), nvec_next = nxt.nvec();
         const uint32_t c1 = static_cast<uint32_t>(cur.idx0 >> 33);
         const uint32_t c2 = tensor_id_base + cur.tensor();
-        if (cur.tensor_vec >> 31) {
+        if ((cur.tensor_vec >> 31) && MODE >= 2 && !kStage) {
+            // direct loads with a register double buffer: my next vector of this chunk is requested before the
+            // current one is computed
+            uint4 pv = make_uint4(0, 0, 0, 0), mv = pv, vv = pv, g0 = pv, g1 = pv;
+            auto load = [&](uint32_t j, uint4& a, uint4& b, uint4& c, uint4& d0, uint4& d1) {
+                if (j < nvec) {
+                    a = ld16(cur.p, j);
+                    b = ld16(cur.m, j);
+                    c = ld16(cur.v, j);
+                    if (G32) {
+                        d0 = ld16(cur.g, 2 * j);
+                        d1 = ld16(cur.g, 2 * j + 1);
+                    } else {
+                        d0 = ld16(cur.g, j);
+                    }
+                }
+            };
+            load(tid, pv, mv, vv, g0, g1);
+            for (uint32_t j = tid; j < nvec; j += kBlockThreads) {
+                uint4 pn = pv, mn = mv, vn = vv, gn0 = g0, gn1 = g1;
+                load(j + kBlockThreads, pn, mn, vn, gn0, gn1);
+                float ge[8];
+                unpack_grad8<G32>(g0, g1, ge);
+                step_vec8_fast_loaded<G32, FLAGS, MODE == 3>(cur.p, cur.g, cur.m, cur.v, j, cur.idx0 + (static_cast<uint64_t>(j) << 3), pv,
+                                                             mv, vv, ge, c1, c2, seed_hi, gscale, K, S);
+                pv = pn; mv = mn; vv = vn; g0 = gn0; g1 = gn1;
+            }
+            const uint32_t done = nvec << 3;
+            if (tid < cur.len - done)
+                step_scalar<G32, FLAGS>(cur.p, cur.g, cur.m, cur.v, done + tid, cur.idx0 + done + tid, c2, seed_hi, gscale, K, S);
+        } else if (cur.tensor_vec >> 31) {
             for (uint32_t j = tid; j < nvec; j += kBlockThreads) {
                 const uint64_t idx0 = cur.idx0 + (static_cast<uint64_t>(j) << 3);
                 if (MODE == 1) {
