@@ -6,6 +6,7 @@ Submodules:
   build    -- compiles the CUDA sources for sm_100a
   synth    -- seeded synthetic workloads (no optimizer arithmetic)
   dist     -- host-side helpers for several ranks (sharding, rank-ordered norm exchange)
+  optim    -- SRAdamW, a torch.optim.Optimizer front end over the tensor-list step
 """
 
-__all__ = ["binding", "build", "dist", "synth"]
+__all__ = ["binding", "build", "dist", "optim", "synth"]
