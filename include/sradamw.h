@@ -63,7 +63,7 @@ typedef enum { SR_DT_BF16 = 0, SR_DT_F32 = 1 } sr_dtype; /* gradient storage; x,
  * Default (flag clear): the AdamW of the optimizer the paper cites, den = sqrt(v/(1-beta2^t)) + eps.
  * SR_FLAG_EPS_INSIDE: the form the paper's analysis uses (appendix: m / sqrt(eps + v)), with the
  * bias correction kept: den = sqrt(v/(1-beta2^t) + eps), evaluated as sqrt(fma(v, 1/(1-beta2^t), eps)).
- * This variant runs the IEEE square-root/division kernels (measured 0.69x the speed of the default). */
+ * Both readings run the same branch-free kernels at the same speed. */
 #define SR_FLAG_EPS_INSIDE 8u
 
 /* Hyper-parameters of one iteration (Algorithm 1, REQUIRE list).  Host memory, read during the call. */

@@ -169,7 +169,8 @@ __device__ __noinline__ void step_vec8_reference(uint16_t* p, const void* g, uin
 // idx0 must be a multiple of 8.  c0 = low word of idx0 >> 1, c1 = idx0 >> 33 (uniform over a launch
 // segment or a chunk, which lets the compiler hoist the round-1/round-2 products that depend only
 // on c1, c2 and the keys).
-template <bool G32, uint32_t FLAGS, bool SCALE>
+// VAR: bit 0 gradient scale, bit 1 epsilon under the square root (see adamw_element_in_range)
+template <bool G32, uint32_t FLAGS, int VAR>
 __device__ __forceinline__ void step_vec8_fast_loaded(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t vec,
                                                       uint64_t idx0, const uint4 pv, const uint4 mv, const uint4 vv,
                                                       const float (&ge)[8], uint32_t c1, uint32_t c2, uint32_t c3,
@@ -187,11 +188,11 @@ __device__ __forceinline__ void step_vec8_fast_loaded(uint16_t* p, const void* g
         const uint32_t pw = word_of(pv, j), mw = word_of(mv, j), vw = word_of(vv, j);
 #if SR_PACKED_F32X2
         ElementOut r0, r1;
-        adamw_pair_in_range<SCALE>(bf16_lo(pw), bf16_hi(pw), ge[2 * j], ge[2 * j + 1], bf16_lo(mw), bf16_hi(mw), bf16_lo(vw),
+        adamw_pair_in_range<VAR>(bf16_lo(pw), bf16_hi(pw), ge[2 * j], ge[2 * j + 1], bf16_lo(mw), bf16_hi(mw), bf16_lo(vw),
                                    bf16_hi(vw), gscale, S, r0, r1);
 #else
-        const ElementOut r0 = adamw_element_in_range<SCALE>(bf16_lo(pw), ge[2 * j], bf16_lo(mw), bf16_lo(vw), gscale, S);
-        const ElementOut r1 = adamw_element_in_range<SCALE>(bf16_hi(pw), ge[2 * j + 1], bf16_hi(mw), bf16_hi(vw), gscale, S);
+        const ElementOut r0 = adamw_element_in_range<VAR>(bf16_lo(pw), ge[2 * j], bf16_lo(mw), bf16_lo(vw), gscale, S);
+        const ElementOut r1 = adamw_element_in_range<VAR>(bf16_hi(pw), ge[2 * j + 1], bf16_hi(mw), bf16_hi(vw), gscale, S);
 #endif
         track.add(r0, r1);
         po[j] = pack_top_halves(round_sum_word<(FLAGS & 1u) != 0, false>(r0.x, word_of(wx, j)),
@@ -212,14 +213,14 @@ __device__ __forceinline__ void step_vec8_fast_loaded(uint16_t* p, const void* g
 }
 
 // the same, loading the vector straight into registers
-template <bool G32, uint32_t FLAGS, bool SCALE>
+template <bool G32, uint32_t FLAGS, int VAR>
 __device__ __forceinline__ void step_vec8_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t vec,
                                                uint64_t idx0, uint32_t c1, uint32_t c2, uint32_t c3, float gscale,
                                                const PhiloxKeys& K, const StepScalars& S) {
     const uint4 pv = ld16(p, vec), mv = ld16(m, vec), vv = ld16(v, vec);
     float ge[8];
     load_grad8<G32>(g, vec, ge);
-    step_vec8_fast_loaded<G32, FLAGS, SCALE>(p, g, m, v, vec, idx0, pv, mv, vv, ge, c1, c2, c3, gscale, K, S);
+    step_vec8_fast_loaded<G32, FLAGS, VAR>(p, g, m, v, vec, idx0, pv, mv, vv, ge, c1, c2, c3, gscale, K, S);
 }
 
 // ---- one element with 2-byte accesses: ragged tails, unaligned buffers ---------------------
@@ -262,9 +263,10 @@ unsigned grid_for(Kernel kernel, uint64_t work_items, const DeviceInfo& dev, int
 }
 
 // The branch-free path needs den = sqrt(v1) * rsqrt_bc2 + eps to stay inside the range its
-// division was validated for, and implements the default placement of epsilon only.
+// division was validated for.  With epsilon under the root den = sqrt(t) and the per-vector range test
+// on t (<= 2^60) already keeps it there; the bounds on the scalars are kept for both.
 inline bool fast_path_allowed(const StepScalars& S) {
-    return !S.eps_inside && S.rsqrt_bc2 >= 1.0f && S.rsqrt_bc2 <= 1024.0f && S.eps >= 0.0f && S.eps <= 1.0f;
+    return S.rsqrt_bc2 >= 1.0f && S.rsqrt_bc2 <= 1024.0f && S.eps >= 0.0f && S.eps <= 1.0f;
 }
 inline bool needs_scale(const StepScalars& S) { return S.gscale_dev != nullptr || S.gscale != 1.0f; }
 

@@ -15,7 +15,8 @@ namespace sradamw {
 //      1: 16-byte vectors, reference arithmetic, elem_offset not a multiple of 8: every vector straddles two
 //         noise groups (six Philox calls per vector)
 //      4: 16-byte vectors, reference arithmetic, one Philox call per (vector, slot): elem_offset a
-//         multiple of 8 but scalars outside what the branch-free arithmetic covers
+//         multiple of 8 but scalars outside what the branch-free arithmetic covers (beta2 so close to 1 that
+//         1/sqrt(1 - beta2^t) > 1024, eps > 1)
 // Persistent grid: thread t takes vectors t, t + T, t + 2T, ... (T = threads in the grid).
 template <bool G32, uint32_t FLAGS, int MODE>
 __global__ void __launch_bounds__(kBlockThreads, kMinBlocksPerSM)
@@ -39,13 +40,13 @@ k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n
 }
 
 // The hot kernel (modes 2 and 3 of the launcher): 16-byte vectors, branch-free arithmetic, gradient
-// used as is (SCALE = false) or multiplied by gscale.  elem_offset is a multiple of 8 and every
+// used as is or multiplied by gscale (VAR bit 0), epsilon outside or under the square root (VAR bit 1).  elem_offset is a multiple of 8 and every
 // index of the launch has the same (index >> 33) = c1.  Same persistent grid.  STAGED = true: each
 // thread keeps its next vectors in flight -- while vector k is computed out of shared memory, the
 // asynchronous copies of vectors k + T, ... are already under way (kFlatStages slots per thread and
 // array).  SHAPE 0: direct loads into registers, kBlockThreads x kMinBlocksPerSM; 1: staged, same
 // block shape, kShortStages; 2: staged, kFlatStagedThreads x kFlatStagedMinBlocks, kFlatStages.
-template <bool G32, uint32_t FLAGS, bool SCALE, int SHAPE>
+template <bool G32, uint32_t FLAGS, int VAR, int SHAPE>
 __global__ void __launch_bounds__(SHAPE == 2 ? kFlatStagedThreads : kBlockThreads, SHAPE == 2 ? kFlatStagedMinBlocks : kMinBlocksPerSM)
 k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset,
                      uint32_t c1, uint32_t tensor_id, uint32_t seed_hi, const __grid_constant__ PhiloxKeys K,
@@ -87,7 +88,7 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
             const uint4 pv = *slot(s, 0), mv = *slot(s, 1), vv = *slot(s, 2);
             float ge[8];
             unpack_grad8<G32>(*slot(s, 3), G32 ? *slot(s, kArrays - 1) : make_uint4(0, 0, 0, 0), ge);
-            step_vec8_fast_loaded<G32, FLAGS, SCALE>(p, g, m, v, vec, elem_offset + (vec << 3), pv, mv, vv, ge, c1,
+            step_vec8_fast_loaded<G32, FLAGS, VAR>(p, g, m, v, vec, elem_offset + (vec << 3), pv, mv, vv, ge, c1,
                                                      tensor_id, seed_hi, gscale, K, S);
             if (++s == kStages) s = 0;
         }
@@ -115,13 +116,13 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
             load(vec + stride, pn, mn, vn, gn0, gn1);
             float ge[8];
             unpack_grad8<G32>(g0, g1, ge);
-            step_vec8_fast_loaded<G32, FLAGS, SCALE>(p, g, m, v, vec, elem_offset + (vec << 3), pv, mv, vv, ge, c1, tensor_id, seed_hi,
+            step_vec8_fast_loaded<G32, FLAGS, VAR>(p, g, m, v, vec, elem_offset + (vec << 3), pv, mv, vv, ge, c1, tensor_id, seed_hi,
                                                      gscale, K, S);
             pv = pn; mv = mn; vv = vn; g0 = gn0; g1 = gn1;
         }
 #else
         for (uint64_t vec = tid; vec < nvec; vec += stride)
-            step_vec8_fast<G32, FLAGS, SCALE>(p, g, m, v, vec, elem_offset + (vec << 3), c1, tensor_id, seed_hi, gscale, K, S);
+            step_vec8_fast<G32, FLAGS, VAR>(p, g, m, v, vec, elem_offset + (vec << 3), c1, tensor_id, seed_hi, gscale, K, S);
 #endif
     }
     const uint64_t done = nvec << 3;
@@ -139,7 +140,7 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
 #define SR_STAGE_F32 0
 #endif
 
-template <bool G32, uint32_t FLAGS, int MODE>
+template <bool G32, uint32_t FLAGS, int MODE, bool EPS_IN = false>
 cudaError_t launch_flat_mode(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset,
                              uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K, const StepScalars& S,
                              const DeviceInfo& dev, cudaStream_t stream) {
@@ -148,11 +149,11 @@ cudaError_t launch_flat_mode(uint16_t* p, const void* g, uint16_t* m, uint16_t* 
         constexpr bool kStaged = G32 ? (SR_STAGE_F32 != 0) : (SR_STAGE_BF16 != 0);
         const uint32_t c1 = static_cast<uint32_t>(elem_offset >> 33);
         if (kStaged && n >= kLongLaunchElems) {
-            auto k = k_sr_adamw_flat_fast<G32, FLAGS, MODE == 3, kStaged ? 2 : 0>;
+            auto k = k_sr_adamw_flat_fast<G32, FLAGS, (MODE == 3 ? 1 : 0) | (EPS_IN ? 2 : 0), kStaged ? 2 : 0>;
             constexpr int kThreads = kStaged ? kFlatStagedThreads : kBlockThreads;
             k<<<grid_for(k, items, dev, kThreads), kThreads, 0, stream>>>(p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
         } else {
-            auto k = k_sr_adamw_flat_fast<G32, FLAGS, MODE == 3, kStaged ? 1 : 0>;
+            auto k = k_sr_adamw_flat_fast<G32, FLAGS, (MODE == 3 ? 1 : 0) | (EPS_IN ? 2 : 0), kStaged ? 1 : 0>;
             k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
         }
     } else {
@@ -186,6 +187,10 @@ cudaError_t launch_flat_flags(uint16_t* p, const void* g, uint16_t* m, uint16_t*
             e = launch_flat_mode<G32, FLAGS, 1>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream);
         else if (!fast_path_allowed(S))
             e = launch_flat_mode<G32, FLAGS, 4>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream);
+        else if (S.eps_inside && needs_scale(S))
+            e = launch_flat_mode<G32, FLAGS, 3, true>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream);
+        else if (S.eps_inside)
+            e = launch_flat_mode<G32, FLAGS, 2, true>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream);
         else if (needs_scale(S))
             e = launch_flat_mode<G32, FLAGS, 3>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream);
         else

@@ -47,12 +47,13 @@ __device__ __forceinline__ WorkRegs no_work() {
 // STAGED (modes 2, 3): every thread keeps its next vector in flight through shared memory with
 // asynchronous copies, across chunk boundaries as well: during its last vector of a chunk it
 // already fetches its first vector of the next chunk.
-template <bool G32, uint32_t FLAGS, int MODE, bool STAGED>
+template <bool G32, uint32_t FLAGS, int MODE, bool STAGED, bool EPS_IN>
 __global__ void __launch_bounds__(kBlockThreads, kMinBlocksPerSM)
 k_sr_adamw_mt(const MtWork* __restrict__ work, uint32_t num_chunks, uint32_t tensor_id_base, uint32_t seed_hi,
               const __grid_constant__ PhiloxKeys K, const __grid_constant__ StepScalars S) {
     constexpr int kArrays = G32 ? 5 : 4;
     constexpr bool kStage = STAGED && MODE >= 2;
+    constexpr int kVar = (MODE == 3 ? 1 : 0) | (EPS_IN ? 2 : 0);   // bit 0: gradient scale, bit 1: epsilon under the root
     __shared__ uint4 stage[kStage ? kMtStages * kArrays * kBlockThreads : 1];
     static_assert(kMtStages == 2, "slot bookkeeping below assumes two stages");
     const float gscale = S.gscale_dev ? __ldg(S.gscale_dev) : S.gscale;
@@ -106,7 +107,7 @@ k_sr_adamw_mt(const MtWork* __restrict__ work, uint32_t num_chunks, uint32_t ten
                 load(j + kBlockThreads, pn, mn, vn, gn0, gn1);
                 float ge[8];
                 unpack_grad8<G32>(g0, g1, ge);
-                step_vec8_fast_loaded<G32, FLAGS, MODE == 3>(cur.p, cur.g, cur.m, cur.v, j, cur.idx0 + (static_cast<uint64_t>(j) << 3), pv,
+                step_vec8_fast_loaded<G32, FLAGS, kVar>(cur.p, cur.g, cur.m, cur.v, j, cur.idx0 + (static_cast<uint64_t>(j) << 3), pv,
                                                              mv, vv, ge, c1, c2, seed_hi, gscale, K, S);
                 pv = pn; mv = mn; vv = vn; g0 = gn0; g1 = gn1;
             }
@@ -119,7 +120,7 @@ k_sr_adamw_mt(const MtWork* __restrict__ work, uint32_t num_chunks, uint32_t ten
                 if (MODE == 1) {
                     step_vec8_reference<G32, FLAGS, true>(cur.p, cur.g, cur.m, cur.v, j, idx0, c2, seed_hi, gscale, K, S);
                 } else if (!kStage) {
-                    step_vec8_fast<G32, FLAGS, MODE == 3>(cur.p, cur.g, cur.m, cur.v, j, idx0, c1, c2, seed_hi, gscale, K, S);
+                    step_vec8_fast<G32, FLAGS, kVar>(cur.p, cur.g, cur.m, cur.v, j, idx0, c1, c2, seed_hi, gscale, K, S);
                 } else {
                     // fetch ahead: my next vector of this chunk, else my first vector of the next chunk
                     if (j + kBlockThreads < nvec) issue(cur, j + kBlockThreads, s ^ 1);
@@ -129,7 +130,7 @@ k_sr_adamw_mt(const MtWork* __restrict__ work, uint32_t num_chunks, uint32_t ten
                     const uint4 pv = *slot(s, 0), mv = *slot(s, 1), vv = *slot(s, 2);
                     float ge[8];
                     unpack_grad8<G32>(*slot(s, 3), G32 ? *slot(s, kArrays - 1) : make_uint4(0, 0, 0, 0), ge);
-                    step_vec8_fast_loaded<G32, FLAGS, MODE == 3>(cur.p, cur.g, cur.m, cur.v, j, idx0, pv, mv, vv, ge, c1, c2,
+                    step_vec8_fast_loaded<G32, FLAGS, kVar>(cur.p, cur.g, cur.m, cur.v, j, idx0, pv, mv, vv, ge, c1, c2,
                                                                  seed_hi, gscale, K, S);
                     s ^= 1;
                 }
@@ -163,11 +164,11 @@ k_sr_adamw_mt(const MtWork* __restrict__ work, uint32_t num_chunks, uint32_t ten
 #define SR_STAGE_MT_F32 0
 #endif
 
-template <bool G32, uint32_t FLAGS, int MODE>
+template <bool G32, uint32_t FLAGS, int MODE, bool EPS_IN = false>
 cudaError_t launch_mt_mode(const MtWork* work, uint32_t num_chunks, uint32_t tensor_id_base, uint32_t seed_hi,
                            const PhiloxKeys& K, const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream) {
     constexpr bool kStaged = G32 ? (SR_STAGE_MT_F32 != 0) : (SR_STAGE_MT_BF16 != 0);
-    auto k = k_sr_adamw_mt<G32, FLAGS, MODE, kStaged>;
+    auto k = k_sr_adamw_mt<G32, FLAGS, MODE, kStaged, EPS_IN>;
     const unsigned resident = static_cast<unsigned>(resident_blocks(k, dev));
     const unsigned grid = num_chunks < resident ? num_chunks : resident;
     k<<<grid, kBlockThreads, 0, stream>>>(work, num_chunks, tensor_id_base, seed_hi, K, S);
@@ -179,6 +180,9 @@ cudaError_t launch_mt_flags(const MtWork* work, uint32_t num_chunks, uint32_t te
                             const PhiloxKeys& K, const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream) {
     if (!fast_path_allowed(S))
         return launch_mt_mode<G32, FLAGS, 1>(work, num_chunks, tensor_id_base, seed_hi, K, S, dev, stream);
+    if (S.eps_inside)
+        return needs_scale(S) ? launch_mt_mode<G32, FLAGS, 3, true>(work, num_chunks, tensor_id_base, seed_hi, K, S, dev, stream)
+                              : launch_mt_mode<G32, FLAGS, 2, true>(work, num_chunks, tensor_id_base, seed_hi, K, S, dev, stream);
     if (needs_scale(S))
         return launch_mt_mode<G32, FLAGS, 3>(work, num_chunks, tensor_id_base, seed_hi, K, S, dev, stream);
     return launch_mt_mode<G32, FLAGS, 2>(work, num_chunks, tensor_id_base, seed_hi, K, S, dev, stream);

@@ -44,7 +44,7 @@ __device__ __forceinline__ void master_scalar(float* p, uint16_t* p16, const voi
 // operand range with the reference arithmetic as fallback for the vector, as in the SR kernels.
 // WIDE: x, m, v (and FP32 g) are 32-byte aligned and move with one 32-byte access per thread and
 // array (measured on B200: 84 % -> 94 % of the copy peak on 832M elements).
-template <bool G32, bool FAST, bool SCALE, bool WIDE>
+template <bool G32, bool FAST, int VAR, bool WIDE>
 __global__ void __launch_bounds__(kBlockThreads, 4)
 k_master_adamw(float* p, uint16_t* p16, const void* g, float* m, float* v, uint64_t n, bool vec_ok,
                const __grid_constant__ StepScalars S) {
@@ -89,8 +89,8 @@ k_master_adamw(float* p, uint16_t* p16, const void* g, float* m, float* v, uint6
             track.init();
 #pragma unroll
             for (int e = 0; e < 8; e += 2) {
-                r[e] = adamw_element_in_range<SCALE>(x[e], ge[e], mm[e], vv[e], gscale, S);
-                r[e + 1] = adamw_element_in_range<SCALE>(x[e + 1], ge[e + 1], mm[e + 1], vv[e + 1], gscale, S);
+                r[e] = adamw_element_in_range<VAR>(x[e], ge[e], mm[e], vv[e], gscale, S);
+                r[e + 1] = adamw_element_in_range<VAR>(x[e + 1], ge[e + 1], mm[e + 1], vv[e + 1], gscale, S);
                 track.add(r[e], r[e + 1]);
             }
             redo = track.left_range();
@@ -125,22 +125,22 @@ k_master_adamw(float* p, uint16_t* p16, const void* g, float* m, float* v, uint6
     if (tid < n - done) master_scalar<G32>(p, p16, g, m, v, done + tid, gscale, S);
 }
 
-template <bool G32, bool FAST, bool SCALE, bool WIDE>
+template <bool G32, bool FAST, int VAR, bool WIDE>
 cudaError_t launch_master_w(float* p, uint16_t* p16, const void* g, float* m, float* v, uint64_t n, bool vec_ok,
                             const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream) {
-    auto k = k_master_adamw<G32, FAST, SCALE, WIDE>;
+    auto k = k_master_adamw<G32, FAST, VAR, WIDE>;
     const uint64_t items = vec_ok ? (n >> 3) + 8 : n;
     k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, p16, g, m, v, n, vec_ok, S);
     return cudaGetLastError();
 }
 
-template <bool G32, bool FAST, bool SCALE>
+template <bool G32, bool FAST, int VAR>
 cudaError_t launch_master_t(float* p, uint16_t* p16, const void* g, float* m, float* v, uint64_t n, bool vec_ok,
                             const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream) {
     auto aligned32 = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 31u) == 0; };
     const bool wide = vec_ok && aligned32(p) && aligned32(m) && aligned32(v) && (!G32 || aligned32(g));
-    return wide ? launch_master_w<G32, FAST, SCALE, true>(p, p16, g, m, v, n, vec_ok, S, dev, stream)
-                : launch_master_w<G32, FAST, SCALE, false>(p, p16, g, m, v, n, vec_ok, S, dev, stream);
+    return wide ? launch_master_w<G32, FAST, VAR, true>(p, p16, g, m, v, n, vec_ok, S, dev, stream)
+                : launch_master_w<G32, FAST, VAR, false>(p, p16, g, m, v, n, vec_ok, S, dev, stream);
 }
 
 }  // namespace
@@ -149,13 +149,25 @@ cudaError_t launch_master_adamw(float* p, uint16_t* p16, const void* g, bool g_f
                                 const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream) {
     const bool vec_ok = aligned16(p) && aligned16(p16) && aligned16(g) && aligned16(m) && aligned16(v);
     const bool fast = fast_path_allowed(S), scale = needs_scale(S);
-#define SR_M(G, F, SC) launch_master_t<G, F, SC>(p, p16, g, m, v, n, vec_ok, S, dev, stream)
+#define SR_M(G, F, VARIANT) launch_master_t<G, F, VARIANT>(p, p16, g, m, v, n, vec_ok, S, dev, stream)
+    // VARIANT: bit 0 gradient scale, bit 1 epsilon under the square root (fast arithmetic only)
+    const int var = (scale ? 1 : 0) | (S.eps_inside ? 2 : 0);
     if (g_f32) {
-        if (!fast) return SR_M(true, false, true);
-        return scale ? SR_M(true, true, true) : SR_M(true, true, false);
+        if (!fast) return SR_M(true, false, 1);
+        switch (var) {
+            case 0: return SR_M(true, true, 0);
+            case 1: return SR_M(true, true, 1);
+            case 2: return SR_M(true, true, 2);
+            default: return SR_M(true, true, 3);
+        }
     }
-    if (!fast) return SR_M(false, false, true);
-    return scale ? SR_M(false, true, true) : SR_M(false, true, false);
+    if (!fast) return SR_M(false, false, 1);
+    switch (var) {
+        case 0: return SR_M(false, true, 0);
+        case 1: return SR_M(false, true, 1);
+        case 2: return SR_M(false, true, 2);
+        default: return SR_M(false, true, 3);
+    }
 #undef SR_M
 }
 

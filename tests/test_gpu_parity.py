@@ -106,7 +106,7 @@ def test_flat_step_rounding_modes(env, flags, g_dtype):
     assert run_both(env, p, g, m, v, HP, seed=3, step=10, gscale=0.125, flags=flags) == (0, 0, 0)
 
 
-@pytest.mark.parametrize("eps", [1e-8, 1e-4])
+@pytest.mark.parametrize("eps", [0.0, 1e-8, 1e-4])
 @pytest.mark.parametrize("flags", [15, 9, 8])
 @pytest.mark.parametrize("g_dtype,n,offset", [(torch.bfloat16, (1 << 20) + 5, 0), (torch.float32, 50001, 24), (torch.bfloat16, 4099, 3)])
 def test_flat_step_eps_inside(env, eps, flags, g_dtype, n, offset):
