@@ -26,7 +26,8 @@
  *   key     = (seed[31:0], step)
  *   counter = (number[31:0], number[63:32], tensor_id, seed[63:32])
  * Element e = index & 7 uses output word e >> 1, its low 16 bits if e is even, its high 16 bits if
- * e is odd; every bit of every call is used once.  sr_downcast_f32_bf16 uses slot 0.
+ * e is odd; every bit of every call is used once.  sr_downcast_f32_bf16 uses slot 0,
+ * sr_accumulate_bf16 slot 3; the FP8 / FP4 casts draw 32 bits per element (layout stated there).
  * Two ranks, two shards or two runs with equal (seed, step, tensor_id, index) therefore round
  * identically, which is what the shared random state of Algorithm 1 is for.
  */
