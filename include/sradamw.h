@@ -125,7 +125,8 @@ sr_status sr_accumulate_bf16(uint16_t* acc, const void* g, sr_dtype g_dtype, uin
  * elem_offset is the global index of element 0, so a shard of a larger buffer rounds as the whole
  * buffer would.  Fastest when all four buffers are 16-byte aligned and elem_offset is a multiple of
  * 8 (shards cut at multiples of 8 elements); other offsets and alignments give the same bits through
- * slower kernels (an offset that is not a multiple of 8 costs about half the throughput). */
+ * slower kernels (an offset that is not a multiple of 8 doubles the Philox calls and costs about a
+ * quarter of the throughput). */
 sr_status sr_adamw_step(uint16_t* p, const void* g, sr_dtype g_dtype, uint16_t* m, uint16_t* v, uint64_t n,
                         const sr_adamw_hparams* hp, uint64_t seed, uint32_t step, uint32_t tensor_id,
                         uint64_t elem_offset, void* stream);

@@ -166,20 +166,27 @@ __device__ __noinline__ void step_vec8_reference(uint16_t* p, const void* g, uin
 }
 
 // ---- fast vector: branch-free arithmetic, one range test per vector ------------------------
-// idx0 must be a multiple of 8.  c0 = low word of idx0 >> 1, c1 = idx0 >> 33 (uniform over a launch
+// idx0 is a multiple of 8 unless VAR bit 2 says otherwise.  c0 = low word of idx0 >> 1, c1 = idx0 >> 33 (uniform over a launch
 // segment or a chunk, which lets the compiler hoist the round-1/round-2 products that depend only
 // on c1, c2 and the keys).
-// VAR: bit 0 gradient scale, bit 1 epsilon under the square root (see adamw_element_in_range)
+// VAR: bit 0 gradient scale, bit 1 epsilon under the square root (see adamw_element_in_range), bit 2: idx0 is not
+// a multiple of 8
 template <bool G32, uint32_t FLAGS, int VAR>
 __device__ __forceinline__ void step_vec8_fast_loaded(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t vec,
                                                       uint64_t idx0, const uint4 pv, const uint4 mv, const uint4 vv,
                                                       const float (&ge)[8], uint32_t c1, uint32_t c2, uint32_t c3,
                                                       float gscale, const PhiloxKeys& K, const StepScalars& S) {
-    const uint32_t c0 = static_cast<uint32_t>(idx0 >> 1);
     uint4 wx = make_uint4(0, 0, 0, 0), wm = wx, wv = wx;
-    if (FLAGS & 1u) wx = philox4x32_10(c0, c1, c2, c3, K);
-    if (FLAGS & 2u) wm = philox4x32_10(c0 + 1, c1, c2, c3, K);
-    if (FLAGS & 4u) wv = philox4x32_10(c0 + 2, c1, c2, c3, K);
+    if (VAR & 4) {   // idx0 is not a multiple of 8: the vector takes its noise from the two groups it straddles
+        if (FLAGS & 1u) wx = straddling_noise(idx0, 0, c2, c3, K);
+        if (FLAGS & 2u) wm = straddling_noise(idx0, 1, c2, c3, K);
+        if (FLAGS & 4u) wv = straddling_noise(idx0, 2, c2, c3, K);
+    } else {
+        const uint32_t c0 = static_cast<uint32_t>(idx0 >> 1);
+        if (FLAGS & 1u) wx = philox4x32_10(c0, c1, c2, c3, K);
+        if (FLAGS & 2u) wm = philox4x32_10(c0 + 1, c1, c2, c3, K);
+        if (FLAGS & 4u) wv = philox4x32_10(c0 + 2, c1, c2, c3, K);
+    }
     RangeTrack track;
     track.init();
     uint32_t po[4], mo[4], vo[4];
@@ -204,7 +211,7 @@ __device__ __forceinline__ void step_vec8_fast_loaded(uint16_t* p, const void* g
     }
     if (track.left_range()) {
         // nothing has been stored yet: redo this vector from memory with the reference arithmetic
-        step_vec8_reference<G32, FLAGS, true>(p, g, m, v, vec, idx0, c2, c3, gscale, K, S);
+        step_vec8_reference<G32, FLAGS, (VAR & 4) == 0>(p, g, m, v, vec, idx0, c2, c3, gscale, K, S);
         return;
     }
     st16(p, vec, make_uint4(po[0], po[1], po[2], po[3]));

@@ -40,7 +40,8 @@ k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n
 }
 
 // The hot kernel (modes 2 and 3 of the launcher): 16-byte vectors, branch-free arithmetic, gradient
-// used as is or multiplied by gscale (VAR bit 0), epsilon outside or under the square root (VAR bit 1).  elem_offset is a multiple of 8 and every
+// used as is or multiplied by gscale (VAR bit 0), epsilon outside or under the square root (VAR bit 1).
+// VAR bit 2: elem_offset is not a multiple of 8.  Every
 // index of the launch has the same (index >> 33) = c1.  Same persistent grid.  STAGED = true: each
 // thread keeps its next vectors in flight -- while vector k is computed out of shared memory, the
 // asynchronous copies of vectors k + T, ... are already under way (kFlatStages slots per thread and
@@ -140,7 +141,7 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
 #define SR_STAGE_F32 0
 #endif
 
-template <bool G32, uint32_t FLAGS, int MODE, bool EPS_IN = false>
+template <bool G32, uint32_t FLAGS, int MODE, bool EPS_IN = false, bool STRADDLE = false>
 cudaError_t launch_flat_mode(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset,
                              uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K, const StepScalars& S,
                              const DeviceInfo& dev, cudaStream_t stream) {
@@ -149,11 +150,11 @@ cudaError_t launch_flat_mode(uint16_t* p, const void* g, uint16_t* m, uint16_t* 
         constexpr bool kStaged = G32 ? (SR_STAGE_F32 != 0) : (SR_STAGE_BF16 != 0);
         const uint32_t c1 = static_cast<uint32_t>(elem_offset >> 33);
         if (kStaged && n >= kLongLaunchElems) {
-            auto k = k_sr_adamw_flat_fast<G32, FLAGS, (MODE == 3 ? 1 : 0) | (EPS_IN ? 2 : 0), kStaged ? 2 : 0>;
+            auto k = k_sr_adamw_flat_fast<G32, FLAGS, (MODE == 3 ? 1 : 0) | (EPS_IN ? 2 : 0) | (STRADDLE ? 4 : 0), kStaged ? 2 : 0>;
             constexpr int kThreads = kStaged ? kFlatStagedThreads : kBlockThreads;
             k<<<grid_for(k, items, dev, kThreads), kThreads, 0, stream>>>(p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
         } else {
-            auto k = k_sr_adamw_flat_fast<G32, FLAGS, (MODE == 3 ? 1 : 0) | (EPS_IN ? 2 : 0), kStaged ? 1 : 0>;
+            auto k = k_sr_adamw_flat_fast<G32, FLAGS, (MODE == 3 ? 1 : 0) | (EPS_IN ? 2 : 0) | (STRADDLE ? 4 : 0), kStaged ? 1 : 0>;
             k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
         }
     } else {
@@ -183,8 +184,13 @@ cudaError_t launch_flat_flags(uint16_t* p, const void* g, uint16_t* m, uint16_t*
         cudaError_t e;
         if (!vec)
             e = launch_flat_mode<G32, FLAGS, 0>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream);
-        else if ((idx & 7u) != 0)
+        else if ((idx & 7u) != 0 && !fast_path_allowed(S))
             e = launch_flat_mode<G32, FLAGS, 1>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream);
+        else if ((idx & 7u) != 0)   // branch-free arithmetic, every vector straddling two noise groups
+            e = S.eps_inside ? (needs_scale(S) ? launch_flat_mode<G32, FLAGS, 3, true, true>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream)
+                                               : launch_flat_mode<G32, FLAGS, 2, true, true>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream))
+                             : (needs_scale(S) ? launch_flat_mode<G32, FLAGS, 3, false, true>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream)
+                                               : launch_flat_mode<G32, FLAGS, 2, false, true>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream));
         else if (!fast_path_allowed(S))
             e = launch_flat_mode<G32, FLAGS, 4>(ps, gs, ms, vs, len, idx, tensor_id, seed_hi, K, S, dev, stream);
         else if (S.eps_inside && needs_scale(S))
