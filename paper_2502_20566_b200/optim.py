@@ -27,6 +27,9 @@ class SRAdamW(torch.optim.Optimizer):
     seed: the shared random state; give every data-parallel replica the same value.
     max_norm: clip the global gradient norm (over all groups) to this value; the norm, the clipping factor and
         the step all stay on the device (``grad_sqnorm_multi_tensor`` -> ``sr_clip_scale`` -> step).
+    Plans are cached by the data pointers of parameters, gradients and moments; creating one copies a table to
+    the device and waits for it.  Keep gradient buffers in place between steps (``zero_grad(set_to_none=False)``)
+    so that the plans are built once.
     ``step(grad_scale=...)`` multiplies the gradients by a host scalar (with clipping: the factor the norm is
     taken under, e.g. 1 / accumulation steps), ``step(grad_scale_dev=t)`` by a device scalar, without an extra
     pass over them.
