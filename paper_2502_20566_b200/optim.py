@@ -146,3 +146,107 @@ class SRAdamW(torch.optim.Optimizer):
         for cached in self._plans.values():
             cached[1].destroy()
         self._plans = {}
+
+
+class FlatSRAdamW(torch.optim.Optimizer):
+    """The same update on flat buffers: every parameter group is packed into one contiguous BF16 buffer (each tensor
+    starting on a multiple of 8 elements, the gaps zero), with flat buffers of the same layout for the gradients and
+    both moments.  ``p.data`` and ``p.grad`` of every parameter become views into them, so autograd accumulates
+    straight into the flat gradient buffer and one ``sr_adamw_step`` launch per group updates the whole model -- the
+    launch shape the 6.7B-parameter measurement uses.  The groups' gradient buffers are slices of one buffer, so with
+    ``max_norm`` the global norm is one ``grad_sqnorm`` call.
+
+    Differences from ``SRAdamW``: the noise index runs over the flat buffer (tensor_id = group index), so the two
+    classes round differently although both follow Algorithm 1; gradients must stay in place (the class's
+    ``zero_grad`` zeroes the flat buffer and never sets ``p.grad`` to None).
+    """
+
+    def __init__(self, params: Iterable, lr: float = 1e-3, betas=(0.9, 0.999), eps: float = 1e-8,
+                 weight_decay: float = 1e-2, seed: int = 0, sr_flags: int = binding.SR_FLAGS_DEFAULT,
+                 eps_inside: bool = False, max_norm: Optional[float] = None, grad_dtype: torch.dtype = torch.bfloat16):
+        if lr < 0 or not 0 <= betas[0] < 1 or not 0 <= betas[1] < 1 or eps < 0:
+            raise ValueError("invalid hyper-parameter")
+        if sr_flags & ~7:
+            raise ValueError("sr_flags: bits 0..2 only")
+        if grad_dtype != torch.bfloat16:
+            raise TypeError("autograd produces gradients of the parameters' type: BF16")
+        super().__init__(params, dict(lr=lr, betas=tuple(betas), eps=eps, weight_decay=weight_decay))
+        self.seed = int(seed)
+        self.flags = int(sr_flags) | (binding.SR_FLAG_EPS_INSIDE if eps_inside else 0)
+        self.max_norm = max_norm
+        self._steps = 0
+        binding.lib()
+        self._flat = []           # per group: dict(p, g, m, v flat tensors, offsets)
+        layouts = []
+        for group in self.param_groups:
+            ps = group["params"]
+            for p in ps:
+                if not p.is_cuda or p.dtype != torch.bfloat16 or not p.is_contiguous():
+                    raise TypeError("FlatSRAdamW needs contiguous BF16 CUDA parameters")
+            offsets, total = [], 0
+            for p in ps:
+                offsets.append(total)
+                total += -(-p.numel() // 8) * 8          # every tensor starts on a multiple of 8 elements (16 bytes)
+            layouts.append((offsets, total))
+        dev = self.param_groups[0]["params"][0].device
+        # one gradient buffer for all groups (each group a slice): the global norm is one grad_sqnorm call
+        self._g_all = torch.zeros(sum(t for _, t in layouts), dtype=torch.bfloat16, device=dev)
+        start = 0
+        for group, (offsets, total) in zip(self.param_groups, layouts):
+            flat = {k: torch.zeros(total, dtype=torch.bfloat16, device=dev) for k in ("p", "m", "v")}
+            flat["g"] = self._g_all[start:start + total]
+            start += total
+            for p, off in zip(group["params"], offsets):
+                n = p.numel()
+                flat["p"][off:off + n].copy_(p.data.reshape(-1))
+                p.data = flat["p"][off:off + n].view(p.shape)
+                if p.grad is not None:
+                    flat["g"][off:off + n].copy_(p.grad.reshape(-1))
+                p.grad = flat["g"][off:off + n].view(p.shape)
+            flat["offsets"] = offsets
+            self._flat.append(flat)
+        self._S = torch.zeros(1, dtype=torch.float64, device=dev)
+        self._gs = torch.zeros(1, dtype=torch.float32, device=dev)
+        need = binding.grad_sqnorm_workspace_bytes(self._g_all.numel())
+        self._ws = torch.empty(max(1, need // 8), dtype=torch.float64, device=dev)
+
+    def zero_grad(self, set_to_none: bool = False):
+        self._g_all.zero_()
+
+    def flat_buffers(self, group: int = 0):
+        """(parameters, gradients, first moments, second moments) of one group as flat BF16 tensors."""
+        f = self._flat[group]
+        return f["p"], f["g"], f["m"], f["v"]
+
+    @torch.no_grad()
+    def step(self, closure=None, grad_scale: float = 1.0):
+        loss = None
+        if closure is not None:
+            with torch.enable_grad():
+                loss = closure()
+        self._steps += 1
+        gs_dev = None
+        if self.max_norm is not None:
+            binding.grad_sqnorm(self._g_all, self._S, self._ws)
+            binding.sr_clip_scale(self._S, grad_scale, self.max_norm, self._gs)
+            gs_dev, grad_scale = self._gs, 1.0
+        for i, (group, flat) in enumerate(zip(self.param_groups, self._flat)):
+            hp = binding.hparams(lr=group["lr"], beta1=group["betas"][0], beta2=group["betas"][1], eps=group["eps"],
+                                 weight_decay=group["weight_decay"], grad_scale=grad_scale, grad_scale_dev=gs_dev,
+                                 flags=self.flags)
+            binding.sr_adamw_step(flat["p"], flat["g"], flat["m"], flat["v"], hp, self.seed, self._steps, tensor_id=i)
+        return loss
+
+    def state_dict(self):
+        return {"sr": {"seed": self.seed, "steps": self._steps, "flags": self.flags},
+                "flat": [{"m": f["m"].clone(), "v": f["v"].clone()} for f in self._flat],
+                "param_groups": [{k: v for k, v in g.items() if k != "params"} for g in self.param_groups]}
+
+    def load_state_dict(self, state_dict):
+        sr = state_dict["sr"]
+        self.seed, self._steps, self.flags = int(sr["seed"]), int(sr["steps"]), int(sr["flags"])
+        for f, saved in zip(self._flat, state_dict["flat"]):
+            f["m"].copy_(saved["m"])
+            f["v"].copy_(saved["v"])
+        for g, saved in zip(self.param_groups, state_dict["param_groups"]):
+            g.update(saved)

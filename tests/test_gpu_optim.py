@@ -177,3 +177,59 @@ def test_clipped_optimizer_step_is_the_oracle_sequence(env):
             oracle.adamw_step(h["p"], gh[i], h["m"], h["v"], oracle.hparams(**kw), 77, step, i, 0, gscale)
             assert np.array_equal(bits(p).reshape(-1), h["p"])
             assert np.array_equal(bits(opt.state[p]["exp_avg"]).reshape(-1), h["m"])
+
+
+def test_flat_optimizer_is_the_oracle_on_the_flat_buffers_and_trains_through_autograd(env):
+    """FlatSRAdamW: parameters and gradients become views of flat buffers; autograd writes into the flat gradient
+    buffer; each step equals norm -> clip -> oracle step on the flat buffers (two groups, padding between tensors)."""
+    oracle, binding, optim, synth, dev = env
+    torch.manual_seed(0)
+    model = torch.nn.Sequential(torch.nn.Linear(37, 53), torch.nn.Tanh(), torch.nn.Linear(53, 11)).to(dev).bfloat16()
+    decay = [p for p in model.parameters() if p.dim() > 1]
+    no_decay = [p for p in model.parameters() if p.dim() == 1]
+    opt = optim.FlatSRAdamW([dict(params=decay, weight_decay=0.1), dict(params=no_decay, weight_decay=0.0)], lr=1e-3,
+                            betas=(0.9, 0.95), seed=31, max_norm=0.05)
+    for p in model.parameters():
+        assert p.data_ptr() % 16 == 0 and p.grad is not None
+    x = torch.randn(256, 37, device=dev).bfloat16()
+    y = torch.randn(256, 11, device=dev).bfloat16()
+    host = []
+    for gi in range(2):
+        fp, fg, fm, fv = opt.flat_buffers(gi)
+        host.append([bits(fp), None, bits(fm), bits(fv)])
+    losses = []
+    for step in (1, 2, 3):
+        opt.zero_grad()
+        loss = torch.nn.functional.mse_loss(model(x).float(), y.float())
+        loss.backward()
+        losses.append(float(loss.detach()))
+        g_all = np.concatenate([bits(opt.flat_buffers(gi)[1]) for gi in range(2)])
+        assert np.count_nonzero(g_all) > g_all.size // 2                      # autograd really wrote into the flat buffer
+        opt.step(grad_scale=1.0)
+        torch.cuda.synchronize()
+        gscale = oracle.clip_scale(oracle.sqnorm(g_all), 1.0, 0.05)
+        for gi, wd in ((0, 0.1), (1, 0.0)):
+            fp, fg, fm, fv = opt.flat_buffers(gi)
+            h = host[gi]
+            oracle.adamw_step(h[0], bits(fg), h[2], h[3], oracle.hparams(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=wd),
+                              31, step, gi, 0, gscale)
+            assert np.array_equal(bits(fp), h[0]) and np.array_equal(bits(fm), h[2]) and np.array_equal(bits(fv), h[3])
+    assert losses[2] < losses[0]                                              # the model views see the updates
+    # resume: parameters + state_dict saved after step 3; step 4 taken twice from that point gives the same bits
+    saved = opt.state_dict()
+    assert saved["sr"]["steps"] == 3
+    params_saved = [opt.flat_buffers(gi)[0].clone() for gi in range(2)]
+
+    def fourth_step():
+        opt.zero_grad()
+        torch.nn.functional.mse_loss(model(x).float(), y.float()).backward()
+        opt.step()
+        torch.cuda.synchronize()
+        return [bits(opt.flat_buffers(gi)[k]) for gi in range(2) for k in (0, 2, 3)]
+
+    first = fourth_step()
+    for gi in range(2):
+        opt.flat_buffers(gi)[0].copy_(params_saved[gi])
+    opt.load_state_dict(saved)
+    second = fourth_step()
+    assert all(np.array_equal(a, b) for a, b in zip(first, second))
