@@ -7,10 +7,10 @@
 // CPU-baseline leg load it.
 //
 // What is defined here, and the passage each item follows:
-//   oracle_philox4x32_10      Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw, SC'11).  The
-//                             paper only asks for "a random state for the optimizer" that is equal
-//                             on every replica (Algorithm 1, REQUIRE list and the r <- r^(opt)
-//                             step); a counter-based generator gives that by construction.
+//   oracle_philox4x32_10      Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw, SC'11).  All
+//                             Algorithm 1 requires (its REQUIRE list and the r <- r^(opt) step) is
+//                             an optimizer random state that every replica holds identically; a
+//                             counter-based generator gives that by construction.
 //   oracle_sr_bf16_bits       stochastic rounding Q_SR of Eq. 2, realised the way Section 3
 //                             describes it: take the FP32 value, add uniform noise below the bits
 //                             that BF16 keeps, shift the fraction out.
@@ -30,15 +30,18 @@
 //   oracle_clip_scale         global-norm clipping coefficient.  (Neither is in the paper; they
 //                             are the usual companions of the update and are defined below.)
 //
-// Floating point: FP32 round-to-nearest-even for the element function (Section 3: the update
-// "temporarily upcasts to FP32"), no flush-to-zero, no contraction except where fmaf is written.
+// Floating point: FP32 round-to-nearest-even for the element function (Section 3: the update is
+// evaluated in FP32 and only its results are rounded), no flush-to-zero, no contraction except where
+// fmaf is written.
 // Build with -ffp-contract=off and without -ffast-math.
 //
 // Pins (tests/, run without a GPU): Philox known-answer vectors of its authors; Eq. 2's two-neighbour
 // property, exact P(up), exact mean (unbiasedness) and exact variance by enumerating all 65536
 // noise values; the stagnation and random-walk examples of Section 2; every FP32 intermediate of
 // the element function against correctly rounded exact rational arithmetic; the step-1 closed
-// form; a library AdamW as a loose bound; the summation tree against exact integer arithmetic.
+// form; a library AdamW as a loose bound; the summation tree against exact integer arithmetic and,
+// for the ORDER of its additions, against a restatement of the rule on order-sensitive data; the
+// rounding decisions of elements and slots that share a Philox call for pairwise independence.
 // Not pinned by the paper (its Algorithm 1 is ambiguous there; "parity unpinned" for that choice
 // alone): where epsilon sits relative to the square root.  The default is the AdamW convention of
 // the optimizer the paper cites, sqrt(v/(1-beta2^t)) + epsilon; flag bit 3 selects the other reading,

@@ -958,3 +958,32 @@ def test_accumulate_noise_is_disjoint_from_the_step(env):
     assert abs(float(up_cast.float().mean()) - 0.25) < 0.02 and abs(float(up_acc.float().mean()) - 0.25) < 0.02
     both = float((up_cast & up_acc).float().mean())
     assert abs(both - 0.0625) < 0.01                                           # independent: P(both) = 1/16
+
+
+def test_decisions_that_share_a_philox_call_are_independent(env):
+    """The 2x2 tables of the oracle's joint-noise pin, taken from the device's outputs: elements that share
+    a word or a call of one slot (through the cast and through the step), and the three slots of one
+    element (through the step), at P(up) = 1/4 over 2^20 indices."""
+    import joint
+    _, binding, _, dev = env
+    n = 1 << 20
+    src = torch.full((n,), joint.QUARTER_F32_BITS, dtype=torch.int32, device=dev).view(torch.float32)
+    dst = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    binding.sr_downcast_f32_bf16(src, dst, seed=11, step=3, tensor_id=2)
+    torch.cuda.synchronize()
+    up = joint.up_decisions(bits(dst), joint.QUARTER_DOWN)
+    assert abs(up.mean() - 0.25) < 4 * np.sqrt(0.1875 / n)
+    for name, (a, b) in joint.pair_tables(up).items():
+        assert joint.chi2_independent_quarters(a, b) < joint.CHI2_3DOF_LIMIT, name
+
+    st = joint.QUARTER_STEP_STATE_BITS
+    p, g, m, v = (torch.full((n,), st[k], dtype=torch.int16, device=dev).view(torch.bfloat16) for k in ("p", "g", "m", "v"))
+    binding.sr_adamw_step(p, g, m, v, binding.hparams(**joint.QUARTER_STEP_HP), (5 << 32) | 9, 1, 4)
+    torch.cuda.synchronize()
+    ups = {k: joint.up_decisions(bits(t), joint.QUARTER_STEP_DOWN[k]) for k, t in (("p", p), ("m", m), ("v", v))}
+    for k, u in ups.items():
+        assert abs(u.mean() - 0.25) < 4 * np.sqrt(0.1875 / n), k
+        for name, (a, b) in joint.pair_tables(u).items():
+            assert joint.chi2_independent_quarters(a, b) < joint.CHI2_3DOF_LIMIT, (k, name)
+    for a, b in (("p", "m"), ("m", "v"), ("p", "v")):
+        assert joint.chi2_independent_quarters(ups[a], ups[b]) < joint.CHI2_3DOF_LIMIT, (a, b)
