@@ -33,11 +33,12 @@ SEED = 1234
 FIRST_STEP = 1000
 BYTES_PER_ELEMENT = 14          # read x, g, m, v (4 x 2 B) + write x, m, v (3 x 2 B)
 FALLBACK_HBM_GBS = 6650.0       # used only when MEASURED_PEAKS.json is absent
-# DRAM bytes (read + write) per element from the ncu capture of the current kernel and launch shape on the
-# 2^30-element case (profiles/k_sr_adamw_flat_fast__long_launch_shape__2pow30.md: 5.794371 TB/s x 2.584544 ms);
-# the traffic of a streaming kernel grows in proportion to the element count, so the full-size figure is
-# this times n.  Set to None whenever the kernel changes until a new capture exists.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = 5.780220e12 * 2.591168e-3 / (1 << 30)
+NOMINAL_HBM_GBS = 7700.0        # data-sheet bandwidth of the HGX B200 (context beside the measured-peak fraction)
+# DRAM bytes (read + write) of one launch of the headline kernel, from a profiler capture of the SAME kernel
+# build and launch shape on a smaller case: (dram bytes read + written, elements of that case).  The traffic of
+# a streaming kernel grows in proportion to the element count, so the full-size figure is bytes / elements * n.
+# None whenever the kernel has changed since the capture was taken.
+NCU_TRAFFIC_CAPTURE = None
 
 
 def parse_args():
@@ -47,10 +48,17 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--elements", type=int, default=0, help="override the buffer length (profiling on a small case)")
+    ap.add_argument("--elem-offset", type=int, default=0,
+                    help="global index of the buffer's first element (profiling the path for offsets that are not multiples of 8)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-elements", type=int, default=1 << 29)
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary kernels (shard step, tensor list, cast)")
+    ap.add_argument("--mode", choices=["replicas", "sharded"], default="replicas",
+                    help="replicas: every rank steps its own full buffer (the paper's data parallelism); sharded: "
+                         "reduce-scatter -> norm -> clip -> shard step -> all-gather over the ranks (torchrun)")
+    ap.add_argument("--sustained-seconds", type=float, default=3.0,
+                    help="length of the second timed region (back-to-back launches under the power cap); 0 skips it")
     ap.add_argument("--case", choices=EXTRA_CASES, default=None,
                     help="run one secondary call alone (with --elements: on a small case) instead of the headline step")
     return ap.parse_args()
@@ -83,17 +91,17 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
-    def stop(self, t0: _dt.datetime, t1: _dt.datetime) -> dict:
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def stop(self) -> None:
+        """End the poller and read its samples; `window` then cuts them to a timed region."""
+        self.rows = []
         if self.proc is None:
-            return out
+            return
         time.sleep(0.12)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        rows = []
         try:
             with open(self.path) as f:
                 for line in f:
@@ -102,12 +110,16 @@ class ClockSampler:
                         continue
                     try:
                         ts = _dt.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f")
-                        rows.append((ts, float(parts[1]), float(parts[2]), float(parts[3]), parts[4:8]))
+                        self.rows.append((ts, float(parts[1]), float(parts[2]), float(parts[3]), parts[4:8]))
                     except ValueError:
                         continue
             os.unlink(self.path)
         except OSError:
-            return out
+            pass
+
+    def window(self, t0: _dt.datetime, t1: _dt.datetime) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        rows = getattr(self, "rows", [])
         inside = [r for r in rows if t0 <= r[0] <= t1] or rows[-3:]
         if not inside:
             return out
@@ -354,6 +366,46 @@ def _extras_accumulate(torch, binding, synth, dev, peak, timed, out, elements):
                                  "frac": 6 * n / t_a / 1e6 / peak}
 
 
+def time_zero_cases(torch, binding, synth, bufs, hp, stream, reps=10, warmup=3):
+    """Headline launch on the 6.7B buffers with (i) a tenth of the 1024-element rows holding zero gradient and zero
+    moments, (ii) a zero gradient everywhere with the usual state, (iii) everything zero.  Leaves the buffers modified."""
+    p, g, m, v = bufs
+    n = p.numel()
+    rows = n // 1024
+    step = [FIRST_STEP + 10000]
+
+    def timed():
+        def one():
+            step[0] += 1
+            binding.sr_adamw_step(p, g, m, v, hp, SEED, step[0])
+        for _ in range(warmup):
+            one()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(stream)
+        for _ in range(reps):
+            one()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    out = {}
+    for t, role in zip(bufs, (synth.ROLE_P, synth.ROLE_G, synth.ROLE_M, synth.ROLE_V)):
+        synth.fill_state(t, role, SEED)
+    mask = torch.rand(rows, device=p.device, generator=torch.Generator(device=p.device).manual_seed(5)) < 0.10
+    for t in (g, m, v):
+        t[:rows * 1024].view(rows, 1024)[mask] = 0
+    out["tenth_of_rows_zero_g_m_v"] = {"ms": timed()}
+    for t, role in zip((m, v), (synth.ROLE_M, synth.ROLE_V)):
+        synth.fill_state(t, role, SEED)
+    g.zero_()
+    out["zero_gradient"] = {"ms": timed()}
+    for t in bufs:
+        t.zero_()
+    out["all_zero"] = {"ms": timed()}
+    return out
+
+
 def hbm_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -403,7 +455,7 @@ def run_ours(args):
             torch.cuda.synchronize()
 
     for w in range(args.warmup):
-        binding.sr_adamw_step(p, g, m, v, hp, SEED, FIRST_STEP + w)
+        binding.sr_adamw_step(p, g, m, v, hp, SEED, FIRST_STEP + w, 0, args.elem_offset)
     sampler = ClockSampler(torch, local) if rank == 0 and not os.environ.get("SRADAMW_NO_CLOCK_SAMPLER") else None
     if sampler is not None:
         time.sleep(0.3)          # let the poller start
@@ -412,13 +464,36 @@ def run_ours(args):
     t_begin = _dt.datetime.now()
     for k in range(args.steps):
         ev[k][0].record(stream)
-        binding.sr_adamw_step(p, g, m, v, hp, SEED, FIRST_STEP + args.warmup + k)
+        binding.sr_adamw_step(p, g, m, v, hp, SEED, FIRST_STEP + args.warmup + k, 0, args.elem_offset)
         ev[k][1].record(stream)
     barrier()
     t_end = _dt.datetime.now()
     total_ms = ev[0][0].elapsed_time(ev[-1][1])
     launch_ms = [a.elapsed_time(b) for a, b in ev]
-    clocks = sampler.stop(t_begin, t_end) if sampler is not None else None
+
+    # second timed region: back-to-back launches for some seconds, long enough for the board to settle on its
+    # power cap (the first region is over before it does); same call, same buffers, its own clock window
+    sustained = None
+    if args.sustained_seconds > 0 and world == 1 and not args.elements:
+        reps = max(args.steps, int(args.sustained_seconds * 1e3 / (sum(launch_ms) / len(launch_ms))) + 1)
+        sev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        torch.cuda.synchronize()
+        ts0 = _dt.datetime.now()
+        for k in range(reps):
+            sev[k][0].record(stream)
+            binding.sr_adamw_step(p, g, m, v, hp, SEED, FIRST_STEP + args.warmup + args.steps + k)
+            sev[k][1].record(stream)
+        torch.cuda.synchronize()
+        ts1 = _dt.datetime.now()
+        sms = [a.elapsed_time(b) for a, b in sev]
+        sustained = {"launches": reps, "seconds": sev[0][0].elapsed_time(sev[-1][1]) * 1e-3, "launch_ms_avg": sum(sms) / reps,
+                     "launch_ms_last_quarter": sum(sms[-(reps // 4):]) / (reps // 4), "window": (ts0, ts1)}
+    if sampler is not None:
+        sampler.stop()
+    clocks = sampler.window(t_begin, t_end) if sampler is not None else None
+    if sustained is not None:
+        w0, w1 = sustained.pop("window")
+        sustained["clocks"] = sampler.window(w0, w1) if sampler is not None else None
     if dist is not None:
         tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
@@ -453,6 +528,12 @@ def run_ours(args):
                "host_checksum": checksum}
         del host, staging
 
+    # the same launch on buffers with exact zeros (rows of 1024 elements): the cases in which the kernel's
+    # branch-free arithmetic used to hand vectors to its reference path
+    zero_cases = None
+    if world == 1 and not args.no_extras and not args.elements:
+        zero_cases = time_zero_cases(torch, binding, synth, bufs, hp, stream)
+
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -461,6 +542,14 @@ def run_ours(args):
     peak, peak_src = hbm_peak()
     avg_launch_ms = sum(launch_ms) / len(launch_ms)
     achieved = BYTES_PER_ELEMENT * n / (avg_launch_ms * 1e-3) / 1e9
+    gbs = lambda ms: BYTES_PER_ELEMENT * n / (ms * 1e-3) / 1e9
+    if sustained is not None:
+        sustained.update(achieved=gbs(sustained["launch_ms_avg"]), frac=gbs(sustained["launch_ms_avg"]) / peak,
+                         achieved_last_quarter=gbs(sustained["launch_ms_last_quarter"]),
+                         frac_last_quarter=gbs(sustained["launch_ms_last_quarter"]) / peak, unit="GB/s")
+    if zero_cases is not None:
+        for c in zero_cases.values():
+            c.update(gbs=gbs(c["ms"]), frac=gbs(c["ms"]) / peak)
     line = {
         "metric": METRIC,
         "value": world * n * args.steps / (total_ms * 1e-3),
@@ -483,15 +572,19 @@ def run_ours(args):
         },
         "hbm_gbs": achieved,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": (NCU_TRAFFIC_BYTES_PER_ELEMENT * n if NCU_TRAFFIC_BYTES_PER_ELEMENT else None),
-                     "peak_source": peak_src, "kernel": "k_sr_adamw_flat_fast", "launch_ms_avg": avg_launch_ms,
+                     "traffic": (NCU_TRAFFIC_CAPTURE[0] / NCU_TRAFFIC_CAPTURE[1] * n if NCU_TRAFFIC_CAPTURE else None),
+                     "peak_source": peak_src, "frac_nominal": achieved / NOMINAL_HBM_GBS, "nominal_gbs": NOMINAL_HBM_GBS,
+                     "kernel": "k_sr_adamw_flat_fast", "launch_ms_avg": avg_launch_ms,
                      "launch_ms_min": min(launch_ms), "launch_ms_median": statistics.median(launch_ms),
-                     "algorithmic_bytes_per_launch": BYTES_PER_ELEMENT * n},
+                     "algorithmic_bytes_per_launch": BYTES_PER_ELEMENT * n,
+                     "sustained": sustained},
         "gpu_launches": args.steps,
         "clocks": clocks,
     }
     if e2e is not None:
         line["e2e"] = e2e
+    if zero_cases is not None:
+        line["zero_cases"] = zero_cases
     del bufs, p, g, m, v
     torch.cuda.empty_cache()
     if world == 1 and not args.no_extras and not args.elements:

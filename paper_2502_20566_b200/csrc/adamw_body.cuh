@@ -121,6 +121,51 @@ __device__ __forceinline__ uint4 straddling_noise(uint64_t idx0, uint32_t slot, 
                       __funnelshift_r(y3, y4, sh));
 }
 
+// The same 128 bits when the 32 lanes of a warp hold consecutive noise groups (lane l: group A + l):
+// lane l's second group is lane l + 1's first, so the words it needs from group A + 1 come from its
+// neighbour by shuffle and nobody computes a call twice.  Lane 31 has no neighbour; the kernels that
+// use this give lanes 0..30 a vector each and let lane 31 compute the noise of the group after lane
+// 30's only.  R = idx0 & 7 (1..7) is the same for every vector of a launch: the kernels switch on it
+// once per vector, so that word selection is fixed at compile time inside each case.
+template <int R>
+__device__ __forceinline__ uint4 straddle_select(const uint4 a, const uint4 b) {
+    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    constexpr int k = R >> 1;
+    if (R & 1)   // half a word further: (w[i] >> 16) | (w[i + 1] << 16)
+        return make_uint4(__byte_perm(w[k], w[k + 1], 0x5432), __byte_perm(w[k + 1], w[k + 2], 0x5432),
+                          __byte_perm(w[k + 2], w[k + 3], 0x5432), __byte_perm(w[k + 3], w[(k + 4) & 7], 0x5432));
+    return make_uint4(w[k], w[k + 1], w[k + 2], w[k + 3]);
+}
+
+// every lane of the warp must call this (full-mask shuffles)
+template <int R>
+__device__ __forceinline__ uint4 straddle_from_neighbour(const uint4 a) {
+    constexpr int need = (R + 1) >> 1;   // words of the next group that the vector reaches into
+    uint4 b = make_uint4(0, 0, 0, 0);
+    b.x = __shfl_down_sync(0xFFFFFFFFu, a.x, 1);
+    if (need > 1) b.y = __shfl_down_sync(0xFFFFFFFFu, a.y, 1);
+    if (need > 2) b.z = __shfl_down_sync(0xFFFFFFFFu, a.z, 1);
+    if (need > 3) b.w = __shfl_down_sync(0xFFFFFFFFu, a.w, 1);
+    return straddle_select<R>(a, b);
+}
+
+// in: each lane's own group calls; out: the noise words of each lane's vector (lanes 0..30)
+template <uint32_t FLAGS>
+__device__ __forceinline__ void straddle_slots(uint32_t r, uint4& wx, uint4& wm, uint4& wv) {
+#define SR_STRADDLE_CASE(R)                                           \
+    case R:                                                           \
+        if (FLAGS & 1u) wx = straddle_from_neighbour<R>(wx);          \
+        if (FLAGS & 2u) wm = straddle_from_neighbour<R>(wm);          \
+        if (FLAGS & 4u) wv = straddle_from_neighbour<R>(wv);          \
+        break;
+    switch (r) {
+        SR_STRADDLE_CASE(1) SR_STRADDLE_CASE(2) SR_STRADDLE_CASE(3) SR_STRADDLE_CASE(4)
+        SR_STRADDLE_CASE(5) SR_STRADDLE_CASE(6) SR_STRADDLE_CASE(7)
+        default: break;
+    }
+#undef SR_STRADDLE_CASE
+}
+
 // ---- reference vector: IEEE square root / division, NaN rule -------------------------------
 // GROUPED = true needs idx0 (global index of the vector's first element) to be a multiple of 8: the
 // vector is then exactly one noise group and three Philox calls serve it.  GROUPED = false is valid
@@ -166,27 +211,15 @@ __device__ __noinline__ void step_vec8_reference(uint16_t* p, const void* g, uin
 }
 
 // ---- fast vector: branch-free arithmetic, one range test per vector ------------------------
-// idx0 is a multiple of 8 unless VAR bit 2 says otherwise.  c0 = low word of idx0 >> 1, c1 = idx0 >> 33 (uniform over a launch
-// segment or a chunk, which lets the compiler hoist the round-1/round-2 products that depend only
-// on c1, c2 and the keys).
 // VAR: bit 0 gradient scale, bit 1 epsilon under the square root (see adamw_element_in_range), bit 2: idx0 is not
-// a multiple of 8
+// a multiple of 8 (only tells the fallback which noise rule applies)
+// the vector's noise words (wx, wm, wv: one 16-bit half per element and slot) are given
 template <bool G32, uint32_t FLAGS, int VAR>
-__device__ __forceinline__ void step_vec8_fast_loaded(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t vec,
-                                                      uint64_t idx0, const uint4 pv, const uint4 mv, const uint4 vv,
-                                                      const float (&ge)[8], uint32_t c1, uint32_t c2, uint32_t c3,
-                                                      float gscale, const PhiloxKeys& K, const StepScalars& S) {
-    uint4 wx = make_uint4(0, 0, 0, 0), wm = wx, wv = wx;
-    if (VAR & 4) {   // idx0 is not a multiple of 8: the vector takes its noise from the two groups it straddles
-        if (FLAGS & 1u) wx = straddling_noise(idx0, 0, c2, c3, K);
-        if (FLAGS & 2u) wm = straddling_noise(idx0, 1, c2, c3, K);
-        if (FLAGS & 4u) wv = straddling_noise(idx0, 2, c2, c3, K);
-    } else {
-        const uint32_t c0 = static_cast<uint32_t>(idx0 >> 1);
-        if (FLAGS & 1u) wx = philox4x32_10(c0, c1, c2, c3, K);
-        if (FLAGS & 2u) wm = philox4x32_10(c0 + 1, c1, c2, c3, K);
-        if (FLAGS & 4u) wv = philox4x32_10(c0 + 2, c1, c2, c3, K);
-    }
+__device__ __forceinline__ void step_vec8_fast_noise(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t vec,
+                                                     uint64_t idx0, const uint4 pv, const uint4 mv, const uint4 vv,
+                                                     const float (&ge)[8], const uint4 wx, const uint4 wm, const uint4 wv,
+                                                     uint32_t c2, uint32_t c3, float gscale, const PhiloxKeys& K,
+                                                     const StepScalars& S) {
     RangeTrack track;
     track.init();
     uint32_t po[4], mo[4], vo[4];
@@ -210,13 +243,41 @@ __device__ __forceinline__ void step_vec8_fast_loaded(uint16_t* p, const void* g
                                 round_sum_word<(FLAGS & 4u) != 0, true>(r1.v, word_of(wv, j)));
     }
     if (track.left_range()) {
-        // nothing has been stored yet: redo this vector from memory with the reference arithmetic
-        step_vec8_reference<G32, FLAGS, (VAR & 4) == 0>(p, g, m, v, vec, idx0, c2, c3, gscale, K, S);
-        return;
+        if (track.zero_vector(S.zero_t_ok)) {
+            // all m1 are +-0: u = m1 / den is +-0 with the sign of m1, which the rounded m keeps; only x is redone
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t pw = word_of(pv, j);
+                const float x0 = bf16_lo(pw), x1 = bf16_hi(pw);
+                const float q0 = __fmaf_rn(S.step_size, bf16_lo(mo[j]), __fmul_rn(S.lr_wd, x0));
+                const float q1 = __fmaf_rn(S.step_size, bf16_hi(mo[j]), __fmul_rn(S.lr_wd, x1));
+                po[j] = pack_top_halves(round_sum_word_nan_safe<(FLAGS & 1u) != 0, false>(__fsub_rn(x0, q0), word_of(wx, j)),
+                                        round_sum_word_nan_safe<(FLAGS & 1u) != 0, true>(__fsub_rn(x1, q1), word_of(wx, j)));
+            }
+        } else {
+            // nothing has been stored yet: redo this vector from memory with the reference arithmetic
+            step_vec8_reference<G32, FLAGS, (VAR & 4) == 0>(p, g, m, v, vec, idx0, c2, c3, gscale, K, S);
+            return;
+        }
     }
     st16(p, vec, make_uint4(po[0], po[1], po[2], po[3]));
     st16(m, vec, make_uint4(mo[0], mo[1], mo[2], mo[3]));
     st16(v, vec, make_uint4(vo[0], vo[1], vo[2], vo[3]));
+}
+
+// a vector that is exactly one noise group (idx0 a multiple of 8): three Philox calls, then the above
+template <bool G32, uint32_t FLAGS, int VAR>
+__device__ __forceinline__ void step_vec8_fast_loaded(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t vec,
+                                                      uint64_t idx0, const uint4 pv, const uint4 mv, const uint4 vv,
+                                                      const float (&ge)[8], uint32_t c1, uint32_t c2, uint32_t c3,
+                                                      float gscale, const PhiloxKeys& K, const StepScalars& S) {
+    static_assert((VAR & 4) == 0, "vectors that straddle two noise groups get their words from the caller");
+    uint4 wx = make_uint4(0, 0, 0, 0), wm = wx, wv = wx;
+    const uint32_t c0 = static_cast<uint32_t>(idx0 >> 1);
+    if (FLAGS & 1u) wx = philox4x32_10(c0, c1, c2, c3, K);
+    if (FLAGS & 2u) wm = philox4x32_10(c0 + 1, c1, c2, c3, K);
+    if (FLAGS & 4u) wv = philox4x32_10(c0 + 2, c1, c2, c3, K);
+    step_vec8_fast_noise<G32, FLAGS, VAR>(p, g, m, v, vec, idx0, pv, mv, vv, ge, wx, wm, wv, c2, c3, gscale, K, S);
 }
 
 // the same, loading the vector straight into registers

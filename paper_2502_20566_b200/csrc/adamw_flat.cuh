@@ -41,7 +41,7 @@ k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n
 
 // The hot kernel (modes 2 and 3 of the launcher): 16-byte vectors, branch-free arithmetic, gradient
 // used as is or multiplied by gscale (VAR bit 0), epsilon outside or under the square root (VAR bit 1).
-// VAR bit 2: elem_offset is not a multiple of 8.  Every
+// VAR bit 2: elem_offset is not a multiple of 8 (31 vectors per warp, noise exchanged between lanes).  Every
 // index of the launch has the same (index >> 33) = c1.  Same persistent grid.  STAGED = true: each
 // thread keeps its next vectors in flight -- while vector k is computed out of shared memory, the
 // asynchronous copies of vectors k + T, ... are already under way (kFlatStages slots per thread and
@@ -61,7 +61,95 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
     const uint64_t tid = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
     const uint64_t nvec = n >> 3;
-    if (STAGED) {
+    if constexpr ((VAR & 4) != 0) {
+        // elem_offset is not a multiple of 8: every vector straddles two noise groups.  Lanes 0..30 of a warp
+        // take 31 consecutive vectors; all 32 lanes compute the calls of 32 consecutive groups (lane 31 only
+        // that), and each vector's second group arrives from the next lane by shuffle: three calls per vector
+        // as in the aligned case, for 1/32 of the lanes.  The loop is uniform over the warp (the shuffles need
+        // every lane); lanes without a vector skip the memory accesses and the arithmetic.
+        const uint32_t lane = threadIdx.x & 31u;
+        const bool worker = lane != 31u;
+        const uint64_t wstride = (stride >> 5) * 31u;              // vectors per pass of the grid
+        const uint32_t r = static_cast<uint32_t>(elem_offset) & 7u;
+        const uint64_t group0 = elem_offset >> 3;                   // noise group of the first element
+        auto noise = [&](uint64_t vec, uint4& wx, uint4& wm, uint4& wv) {
+            const uint32_t c0 = static_cast<uint32_t>((group0 + vec) << 2);   // call number 4 * group + slot, low word
+            if (FLAGS & 1u) wx = philox4x32_10(c0, c1, tensor_id, seed_hi, K);
+            if (FLAGS & 2u) wm = philox4x32_10(c0 + 1, c1, tensor_id, seed_hi, K);
+            if (FLAGS & 4u) wv = philox4x32_10(c0 + 2, c1, tensor_id, seed_hi, K);
+            straddle_slots<FLAGS>(r, wx, wm, wv);
+        };
+        uint64_t wb = (tid >> 5) * 31u;                             // first vector of this warp in this pass
+        if (STAGED) {
+            uint4* const mine = stage + threadIdx.x;
+            auto slot = [&](int s, int a) -> uint4* { return mine + (s * kArrays + a) * kThreads; };
+            auto issue = [&](uint64_t vec, int s) {
+                if (worker && vec < nvec) {
+                    async_copy16(slot(s, 0), reinterpret_cast<const uint4*>(p) + vec);
+                    async_copy16(slot(s, 1), reinterpret_cast<const uint4*>(m) + vec);
+                    async_copy16(slot(s, 2), reinterpret_cast<const uint4*>(v) + vec);
+                    if (G32) {
+                        async_copy16(slot(s, 3), reinterpret_cast<const uint4*>(g) + 2 * vec);
+                        async_copy16(slot(s, 4), reinterpret_cast<const uint4*>(g) + 2 * vec + 1);
+                    } else {
+                        async_copy16(slot(s, 3), reinterpret_cast<const uint4*>(g) + vec);
+                    }
+                }
+                async_copy_commit();
+            };
+#pragma unroll
+            for (int s = 0; s < kStages - 1; ++s) issue(wb + s * wstride + lane, s);
+            int s = 0;
+            for (; wb < nvec; wb += wstride) {
+                const uint64_t vec = wb + lane;
+                int ahead = s + kStages - 1;
+                if (ahead >= kStages) ahead -= kStages;
+                issue(vec + (kStages - 1) * wstride, ahead);
+                uint4 wx = make_uint4(0, 0, 0, 0), wm = wx, wv = wx;
+                noise(vec, wx, wm, wv);
+                async_copy_wait<kStages - 1>();
+                if (worker && vec < nvec) {
+                    const uint4 pv = *slot(s, 0), mv = *slot(s, 1), vv = *slot(s, 2);
+                    float ge[8];
+                    unpack_grad8<G32>(*slot(s, 3), G32 ? *slot(s, kArrays - 1) : make_uint4(0, 0, 0, 0), ge);
+                    step_vec8_fast_noise<G32, FLAGS, VAR>(p, g, m, v, vec, elem_offset + (vec << 3), pv, mv, vv, ge, wx, wm, wv,
+                                                            tensor_id, seed_hi, gscale, K, S);
+                }
+                if (++s == kStages) s = 0;
+            }
+            async_copy_wait<0>();
+        } else {
+            uint4 pv = make_uint4(0, 0, 0, 0), mv = pv, vv = pv, g0 = pv, g1 = pv;
+            auto load = [&](uint64_t vec, uint4& a, uint4& b, uint4& c, uint4& d0, uint4& d1) {
+                if (worker && vec < nvec) {
+                    a = ld16(p, vec);
+                    b = ld16(m, vec);
+                    c = ld16(v, vec);
+                    if (G32) {
+                        d0 = ld16(g, 2 * vec);
+                        d1 = ld16(g, 2 * vec + 1);
+                    } else {
+                        d0 = ld16(g, vec);
+                    }
+                }
+            };
+            load(wb + lane, pv, mv, vv, g0, g1);
+            for (; wb < nvec; wb += wstride) {
+                const uint64_t vec = wb + lane;
+                uint4 pn = pv, mn = mv, vn = vv, gn0 = g0, gn1 = g1;
+                load(vec + wstride, pn, mn, vn, gn0, gn1);
+                uint4 wx = make_uint4(0, 0, 0, 0), wm = wx, wv = wx;
+                noise(vec, wx, wm, wv);
+                if (worker && vec < nvec) {
+                    float ge[8];
+                    unpack_grad8<G32>(g0, g1, ge);
+                    step_vec8_fast_noise<G32, FLAGS, VAR>(p, g, m, v, vec, elem_offset + (vec << 3), pv, mv, vv, ge, wx, wm, wv,
+                                                            tensor_id, seed_hi, gscale, K, S);
+                }
+                pv = pn; mv = mn; vv = vn; g0 = gn0; g1 = gn1;
+            }
+        }
+    } else if (STAGED) {
         uint4* const mine = stage + threadIdx.x;
         auto slot = [&](int s, int a) -> uint4* { return mine + (s * kArrays + a) * kThreads; };
         auto issue = [&](uint64_t vec, int s) {
@@ -145,7 +233,8 @@ template <bool G32, uint32_t FLAGS, int MODE, bool EPS_IN = false, bool STRADDLE
 cudaError_t launch_flat_mode(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset,
                              uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K, const StepScalars& S,
                              const DeviceInfo& dev, cudaStream_t stream) {
-    const uint64_t items = MODE == 0 ? n : (n >> 3) + 8;   // + 8: enough threads for the ragged tail
+    // + 8: enough threads for the ragged tail; straddling launches give a vector to 31 of every 32 threads
+    const uint64_t items = MODE == 0 ? n : STRADDLE ? ((n >> 3) / 31 + 1) * 32 + 8 : (n >> 3) + 8;
     if (MODE == 2 || MODE == 3) {
         constexpr bool kStaged = G32 ? (SR_STAGE_F32 != 0) : (SR_STAGE_BF16 != 0);
         const uint32_t c1 = static_cast<uint32_t>(elem_offset >> 33);

@@ -29,8 +29,9 @@ struct DeviceSlot {
 };
 DeviceSlot g_devices[kMaxDevices];
 
-// Properties of the current device, queried once per device.  Racing first calls write the same
-// values; the flag is published after them.
+std::mutex g_device_mutex;   // first query of a device: one thread fills the slot, the others wait
+
+// Properties of the current device, queried once per device (a failed query is retried by the next call).
 sr_status current_device(DeviceInfo* out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -38,14 +39,17 @@ sr_status current_device(DeviceInfo* out) {
     if (dev < 0 || dev >= kMaxDevices) return SR_ERR_UNSUPPORTED_DEVICE;
     DeviceSlot& slot = g_devices[dev];
     if (!slot.known.load(std::memory_order_acquire)) {
-        int sm = 0, major = 0;
-        e = cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return cuda_fail(e);
-        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
-        if (e != cudaSuccess) return cuda_fail(e);
-        slot.info.sm_count = sm;
-        slot.info.cc_major = major;
-        slot.known.store(true, std::memory_order_release);
+        std::lock_guard<std::mutex> lock(g_device_mutex);
+        if (!slot.known.load(std::memory_order_relaxed)) {
+            int sm = 0, major = 0;
+            e = cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
+            if (e != cudaSuccess) return cuda_fail(e);
+            e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+            if (e != cudaSuccess) return cuda_fail(e);
+            slot.info.sm_count = sm;
+            slot.info.cc_major = major;
+            slot.known.store(true, std::memory_order_release);
+        }
     }
     if (slot.info.cc_major != 10) return SR_ERR_UNSUPPORTED_DEVICE;
     *out = slot.info;
@@ -110,6 +114,8 @@ sr_status make_scalars(const sr_adamw_hparams* hp, uint32_t step, StepScalars* S
         S->post_mul = S->rsqrt_bc2;
         S->post_add = hp->eps;
     }
+    // a zero argument of the square root leaves den = eps: inside the branch-free division's range from 2^-30 on
+    S->zero_t_ok = (!S->eps_inside && hp->eps >= 9.313225746154785e-10f) ? 1u : 0u;
     return SR_OK;
 }
 
@@ -117,6 +123,11 @@ sr_status make_scalars(const sr_adamw_hparams* hp, uint32_t step, StepScalars* S
 
 namespace sradamw {
 int note_cuda_error(cudaError_t e) { return static_cast<int>(cuda_fail(e)); }
+int current_device_info(DeviceInfo* out, int* device_index) {
+    const sr_status st = current_device(out);
+    if (st == SR_OK && device_index != nullptr && cudaGetDevice(device_index) != cudaSuccess) return SR_ERR_CUDA;
+    return static_cast<int>(st);
+}
 }  // namespace sradamw
 
 struct sr_mt_plan {
@@ -262,15 +273,38 @@ sr_status sr_adamw_step_host(uint16_t* p_host, const void* g_host, sr_dtype g_dt
     HostPipe& pipe = g_pipes[dev_id];
     cudaError_t e;
     if (!pipe.ready) {
-        if ((e = cudaStreamCreateWithFlags(&pipe.side, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaEventCreateWithFlags(&pipe.fork, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaEventCreateWithFlags(&pipe.join, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        // all three objects or none: a partial set is destroyed, so a later call starts from scratch
+        cudaStream_t side = nullptr;
+        cudaEvent_t fork = nullptr, join = nullptr;
+        if ((e = cudaStreamCreateWithFlags(&side, cudaStreamNonBlocking)) == cudaSuccess &&
+            (e = cudaEventCreateWithFlags(&fork, cudaEventDisableTiming)) == cudaSuccess)
+            e = cudaEventCreateWithFlags(&join, cudaEventDisableTiming);
+        if (e != cudaSuccess) {
+            if (join) cudaEventDestroy(join);
+            if (fork) cudaEventDestroy(fork);
+            if (side) cudaStreamDestroy(side);
+            return cuda_fail(e);
+        }
+        pipe.side = side;
+        pipe.fork = fork;
+        pipe.join = join;
         pipe.ready = true;
     }
     cudaStream_t streams[2] = {static_cast<cudaStream_t>(stream), pipe.side};
     // the side stream starts after whatever the caller queued before this call
     if ((e = cudaEventRecord(pipe.fork, streams[0])) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamWaitEvent(pipe.side, pipe.fork, 0)) != cudaSuccess) return cuda_fail(e);
+    // From here on the side stream is forked off the caller's: every return, failures included, joins it
+    // back, so that work queued on the caller's stream afterwards is ordered behind everything enqueued here.
+    auto join_side = [&]() -> cudaError_t {
+        cudaError_t j = cudaEventRecord(pipe.join, pipe.side);
+        if (j == cudaSuccess) j = cudaStreamWaitEvent(streams[0], pipe.join, 0);
+        return j;
+    };
+    auto fail = [&](cudaError_t err) -> sr_status {
+        join_side();
+        return cuda_fail(err);
+    };
 
     const PhiloxKeys K = make_keys(seed, step);
     const uint32_t seed_hi = static_cast<uint32_t>(seed >> 32);
@@ -287,19 +321,18 @@ sr_status sr_adamw_step_host(uint16_t* p_host, const void* g_host, sr_dtype g_dt
         uint16_t* dv = reinterpret_cast<uint16_t*>(base + 2 * region);
         void* dg = base + 3 * region;
         const char* gh = static_cast<const char*>(g_host) + start * gsz;
-        if ((e = cudaMemcpyAsync(dp, p_host + start, len * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpyAsync(dg, gh, len * gsz, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpyAsync(dm, m_host + start, len * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpyAsync(dv, v_host + start, len * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpyAsync(dp, p_host + start, len * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return fail(e);
+        if ((e = cudaMemcpyAsync(dg, gh, len * gsz, cudaMemcpyHostToDevice, s)) != cudaSuccess) return fail(e);
+        if ((e = cudaMemcpyAsync(dm, m_host + start, len * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return fail(e);
+        if ((e = cudaMemcpyAsync(dv, v_host + start, len * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return fail(e);
         e = launch_adamw_flat(dp, dg, g_f32, dm, dv, len, elem_offset + start, tensor_id, seed_hi, hp->flags, K, S, dev, s);
-        if (e != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpyAsync(p_host + start, dp, len * 2, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpyAsync(m_host + start, dm, len * 2, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpyAsync(v_host + start, dv, len * 2, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+        if (e != cudaSuccess) return fail(e);
+        if ((e = cudaMemcpyAsync(p_host + start, dp, len * 2, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return fail(e);
+        if ((e = cudaMemcpyAsync(m_host + start, dm, len * 2, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return fail(e);
+        if ((e = cudaMemcpyAsync(v_host + start, dv, len * 2, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return fail(e);
     }
     // the caller's stream finishes only after the side stream has
-    if ((e = cudaEventRecord(pipe.join, pipe.side)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaStreamWaitEvent(streams[0], pipe.join, 0)) != cudaSuccess) return cuda_fail(e);
+    if ((e = join_side()) != cudaSuccess) return cuda_fail(e);
     return SR_OK;
 }
 

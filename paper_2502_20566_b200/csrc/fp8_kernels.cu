@@ -55,11 +55,6 @@ __device__ __forceinline__ uint64_t add_rz2(uint64_t a, uint64_t b) {
     asm("add.rz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
-__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
-    uint64_t d;
-    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
 
 template <int FMT>
 __device__ __forceinline__ uint32_t finish_code(uint32_t abits, uint32_t eqb, float t, float fscaled, uint32_t r) {

@@ -81,6 +81,9 @@ cudaError_t launch_downcast_fp8(const float* src, uint8_t* dst, uint64_t n, bool
 
 // records e for sr_last_cuda_error() of the calling thread and returns the value of SR_ERR_CUDA
 int note_cuda_error(cudaError_t e);
+// properties of the current device (cached per device, thread-safe) and, optionally, its index;
+// returns an sr_status value
+int current_device_info(DeviceInfo* out, int* device_index);
 
 cudaError_t launch_downcast_fp4(const float* src, uint8_t* dst, uint64_t n, uint64_t elem_offset, uint32_t tensor_id,
                                 uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev, cudaStream_t stream);

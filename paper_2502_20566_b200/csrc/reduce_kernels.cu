@@ -8,6 +8,7 @@
 // loads of one r are 16-byte, fully coalesced.  HBM-bound: 4 (FP32) or 2 (BF16) bytes per element.
 
 #include <atomic>
+#include <mutex>
 
 #include "../../include/sradamw.h"
 #include "launch.h"
@@ -292,12 +293,12 @@ constexpr uint64_t kStaticScratchDoubles = 131072;   // 1 MiB per GPU that loads
 static __device__ __align__(256) double g_sqnorm_static_scratch[kStaticScratchDoubles];
 
 struct StaticScratchSlot {
-    std::atomic<bool> ready{false};   // published after the fields below
-    double* ptr = nullptr;      // device address of g_sqnorm_static_scratch on this device
-    sradamw::DeviceInfo info{};
+    std::atomic<bool> ready{false};   // published after ptr
+    double* ptr = nullptr;            // device address of g_sqnorm_static_scratch on this device
 };
 constexpr int kStaticMaxDevices = 64;
 StaticScratchSlot g_static_slots[kStaticMaxDevices];
+std::mutex g_static_mutex;            // first call on a device: one thread resolves the address, the others wait
 
 }  // namespace
 
@@ -317,27 +318,25 @@ extern "C" sr_status grad_sqnorm_static(const void* g, sr_dtype g_dtype, uint64_
     if (n != 0 && g == nullptr) return SR_ERR_INVALID_ARG;
     if (sradamw::sqnorm_scratch_doubles(n) > kStaticScratchDoubles) return SR_ERR_WORKSPACE;   // n too large
     int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return static_cast<sr_status>(sradamw::note_cuda_error(e));
+    sradamw::DeviceInfo info;
+    const int st = sradamw::current_device_info(&info, &dev);
+    if (st != SR_OK) return static_cast<sr_status>(st);
     if (dev < 0 || dev >= kStaticMaxDevices) return SR_ERR_UNSUPPORTED_DEVICE;
     StaticScratchSlot& slot = g_static_slots[dev];
+    cudaError_t e;
     if (!slot.ready.load(std::memory_order_acquire)) {
         // once per device, with that device current: the array's name is only a host-side handle,
         // the kernels need its address on this device
-        int sm = 0, major = 0;
-        if ((e = cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess ||
-            (e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess)
-            return static_cast<sr_status>(sradamw::note_cuda_error(e));
-        if (major != 10) return SR_ERR_UNSUPPORTED_DEVICE;
-        void* addr = nullptr;
-        if ((e = cudaGetSymbolAddress(&addr, g_sqnorm_static_scratch)) != cudaSuccess)
-            return static_cast<sr_status>(sradamw::note_cuda_error(e));
-        if (addr == nullptr) return static_cast<sr_status>(sradamw::note_cuda_error(cudaErrorInvalidSymbol));
-        slot.ptr = static_cast<double*>(addr);
-        slot.info.sm_count = sm;
-        slot.info.cc_major = major;
-        slot.ready.store(true, std::memory_order_release);
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!slot.ready.load(std::memory_order_relaxed)) {
+            void* addr = nullptr;
+            if ((e = cudaGetSymbolAddress(&addr, g_sqnorm_static_scratch)) != cudaSuccess)
+                return static_cast<sr_status>(sradamw::note_cuda_error(e));
+            if (addr == nullptr) return static_cast<sr_status>(sradamw::note_cuda_error(cudaErrorInvalidSymbol));
+            slot.ptr = static_cast<double*>(addr);
+            slot.ready.store(true, std::memory_order_release);
+        }
     }
-    e = sradamw::launch_sqnorm(g, g_dtype == SR_DT_F32, n, out_dev, slot.ptr, slot.info, static_cast<cudaStream_t>(stream));
+    e = sradamw::launch_sqnorm(g, g_dtype == SR_DT_F32, n, out_dev, slot.ptr, info, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? SR_OK : static_cast<sr_status>(sradamw::note_cuda_error(e));
 }

@@ -58,18 +58,34 @@ def max_over_ranks(value: float, device, group=None) -> float:
     return float(t.item())
 
 
+def wire_bytes(n: int, world_size: int, grad_dtype: torch.dtype) -> dict:
+    """Bytes one rank sends per iteration of ``sharded_clipped_step`` on a buffer of n elements: the
+    reduce-scatter of the gradient in ``grad_dtype`` and the all-gather of the BF16 parameters each move
+    (world - 1) / world of the buffer per rank (ring or switch alike: every rank must ship every slice it does
+    not own once), the norm exchange one double to every peer.  The BF16 + stochastic-rounding recipe
+    communicates gradients in BF16 (Section 3), mixed precision in FP32: half the reduce-scatter bytes."""
+    gsz = torch.empty(0, dtype=grad_dtype).element_size()
+    share = (world_size - 1) / world_size if world_size > 0 else 0.0
+    return {"reduce_scatter": int(n * gsz * share), "all_gather": int(n * 2 * share),
+            "norm_exchange": 8 * max(0, world_size - 1), "grad_bytes_per_element": gsz}
+
+
 def sharded_clipped_step(shard_p, shard_m, shard_v, full_grad, hp_kwargs: dict, seed: int, step: int, *, max_norm: float,
-                         accum_scale: float = 1.0, tensor_id: int = 0, group=None, full_param_out=None, ops=None):
+                         accum_scale: float = 1.0, tensor_id: int = 0, group=None, full_param_out=None, ops=None,
+                         phase_hook=None, shard_grad_out=None):
     """One optimizer iteration with the state sharded over the ranks of ``group`` (ZeRO-1 shape):
 
         reduce-scatter(full_grad) -> grad_sqnorm -> rank-ordered global norm -> sr_clip_scale
         -> sr_adamw_step on this rank's slice with elem_offset = slice start -> all-gather(x)
 
     ``shard_p/m/v``: this rank's BF16 slice (length = partition(n)[rank][1]); ``full_grad``: this
-    rank's full-length local gradient (FP32; summed over ranks by the reduce-scatter, the factor
-    1/world belongs in ``accum_scale``); ``full_param_out``: optional full-length BF16 buffer that
-    receives every rank's updated slice.  All slices must have equal length (n divisible by
-    8 * world), which is what the collectives need.  The collectives are torch.distributed calls
+    rank's full-length local gradient (FP32, or BF16 for the recipe's BF16 gradient communication;
+    summed over ranks in that type by the reduce-scatter, the factor 1/world belongs in
+    ``accum_scale``); ``full_param_out``: optional full-length BF16 buffer that receives every rank's
+    updated slice; ``shard_grad_out``: optional buffer for the reduced slice (else allocated per call);
+    ``phase_hook(name)``: called at the start of each phase and at the end ("reduce_scatter", "sqnorm",
+    "norm_exchange", "clip_scale", "step", "all_gather", "end"), e.g. to record timing events.
+    All slices must have equal length (n divisible by 8 * world), which is what the collectives need.  The collectives are torch.distributed calls
     (NCCL over NVLink on GPUs); every arithmetic step runs in the library's kernels.  ``ops`` lets a
     test substitute the four kernel calls; by default they are the CUDA binding's.
     Returns the global squared norm (one float64 tensor, identical on every rank).
@@ -101,14 +117,24 @@ def sharded_clipped_step(shard_p, shard_m, shard_v, full_grad, hp_kwargs: dict, 
                                       tensor_id, offset)
 
     dev = full_grad.device
-    shard_g = torch.empty(per, dtype=full_grad.dtype, device=dev)
+    mark = phase_hook if phase_hook is not None else (lambda name: None)
+    shard_g = shard_grad_out if shard_grad_out is not None else torch.empty(per, dtype=full_grad.dtype, device=dev)
+    if shard_g.numel() != per or shard_g.dtype != full_grad.dtype:
+        raise ValueError("shard_grad_out must hold one slice of the gradient's type")
+    mark("reduce_scatter")
     dist.reduce_scatter_tensor(shard_g, full_grad.contiguous(), op=dist.ReduceOp.SUM, group=group)
+    mark("sqnorm")
     local = torch.zeros(1, dtype=torch.float64, device=dev)
     ops.sqnorm(shard_g, local)
+    mark("norm_exchange")
     total = global_sqnorm(local, group)
+    mark("clip_scale")
     gscale = torch.zeros(1, dtype=torch.float32, device=dev)
     ops.clip_scale(total, accum_scale, max_norm, gscale)
+    mark("step")
     ops.step(shard_p, shard_g, shard_m, shard_v, gscale, rank * per)
+    mark("all_gather")
     if full_param_out is not None:
         dist.all_gather_into_tensor(full_param_out, shard_p.contiguous(), group=group)
+    mark("end")
     return total

@@ -157,8 +157,9 @@ class FlatSRAdamW(torch.optim.Optimizer):
     ``max_norm`` the global norm is one ``grad_sqnorm`` call.
 
     Differences from ``SRAdamW``: the noise index runs over the flat buffer (tensor_id = group index), so the two
-    classes round differently although both follow Algorithm 1; gradients must stay in place (the class's
-    ``zero_grad`` zeroes the flat buffer and never sets ``p.grad`` to None).
+    classes round differently although both follow Algorithm 1; the class's ``zero_grad`` zeroes the flat buffer
+    and keeps ``p.grad`` in place, and ``step`` repairs gradients that were moved or dropped by other code (one
+    copy each; see ``_rebind``).
     """
 
     def __init__(self, params: Iterable, lr: float = 1e-3, betas=(0.9, 0.999), eps: float = 1e-8,
@@ -218,12 +219,36 @@ class FlatSRAdamW(torch.optim.Optimizer):
         f = self._flat[group]
         return f["p"], f["g"], f["m"], f["v"]
 
+    def _rebind(self):
+        """Host-side pointer check before every step (no synchronisation): the kernels read the flat buffers, so
+        a gradient that autograd or user code put somewhere else (``model.zero_grad()`` sets ``p.grad`` to None
+        and the next backward pass allocates a fresh tensor) is copied into its slice and ``p.grad`` is made a
+        view of the slice again; a missing gradient counts as zero.  Parameters that no longer live in the flat
+        buffer cannot be repaired silently and raise."""
+        esize = 2
+        for group, flat in zip(self.param_groups, self._flat):
+            pbase, gbase = flat["p"].data_ptr(), flat["g"].data_ptr()
+            for p, off in zip(group["params"], flat["offsets"]):
+                n = p.numel()
+                if p.data.data_ptr() != pbase + esize * off:
+                    raise RuntimeError("FlatSRAdamW: a parameter's storage was replaced; it must stay a view of the flat buffer")
+                g = p.grad
+                if g is not None and g.data_ptr() == gbase + esize * off and g.dtype == torch.bfloat16:
+                    continue
+                piece = flat["g"][off:off + n]
+                if g is None:
+                    piece.zero_()
+                else:
+                    piece.copy_(g.reshape(-1))
+                p.grad = piece.view(p.shape)
+
     @torch.no_grad()
     def step(self, closure=None, grad_scale: float = 1.0):
         loss = None
         if closure is not None:
             with torch.enable_grad():
                 loss = closure()
+        self._rebind()
         self._steps += 1
         gs_dev = None
         if self.max_norm is not None:

@@ -46,8 +46,9 @@ def _worker(rank, world, port, out_dir):
     dist.destroy_process_group()
 
 
-def _sharded_worker(rank, world, port, out_dir):
+def _sharded_worker(rank, world, port, out_dir, grad_dtype_name="float32"):
     """sharded_clipped_step with the kernel calls replaced by the oracle (CPU tensors, gloo)."""
+    grad_dtype = getattr(torch, grad_dtype_name)
     sys.path.insert(0, ROOT)
     os.environ["MASTER_ADDR"] = "127.0.0.1"
     os.environ["MASTER_PORT"] = str(port)
@@ -57,15 +58,18 @@ def _sharded_worker(rank, world, port, out_dir):
     from paper_2502_20566_b200.dist import sharded_clipped_step
     n = 8 * world * 1500
     p, _, m, v = synth.adamw_state(n, 88, "cpu")
-    g_local = synth.state_chunk(synth.ROLE_G, 500 + rank, 0, n, "cpu", g_dtype=torch.float32, outlier_fraction=0.01)
+    g_local = synth.state_chunk(synth.ROLE_G, 500 + rank, 0, n, "cpu", g_dtype=grad_dtype, outlier_fraction=0.01)
     per = n // world
     sl = slice(rank * per, (rank + 1) * per)
     sp, sm, sv = (t[sl].clone() for t in (p, m, v))
 
+    def as_host(t):      # FP32 values, or BF16 bit patterns
+        return t.numpy().copy() if t.dtype == torch.float32 else synth.bits16(t).copy()
+
     class ops:
         @staticmethod
         def sqnorm(g, out):
-            out[0] = oracle.sqnorm(g.numpy().copy())
+            out[0] = oracle.sqnorm(as_host(g))
 
         @staticmethod
         def clip_scale(total, accum, mx, out):
@@ -74,7 +78,7 @@ def _sharded_worker(rank, world, port, out_dir):
         @staticmethod
         def step(pp, gg, mm, vv, gscale_dev, offset):
             pb, mb, vb = (synth.bits16(t) for t in (pp, mm, vv))       # views: updated in place
-            oracle.adamw_step(pb, gg.numpy().copy(), mb, vb, oracle.hparams(**HP), 1234, 7, 0, offset, float(gscale_dev.item()))
+            oracle.adamw_step(pb, as_host(gg), mb, vb, oracle.hparams(**HP), 1234, 7, 0, offset, float(gscale_dev.item()))
 
     full = torch.empty(n, dtype=torch.bfloat16)
     # gloo has no reduce_scatter_tensor / all_gather_into_tensor on every build: fall back to the list forms
@@ -90,27 +94,49 @@ def _sharded_worker(rank, world, port, out_dir):
             out.copy_(torch.cat(parts))
         dist._orig_rs = dist.reduce_scatter_tensor
         dist.reduce_scatter_tensor, dist.all_gather_into_tensor = rs, ag
+    phases = []
+    shard_g = torch.empty(per, dtype=grad_dtype)
     total = sharded_clipped_step(sp, sm, sv, g_local, HP, 1234, 7, max_norm=1.0, accum_scale=1.0 / world,
-                                 full_param_out=full, ops=ops)
+                                 full_param_out=full, ops=ops, phase_hook=phases.append, shard_grad_out=shard_g)
     np.savez(os.path.join(out_dir, f"s{rank}.npz"), full=synth.bits16(full), m=synth.bits16(sm), v=synth.bits16(sv),
-             total=total.numpy(), g=g_local.numpy())
+             total=total.numpy(), g=g_local.float().numpy(), shard_g=shard_g.float().numpy(), phases=np.array(phases))
     dist.barrier()
     dist.destroy_process_group()
 
 
-def test_sharded_clipped_step_orchestration(tmp_path):
+import pytest
+
+
+@pytest.mark.parametrize("grad_dtype_name", ["float32", "bfloat16"])
+def test_sharded_clipped_step_orchestration(tmp_path, grad_dtype_name):
     """reduce-scatter -> norm exchange -> clip -> shard step -> all-gather on two gloo ranks equals the
-    single-process computation on the summed gradient."""
+    single-process computation on the summed gradient, with the gradient communicated in FP32 (mixed
+    precision) and in BF16 (the recipe of Section 3: the sum of the two ranks' BF16 gradients is itself
+    rounded to BF16 by the collective, and everything downstream works on that BF16 slice)."""
     world, port = 2, _free_port()
-    mp.spawn(_sharded_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    mp.spawn(_sharded_worker, args=(world, port, str(tmp_path), grad_dtype_name), nprocs=world, join=True)
     sys.path.insert(0, ROOT)
     import oracle
     from paper_2502_20566_b200 import synth
+    from paper_2502_20566_b200.dist import wire_bytes
     r = [np.load(tmp_path / f"s{k}.npz") for k in range(world)]
     n = 8 * world * 1500
     per = n // world
     p, _, m, v = synth.adamw_state(n, 88, "cpu")
-    g_sum = r[0]["g"] + r[1]["g"]
+    assert list(r[0]["phases"]) == ["reduce_scatter", "sqnorm", "norm_exchange", "clip_scale", "step", "all_gather", "end"]
+    exact = r[0]["g"].astype(np.float64) + r[1]["g"].astype(np.float64)
+    g_sum = np.concatenate([r[k]["shard_g"] for k in range(world)])          # what the collective delivered
+    if grad_dtype_name == "float32":
+        assert np.array_equal(g_sum, r[0]["g"] + r[1]["g"])
+    else:
+        # a BF16 value next to the exact sum (8 significant bits), and exactly representable in BF16
+        assert np.all(np.abs(g_sum - exact) <= np.abs(exact) * 2.0 ** -8 + 1e-30)
+        assert np.array_equal(g_sum.view(np.uint32) & 0xFFFF, np.zeros(n, np.uint32))
+        g_sum = (g_sum.view(np.uint32) >> 16).astype(np.uint16)                # BF16 bit patterns for the oracle
+    b = {t: wire_bytes(n, world, getattr(torch, t)) for t in ("float32", "bfloat16")}
+    assert b["float32"]["reduce_scatter"] == 2 * b["bfloat16"]["reduce_scatter"] == n * 4 // 2
+    assert b["float32"]["all_gather"] == b["bfloat16"]["all_gather"] == n * 2 // 2
+    assert wire_bytes(n, 1, torch.float32)["reduce_scatter"] == 0
     S = sum(oracle.sqnorm(np.ascontiguousarray(g_sum[k * per:(k + 1) * per])) for k in range(world))
     assert float(r[0]["total"][0]) == S and r[0]["total"].tobytes() == r[1]["total"].tobytes()
     gscale = oracle.clip_scale(S, 1.0 / world, 1.0)

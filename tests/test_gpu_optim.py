@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 @pytest.fixture(scope="module")
 def env():
     if not torch.cuda.is_available():
-        pytest.skip("needs a CUDA device")
+        pytest.fail("GPU tests need a CUDA device")
     import oracle
     from paper_2502_20566_b200 import binding, optim, synth
     binding.lib()
@@ -233,3 +233,36 @@ def test_flat_optimizer_is_the_oracle_on_the_flat_buffers_and_trains_through_aut
     opt.load_state_dict(saved)
     second = fourth_step()
     assert all(np.array_equal(a, b) for a, b in zip(first, second))
+
+
+def test_flat_optimizer_survives_model_zero_grad(env):
+    """``model.zero_grad()`` drops every ``p.grad``; the next backward pass allocates gradients outside the flat
+    buffer.  The step must see them all the same: two models trained in lock-step, one cleared through the
+    optimizer and one through the model, stay bit-identical, and the gradients are views of the flat buffer again."""
+    _, _, optim, _, dev = env
+    x = torch.randn(64, 19, device=dev).bfloat16()
+    y = torch.randn(64, 5, device=dev).bfloat16()
+    runs = []
+    for clear_through_model in (False, True):
+        torch.manual_seed(3)
+        model = torch.nn.Sequential(torch.nn.Linear(19, 33), torch.nn.Tanh(), torch.nn.Linear(33, 5)).to(dev).bfloat16()
+        opt = optim.FlatSRAdamW(model.parameters(), lr=1e-3, betas=(0.9, 0.95), seed=7, max_norm=1.0)
+        for step in range(3):
+            if clear_through_model:
+                model.zero_grad()                       # set_to_none=True by default
+                assert all(p.grad is None for p in model.parameters())
+            else:
+                opt.zero_grad()
+            torch.nn.functional.mse_loss(model(x).float(), y.float()).backward()
+            if clear_through_model and step == 2:
+                list(model.parameters())[1].grad = None     # a parameter without a gradient counts as zero
+            elif step == 2:
+                list(model.parameters())[1].grad.zero_()
+            opt.step()
+        torch.cuda.synchronize()
+        fp, fg, _, _ = opt.flat_buffers(0)
+        for p in model.parameters():
+            assert fg.data_ptr() <= p.grad.data_ptr() < fg.data_ptr() + 2 * fg.numel()
+        runs.append([bits(t) for t in opt.flat_buffers(0)])
+    assert all(np.array_equal(a, b) for a, b in zip(*runs))
+    assert np.count_nonzero(runs[0][2]) > 0

@@ -987,3 +987,111 @@ def test_decisions_that_share_a_philox_call_are_independent(env):
             assert joint.chi2_independent_quarters(a, b) < joint.CHI2_3DOF_LIMIT, (k, name)
     for a, b in (("p", "m"), ("m", "v"), ("p", "v")):
         assert joint.chi2_independent_quarters(ups[a], ups[b]) < joint.CHI2_3DOF_LIMIT, (a, b)
+
+
+# ---------------------------------------------------------------------------------------------
+# exact zeros
+# ---------------------------------------------------------------------------------------------
+
+def _plant_zero_patterns(p, g, m, v, row=1024, seed=3):
+    """Rows of `row` elements with the zero patterns that occur in training: gradient and both moments zero
+    (a row no batch has touched), everything zero (padding), only the gradient zero, only one moment zero,
+    and negative zeros in every combination that decides the sign of a zero result."""
+    dev = p.device
+    n = p.numel()
+    rows = n // row
+    gen = torch.Generator(device=dev).manual_seed(seed)
+    kind = torch.randint(0, 12, (rows,), generator=gen, device=dev)
+    view = lambda t: t[:rows * row].view(rows, row)
+    P, G, M, V = view(p), view(g), view(m), view(v)
+    neg0 = lambda t, sel: t.__setitem__(sel, torch.tensor(-0.0, dtype=t.dtype, device=dev))
+    for t in (G, M, V):
+        t[kind == 0] = 0                      # untouched row, x arbitrary
+    for t in (P, G, M, V):
+        t[kind == 1] = 0                      # padding
+    G[kind == 2] = 0                          # gradient zero, state alive
+    M[kind == 3] = 0
+    G[kind == 3] = 0                          # m' = 0, v' > 0
+    V[kind == 4] = 0
+    G[kind == 4] = 0                          # v' = 0, m' != 0
+    for t in (P, G, M):                       # x = -0, g = -0, m = -0, v = 0: the sign of every zero matters
+        neg0(t, kind == 5)
+    V[kind == 5] = 0
+    neg0(M, kind == 6)                        # m = -0, g = +0, x = -0
+    G[kind == 6] = 0
+    neg0(P, kind == 6)
+    neg0(M, kind == 7)                        # m = -0, g = -0, x = +0, v alive
+    neg0(G, kind == 7)
+    P[kind == 7] = 0
+    # zeros scattered inside otherwise ordinary vectors
+    sel = torch.rand(n, generator=gen, device=dev) < 0.02
+    g[sel] = 0
+    m[sel] = 0
+    v[sel] = 0
+    return int((kind <= 7).sum())
+
+
+@pytest.mark.parametrize("kw", [HP, dict(HP, eps=0.0), dict(HP, eps=1e-10), dict(HP, eps=1.0, weight_decay=0.0),
+                                dict(HP, lr=0.0), dict(HP, beta1=0.0, beta2=0.0)])
+@pytest.mark.parametrize("g_dtype,flags,gscale,offset", [(torch.bfloat16, 7, 1.0, 0), (torch.float32, 7, 0.125, 8 * 31),
+                                                        (torch.bfloat16, 15, 1.0, 0), (torch.bfloat16, 1, 1.0, 5)])
+def test_exact_zeros_stay_bit_exact(env, kw, g_dtype, flags, gscale, offset):
+    """Zero rows run the branch-free arithmetic when epsilon allows it (default reading, eps >= 2^-30) and the
+    reference arithmetic otherwise; either way every bit, signs of zeros included, equals the oracle's."""
+    _, _, synth, dev = env
+    n = 300 * 1024 + 5
+    p, g, m, v = synth.adamw_state(n, 21, dev, g_dtype=g_dtype)
+    assert _plant_zero_patterns(p, g, m, v) > 100
+    assert run_both(env, p, g, m, v, kw, seed=12, step=7, tensor_id=1, elem_offset=offset, gscale=gscale, flags=flags) == (0, 0, 0)
+    assert run_both(env, p, g, m, v, kw, seed=12, step=8, tensor_id=1, elem_offset=offset, gscale=gscale, flags=flags) == (0, 0, 0)
+
+
+def test_exact_zeros_in_the_tensor_list_and_the_master_recipe(env):
+    oracle, binding, synth, dev = env
+    sizes = [64 * 1024, 8192 + 24, 1024, 40 * 1024 + 8]
+    P, G, M, V = [], [], [], []
+    for i, n in enumerate(sizes):
+        p, g, m, v = synth.adamw_state(n, 30 + i, dev)
+        _plant_zero_patterns(p, g, m, v, seed=i)
+        P.append(p); G.append(g); M.append(m); V.append(v)
+    want = [[bits(t) for t in L] for L in (P, G, M, V)]
+    plan = binding.sr_mt_plan_create(P, G, M, V)
+    binding.sr_adamw_multi_tensor(plan, binding.hparams(**HP), 99, 3, 10)
+    torch.cuda.synchronize()
+    plan.destroy()
+    for i in range(len(sizes)):
+        oracle.adamw_step(want[0][i], want[1][i], want[2][i], want[3][i], oracle.hparams(**HP), 99, 3, 10 + i)
+        assert [mismatches(bits(t[i]), want[k][i]) for k, t in ((0, P), (2, M), (3, V))] == [0, 0, 0]
+    # FP32 master recipe: results are kept in FP32, so every sign of zero is visible
+    n = 100 * 1024 + 3
+    p, g, m, v = synth.adamw_state(n, 41, dev)
+    _plant_zero_patterns(p, g, m, v)
+    p32, m32, v32 = p.float(), m.float(), v.float()
+    p16 = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    hp, ho = binding.hparams(**HP), oracle.hparams(**HP)
+    po, mo, vo = (t.cpu().numpy().copy() for t in (p32, m32, v32))
+    p16o = oracle.master_adamw_step(po, bits(g), mo, vo, ho, 5)
+    binding.sr_master_adamw_step(p32, p16, g, m32, v32, hp, 5)
+    torch.cuda.synchronize()
+    for got, ref in ((p32, po), (m32, mo), (v32, vo)):
+        assert np.array_equal(got.cpu().numpy().view(np.uint32), ref.view(np.uint32))
+    assert mismatches(bits(p16), p16o) == 0
+
+
+def test_long_launch_with_zero_rows(env):
+    """The long-launch shape (2^29 elements and more) with a tenth of its 1024-element rows holding zero
+    gradient and moments and some all-zero rows: every element compared."""
+    oracle, binding, synth, dev = env
+    n = (1 << 29) + 5 * 1024 + 77
+    p, g, m, v = synth.adamw_state(n, 55, dev)
+    rows = n // 1024
+    gen = torch.Generator(device=dev).manual_seed(8)
+    r = torch.rand(rows, generator=gen, device=dev)
+    for t in (g, m, v):
+        t[:rows * 1024].view(rows, 1024)[r < 0.10] = 0
+    p[:rows * 1024].view(rows, 1024)[r < 0.02] = 0
+    pre = [bits(t) for t in (p, g, m, v)]
+    binding.sr_adamw_step(p, g, m, v, binding.hparams(**HP), 2024, 1000)
+    torch.cuda.synchronize()
+    oracle.adamw_step(*pre, oracle.hparams(**HP), 2024, 1000)
+    assert [mismatches(bits(t), pre[k]) for k, t in ((0, p), (2, m), (3, v))] == [0, 0, 0]
