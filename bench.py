@@ -201,7 +201,8 @@ def run_reference(args):
 # CUDA arm
 # ---------------------------------------------------------------------------------------------
 
-EXTRA_CASES = ("shard_fp32_grads", "fp32_master_recipe", "tensor_list", "cast_bf16", "cast_fp8", "cast_fp4", "accumulate")
+EXTRA_CASES = ("shard_fp32_grads", "fp32_master_recipe", "tensor_list", "tensor_list_6p7b", "offset_not_multiple_of_8",
+               "cast_bf16", "cast_fp8", "cast_fp4", "accumulate")
 
 
 def time_extras(torch, binding, synth, dev, peak, only=None, elements=0, reps=10, warmup=3):
@@ -227,8 +228,12 @@ def time_extras(torch, binding, synth, dev, peak, only=None, elements=0, reps=10
     out = {}
     if want("shard_fp32_grads", "fp32_master_recipe"):
         _extras_shard(torch, binding, synth, dev, peak, timed, out, want, elements)
+    if want("offset_not_multiple_of_8"):
+        _extras_offset(torch, binding, synth, dev, peak, timed, out, elements)
     if want("tensor_list"):
         _extras_list(torch, binding, synth, dev, peak, timed, out, compare_flat=only is None)
+    if want("tensor_list_6p7b"):
+        _extras_list_6p7b(torch, binding, synth, dev, peak, timed, out)
     if want("cast_bf16", "cast_fp8", "cast_fp4"):
         _extras_casts(torch, binding, synth, dev, peak, timed, out, want, elements)
     if want("accumulate"):
@@ -329,6 +334,71 @@ def _extras_list(torch, binding, synth, dev, peak, timed, out, compare_flat):
     fp, fg, fm, fv = synth.adamw_state(ne, SEED, dev)
     t_f = timed(lambda: binding.sr_adamw_step(fp, fg, fm, fv, hp, SEED, FIRST_STEP))
     out["flat_same_length_as_list"] = {"elements": ne, "ms": t_f, "gbs": 14 * ne / t_f / 1e6, "frac": 14 * ne / t_f / 1e6 / peak}
+
+
+def _extras_offset(torch, binding, synth, dev, peak, timed, out, elements):
+    # the 1/8 shard (BF16 gradients) placed at a global offset that is 3 modulo 8: every 16-byte vector then
+    # straddles two noise groups; beside it the cast and the accumulation at the same offset
+    n = elements or synth.gpt_flat_numel() // 8
+    p, g, m, v = synth.adamw_state(n, SEED, dev)
+    hp = binding.hparams(**HP)
+    off = 3 * n + 3
+    step = [FIRST_STEP]
+
+    def one(offset):
+        step[0] += 1
+        binding.sr_adamw_step(p, g, m, v, hp, SEED, step[0], 0, offset)
+    t_al = timed(lambda: one(3 * n))
+    t_off = timed(lambda: one(off))
+    res = {"elements": n, "elem_offset": off,
+           "sr_adamw_step": {"ms": t_off, "gbs": 14 * n / t_off / 1e6, "frac": 14 * n / t_off / 1e6 / peak,
+                             "ms_at_aligned_offset": t_al, "frac_at_aligned_offset": 14 * n / t_al / 1e6 / peak}}
+
+    def acc():
+        step[0] += 1
+        binding.sr_accumulate_bf16(m, g, 0.125, SEED, step[0], 0, off)
+    t_a = timed(acc)
+    res["sr_accumulate_bf16"] = {"ms": t_a, "gbs": 6 * n / t_a / 1e6, "frac": 6 * n / t_a / 1e6 / peak}
+    del p, m, v
+    nc = min(n, 1 << 28)
+    src = synth.downcast_mix(nc, 7, dev)
+    dst = torch.empty(nc, dtype=torch.bfloat16, device=dev)
+    t_c = timed(lambda: binding.sr_downcast_f32_bf16(src, dst, seed=7, elem_offset=off))
+    res["sr_downcast_f32_bf16"] = {"elements": nc, "ms": t_c, "gbs": 6 * nc / t_c / 1e6, "frac": 6 * nc / t_c / 1e6 / peak}
+    out["flat_offset_not_multiple_of_8"] = res
+
+
+def _extras_list_6p7b(torch, binding, synth, dev, peak, timed, out):
+    # the 6.7B model as a tensor list (388 tensors, each its own allocation; same element count as the flat buffer):
+    # one sr_adamw_multi_tensor launch per step, and the list norm
+    specs = synth.gpt2_param_list(layers=32, d=4096, vocab=50257, ctx=2048)
+    P = [synth.init_param(sp, SEED, i, dev) for i, sp in enumerate(specs)]
+    G = [synth.fresh_grad(sp, 4321, 1, i, dev) for i, sp in enumerate(specs)]
+    M, V = [], []
+    for i, sp in enumerate(specs):
+        mm = torch.empty(sp.numel, dtype=torch.bfloat16, device=dev)
+        vv = torch.empty(sp.numel, dtype=torch.bfloat16, device=dev)
+        synth.fill_state(mm, synth.ROLE_M, SEED, stream_id=i)
+        synth.fill_state(vv, synth.ROLE_V, SEED, stream_id=i)
+        M.append(mm)
+        V.append(vv)
+    plan = binding.sr_mt_plan_create(P, G, M, V)
+    hp = binding.hparams(**HP)
+    step = [FIRST_STEP]
+
+    def mt():
+        step[0] += 1
+        binding.sr_adamw_multi_tensor(plan, hp, SEED, step[0])
+    t_mt = timed(mt)
+    ne = plan.total_elements
+    ws = torch.empty(max(1, binding.grad_sqnorm_multi_tensor_workspace_bytes(plan) // 8), dtype=torch.float64, device=dev)
+    S = torch.zeros(1, dtype=torch.float64, device=dev)
+    t_norm = timed(lambda: binding.grad_sqnorm_multi_tensor(plan, S, ws))
+    out["tensor_list_6p7b"] = {"tensors": len(specs), "elements": ne, "ms": t_mt, "params_per_s": ne / t_mt * 1e3,
+                               "gbs": 14 * ne / t_mt / 1e6, "frac": 14 * ne / t_mt / 1e6 / peak,
+                               "grad_sqnorm_multi_tensor": {"ms": t_norm, "gbs": 2 * ne / t_norm / 1e6,
+                                                            "frac": 2 * ne / t_norm / 1e6 / peak}}
+    plan.destroy()
 
 
 def _extras_casts(torch, binding, synth, dev, peak, timed, out, want, elements):
@@ -597,10 +667,130 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+
+# ---------------------------------------------------------------------------------------------
+# sharded arm (ZeRO-1 shape): reduce-scatter -> norm -> clip -> shard step -> all-gather
+# ---------------------------------------------------------------------------------------------
+
+SHARDED_METRIC = "sharded SR-AdamW iteration (reduce-scatter, global-norm clip, shard step, all-gather) params/sec"
+PHASES = ("reduce_scatter", "sqnorm", "norm_exchange", "clip_scale", "step", "all_gather")
+
+
+def run_sharded(args):
+    """One optimizer iteration with the optimizer state sharded over the ranks, timed phase by phase with the
+    gradient communicated in BF16 (the recipe of Section 3) and in FP32 (mixed precision).  The collectives are
+    plain NCCL calls through torch.distributed; every arithmetic step is a call of the library.  With one rank
+    the collectives are copies; the arm exists so that a multi-GPU node measures the real thing."""
+    import torch
+    import torch.distributed as dist
+    from paper_2502_20566_b200 import binding, synth
+    from paper_2502_20566_b200 import dist as srdist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29555")
+    # the communicator's own account of what it uses (rings / trees / NVLS), kept out of stdout
+    nccl_log = os.path.join(tempfile.gettempdir(), f"sradamw_nccl_rank{rank}.log")
+    os.environ.setdefault("NCCL_DEBUG", "INFO")
+    os.environ.setdefault("NCCL_DEBUG_FILE", nccl_log)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    binding.lib()
+    n = args.elements or synth.gpt_flat_numel()
+    n -= n % (8 * world)
+    per = n // world
+    stream = torch.cuda.current_stream()
+    results = {}
+    for gname, gdtype in (("bf16", torch.bfloat16), ("fp32", torch.float32)):
+        full_p = torch.empty(n, dtype=torch.bfloat16, device=dev)
+        synth.fill_state(full_p, synth.ROLE_P, SEED)
+        full_g = torch.empty(n, dtype=gdtype, device=dev)
+        synth.fill_state(full_g, synth.ROLE_G, SEED + 100 * (rank + 1))          # every rank its own local gradient
+        shard_p = full_p[rank * per:(rank + 1) * per].clone()
+        shard_m = torch.empty(per, dtype=torch.bfloat16, device=dev)
+        shard_v = torch.empty(per, dtype=torch.bfloat16, device=dev)
+        synth.fill_state(shard_m, synth.ROLE_M, SEED, stream_id=rank)
+        synth.fill_state(shard_v, synth.ROLE_V, SEED, stream_id=rank)
+        shard_g = torch.empty(per, dtype=gdtype, device=dev)
+        marks = []
+
+        def hook(name):
+            e = torch.cuda.Event(enable_timing=True)
+            e.record(stream)
+            marks.append((name, e))
+
+        def iteration(k):
+            srdist.sharded_clipped_step(shard_p, shard_m, shard_v, full_g, HP, SEED, FIRST_STEP + k, max_norm=1.0,
+                                        accum_scale=1.0 / world, full_param_out=full_p, phase_hook=hook,
+                                        shard_grad_out=shard_g)
+
+        for w in range(args.warmup):
+            iteration(w)
+        torch.cuda.synchronize()
+        dist.barrier()
+        torch.cuda.synchronize()
+        marks.clear()
+        for k in range(args.steps):
+            iteration(args.warmup + k)
+        torch.cuda.synchronize()
+        dist.barrier()
+        torch.cuda.synchronize()
+        per_iter = len(PHASES) + 1
+        assert len(marks) == per_iter * args.steps
+        total_ms = marks[0][1].elapsed_time(marks[-1][1])
+        phase_ms = {ph: 0.0 for ph in PHASES}
+        for k in range(args.steps):
+            row = marks[k * per_iter:(k + 1) * per_iter]
+            for (name, e0), (_, e1) in zip(row[:-1], row[1:]):
+                phase_ms[name] += e0.elapsed_time(e1) / args.steps
+        vals = torch.tensor([total_ms] + [phase_ms[ph] for ph in PHASES], dtype=torch.float64, device=dev)
+        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
+        vals = vals.tolist()
+        total_ms = vals[0]
+        wire = srdist.wire_bytes(n, world, gdtype)
+        results[gname] = {"ms_per_step": total_ms / args.steps, "params_per_s": n * args.steps / (total_ms * 1e-3),
+                          "phase_ms": dict(zip(PHASES, vals[1:])), "wire_bytes_per_rank": wire,
+                          "hbm_bytes_per_shard_element": {"sqnorm": wire["grad_bytes_per_element"],
+                                                          "step": 12 + wire["grad_bytes_per_element"]}}
+        del full_p, full_g, shard_p, shard_m, shard_v, shard_g
+        torch.cuda.empty_cache()
+    if rank == 0:
+        nvls = None
+        try:
+            with open(os.environ["NCCL_DEBUG_FILE"]) as f:
+                text = f.read()
+            nvls = "NVLS" in text
+        except OSError:
+            pass
+        rec = results["bf16"]
+        line = {"metric": SHARDED_METRIC, "mode": "sharded", "value": rec["params_per_s"], "unit": "params/s",
+                "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": rec["ms_per_step"],
+                "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": f"6.7B flat buffer sharded over {world} rank(s): {n} elements, {per} per rank; "
+                                       "gradient reduce-scatter in BF16 (value) and in FP32 (beside it), FP64 norm exchange in "
+                                       "rank order, clip to norm 1, shard step at elem_offset = rank * n / R, BF16 all-gather",
+                           "elements": n, "per_rank": per},
+                "gradient_communication": results,
+                "reduce_scatter_bytes_bf16_over_fp32": (results["bf16"]["wire_bytes_per_rank"]["reduce_scatter"]
+                                                        / results["fp32"]["wire_bytes_per_rank"]["reduce_scatter"]
+                                                        if world > 1 else None),
+                "nccl": {"debug": os.environ.get("NCCL_DEBUG"), "debug_file": os.environ["NCCL_DEBUG_FILE"], "nvls_in_log": nvls},
+                "gpu_launches": args.steps * 4 * 2}
+        print(json.dumps(line), flush=True)
+    dist.destroy_process_group()
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.mode == "sharded":
+        run_sharded(args)
     else:
         run_ours(args)
 

@@ -31,28 +31,40 @@ k_sr_accumulate(uint16_t* acc, const void* g, uint64_t n, float scale, uint64_t 
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
     uint64_t done = 0;
     if (MODE != 0) {
+        // MODE 1 (every vector straddles two noise groups): lanes 0..30 take a vector each, all 32 lanes compute one
+        // group's call and pass its words to the lane before them; MODE 2: one thread, one vector, one call
         const uint64_t nvec = n >> 3;
-        for (uint64_t vec = tid; vec < nvec; vec += stride) {
-            const uint4 av = ld16(acc, vec);
-            float ge[8];
-            load_grad8<G32>(g, vec, ge);
-            const uint64_t idx0 = elem_offset + (vec << 3);
-            uint4 w = make_uint4(0, 0, 0, 0);
-            if (SR && MODE == 2)
-                w = philox4x32_10(static_cast<uint32_t>(idx0 >> 1) | kAccumSlot, static_cast<uint32_t>(idx0 >> 33), tensor_id,
-                                  seed_hi, K);
-            else if (SR)
-                w = straddling_noise(idx0, kAccumSlot, tensor_id, seed_hi, K);
-            uint32_t o[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint32_t aw = word_of(av, j);
-                const float s0 = accumulate(bf16_lo(aw), ge[2 * j], scale);
-                const float s1 = accumulate(bf16_hi(aw), ge[2 * j + 1], scale);
-                o[j] = pack_top_halves(round_sum_word_nan_safe<SR, false>(s0, word_of(w, j)),
-                                       round_sum_word_nan_safe<SR, true>(s1, word_of(w, j)));
+        const uint32_t lane = threadIdx.x & 31u;
+        const uint64_t first = MODE == 1 ? (tid >> 5) * 31u : tid;
+        const uint64_t step = MODE == 1 ? (stride >> 5) * 31u : stride;
+        const uint32_t r = static_cast<uint32_t>(elem_offset) & 7u;
+        for (uint64_t base = first; base < nvec; base += step) {
+            const uint64_t vec = MODE == 1 ? base + lane : base;
+            const bool mine = MODE == 2 || (lane != 31u && vec < nvec);
+            uint4 av = make_uint4(0, 0, 0, 0);
+            float ge[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
+            if (mine) {
+                av = ld16(acc, vec);
+                load_grad8<G32>(g, vec, ge);
             }
-            st16(acc, vec, make_uint4(o[0], o[1], o[2], o[3]));
+            uint4 w = make_uint4(0, 0, 0, 0);
+            if (SR) {
+                const uint64_t number = (((elem_offset >> 3) + vec) << 2) | kAccumSlot;
+                w = philox4x32_10(static_cast<uint32_t>(number), static_cast<uint32_t>(number >> 32), tensor_id, seed_hi, K);
+                if (MODE == 1) w = straddle_slot(r, w);
+            }
+            if (mine) {
+                uint32_t o[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t aw = word_of(av, j);
+                    const float s0 = accumulate(bf16_lo(aw), ge[2 * j], scale);
+                    const float s1 = accumulate(bf16_hi(aw), ge[2 * j + 1], scale);
+                    o[j] = pack_top_halves(round_sum_word_nan_safe<SR, false>(s0, word_of(w, j)),
+                                           round_sum_word_nan_safe<SR, true>(s1, word_of(w, j)));
+                }
+                st16(acc, vec, make_uint4(o[0], o[1], o[2], o[3]));
+            }
         }
         done = nvec << 3;
     }
@@ -68,7 +80,7 @@ cudaError_t launch_accum_mode(uint16_t* acc, const void* g, uint64_t n, float sc
                               uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev,
                               cudaStream_t stream) {
     auto k = k_sr_accumulate<G32, SR, MODE>;
-    const uint64_t items = MODE == 0 ? n : (n >> 3) + 8;
+    const uint64_t items = MODE == 0 ? n : MODE == 1 ? ((n >> 3) / 31 + 1) * 32 + 8 : (n >> 3) + 8;
     k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(acc, g, n, scale, elem_offset, tensor_id, seed_hi, K);
     return cudaGetLastError();
 }

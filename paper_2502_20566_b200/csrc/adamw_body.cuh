@@ -149,6 +149,20 @@ __device__ __forceinline__ uint4 straddle_from_neighbour(const uint4 a) {
     return straddle_select<R>(a, b);
 }
 
+// one slot: in, the lane's own group call; out, the noise words of the lane's vector (lanes 0..30)
+__device__ __forceinline__ uint4 straddle_slot(uint32_t r, const uint4 w) {
+    switch (r) {
+        case 1: return straddle_from_neighbour<1>(w);
+        case 2: return straddle_from_neighbour<2>(w);
+        case 3: return straddle_from_neighbour<3>(w);
+        case 4: return straddle_from_neighbour<4>(w);
+        case 5: return straddle_from_neighbour<5>(w);
+        case 6: return straddle_from_neighbour<6>(w);
+        case 7: return straddle_from_neighbour<7>(w);
+        default: return w;
+    }
+}
+
 // in: each lane's own group calls; out: the noise words of each lane's vector (lanes 0..30)
 template <uint32_t FLAGS>
 __device__ __forceinline__ void straddle_slots(uint32_t r, uint4& wx, uint4& wm, uint4& wv) {

@@ -72,12 +72,15 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
         const uint64_t wstride = (stride >> 5) * 31u;              // vectors per pass of the grid
         const uint32_t r = static_cast<uint32_t>(elem_offset) & 7u;
         const uint64_t group0 = elem_offset >> 3;                   // noise group of the first element
-        auto noise = [&](uint64_t vec, uint4& wx, uint4& wm, uint4& wv) {
-            const uint32_t c0 = static_cast<uint32_t>((group0 + vec) << 2);   // call number 4 * group + slot, low word
+        // call number 4 * group + slot, low word; advances by 4 * wstride per pass (the high word c1 is fixed)
+        uint32_t c0 = static_cast<uint32_t>((group0 + (tid >> 5) * 31u + lane) << 2);
+        const uint32_t c0_step = static_cast<uint32_t>(wstride << 2);
+        auto noise = [&](uint4& wx, uint4& wm, uint4& wv) {
             if (FLAGS & 1u) wx = philox4x32_10(c0, c1, tensor_id, seed_hi, K);
             if (FLAGS & 2u) wm = philox4x32_10(c0 + 1, c1, tensor_id, seed_hi, K);
             if (FLAGS & 4u) wv = philox4x32_10(c0 + 2, c1, tensor_id, seed_hi, K);
             straddle_slots<FLAGS>(r, wx, wm, wv);
+            c0 += c0_step;
         };
         uint64_t wb = (tid >> 5) * 31u;                             // first vector of this warp in this pass
         if (STAGED) {
@@ -106,7 +109,7 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
                 if (ahead >= kStages) ahead -= kStages;
                 issue(vec + (kStages - 1) * wstride, ahead);
                 uint4 wx = make_uint4(0, 0, 0, 0), wm = wx, wv = wx;
-                noise(vec, wx, wm, wv);
+                noise(wx, wm, wv);
                 async_copy_wait<kStages - 1>();
                 if (worker && vec < nvec) {
                     const uint4 pv = *slot(s, 0), mv = *slot(s, 1), vv = *slot(s, 2);
@@ -139,7 +142,7 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
                 uint4 pn = pv, mn = mv, vn = vv, gn0 = g0, gn1 = g1;
                 load(vec + wstride, pn, mn, vn, gn0, gn1);
                 uint4 wx = make_uint4(0, 0, 0, 0), wm = wx, wv = wx;
-                noise(vec, wx, wm, wv);
+                noise(wx, wm, wv);
                 if (worker && vec < nvec) {
                     float ge[8];
                     unpack_grad8<G32>(g0, g1, ge);
@@ -225,6 +228,12 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
 #ifndef SR_STAGE_BF16
 #define SR_STAGE_BF16 1
 #endif
+// Launches whose offset is not a multiple of 8 keep the short shape at every length.  Measured on B200,
+// 6.7B elements, same GPU: 20.7 ms with 128 x 5 blocks, 21.3 ms with 256 x 2 (and 21.7 ms for the version
+// in which every thread computed both straddled groups itself).
+#ifndef SR_STRADDLE_LONG_SHAPE
+#define SR_STRADDLE_LONG_SHAPE 0
+#endif
 #ifndef SR_STAGE_F32
 #define SR_STAGE_F32 0
 #endif
@@ -238,7 +247,7 @@ cudaError_t launch_flat_mode(uint16_t* p, const void* g, uint16_t* m, uint16_t* 
     if (MODE == 2 || MODE == 3) {
         constexpr bool kStaged = G32 ? (SR_STAGE_F32 != 0) : (SR_STAGE_BF16 != 0);
         const uint32_t c1 = static_cast<uint32_t>(elem_offset >> 33);
-        if (kStaged && n >= kLongLaunchElems) {
+        if (kStaged && n >= kLongLaunchElems && (!STRADDLE || SR_STRADDLE_LONG_SHAPE)) {
             auto k = k_sr_adamw_flat_fast<G32, FLAGS, (MODE == 3 ? 1 : 0) | (EPS_IN ? 2 : 0) | (STRADDLE ? 4 : 0), kStaged ? 2 : 0>;
             constexpr int kThreads = kStaged ? kFlatStagedThreads : kBlockThreads;
             k<<<grid_for(k, items, dev, kThreads), kThreads, 0, stream>>>(p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
