@@ -23,48 +23,51 @@ __device__ __forceinline__ float accumulate(float acc, float g, float scale) {
 }
 
 // MODE 0: element-wise; 1: 16-byte vectors straddling two noise groups (offset not a multiple of 8); 2: vectors, grouped
+#ifndef SR_ACCUM_STRADDLE_MIN_BLOCKS
+#define SR_ACCUM_STRADDLE_MIN_BLOCKS 1
+#endif
 template <bool G32, bool SR, int MODE>
-__global__ void __launch_bounds__(kBlockThreads)
+__global__ void __launch_bounds__(kBlockThreads, MODE == 1 ? SR_ACCUM_STRADDLE_MIN_BLOCKS : 1)
 k_sr_accumulate(uint16_t* acc, const void* g, uint64_t n, float scale, uint64_t elem_offset, uint32_t tensor_id,
                 uint32_t seed_hi, const __grid_constant__ PhiloxKeys K) {
     const uint64_t tid = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
     uint64_t done = 0;
     if (MODE != 0) {
-        // MODE 1 (every vector straddles two noise groups): lanes 0..30 take a vector each, all 32 lanes compute one
-        // group's call and pass its words to the lane before them; MODE 2: one thread, one vector, one call
-        const uint64_t nvec = n >> 3;
+        // MODE 1 (every vector straddles two noise groups): every lane computes the call of the group its vector ends
+        // in and takes the other group's words from the lane below (RowChain), whole rows of 32 vectors only (the
+        // rest goes element by element); MODE 2: one thread, one vector, one call
+        using Chain = RowChain<1u << kAccumSlot, false>;
+        __shared__ uint4 heads[MODE == 1 ? (kBlockThreads / 32) * Chain::kTableEntries : 1];
+        const uint64_t nvec = MODE == 1 ? (n >> 3) & ~static_cast<uint64_t>(31) : n >> 3;
         const uint32_t lane = threadIdx.x & 31u;
-        const uint64_t first = MODE == 1 ? (tid >> 5) * 31u : tid;
-        const uint64_t step = MODE == 1 ? (stride >> 5) * 31u : stride;
-        const uint32_t r = static_cast<uint32_t>(elem_offset) & 7u;
-        for (uint64_t base = first; base < nvec; base += step) {
-            const uint64_t vec = MODE == 1 ? base + lane : base;
-            const bool mine = MODE == 2 || (lane != 31u && vec < nvec);
-            uint4 av = make_uint4(0, 0, 0, 0);
-            float ge[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
-            if (mine) {
-                av = ld16(acc, vec);
-                load_grad8<G32>(g, vec, ge);
-            }
+        const Chain chain{heads + (MODE == 1 ? (threadIdx.x >> 5) * Chain::kTableEntries : 0), elem_offset >> 3, stride,
+                          static_cast<uint32_t>(elem_offset) & 7u, lane, 0u, tensor_id, seed_hi};
+        uint32_t k = 0;
+        for (uint64_t vec = tid; vec < nvec; vec += stride, ++k) {
+            const uint4 av = ld16(acc, vec);
+            float ge[8];
+            load_grad8<G32>(g, vec, ge);
             uint4 w = make_uint4(0, 0, 0, 0);
-            if (SR) {
+            if (SR && MODE == 1) {
+                if ((k & 31u) == 0u) chain.refill(vec - lane, K);
+                uint4 w4[4];
+                chain.words(vec, k, K, w4);
+                w = w4[kAccumSlot];
+            } else if (SR) {
                 const uint64_t number = (((elem_offset >> 3) + vec) << 2) | kAccumSlot;
                 w = philox4x32_10(static_cast<uint32_t>(number), static_cast<uint32_t>(number >> 32), tensor_id, seed_hi, K);
-                if (MODE == 1) w = straddle_slot(r, w);
             }
-            if (mine) {
-                uint32_t o[4];
+            uint32_t o[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t aw = word_of(av, j);
-                    const float s0 = accumulate(bf16_lo(aw), ge[2 * j], scale);
-                    const float s1 = accumulate(bf16_hi(aw), ge[2 * j + 1], scale);
-                    o[j] = pack_top_halves(round_sum_word_nan_safe<SR, false>(s0, word_of(w, j)),
-                                           round_sum_word_nan_safe<SR, true>(s1, word_of(w, j)));
-                }
-                st16(acc, vec, make_uint4(o[0], o[1], o[2], o[3]));
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t aw = word_of(av, j);
+                const float s0 = accumulate(bf16_lo(aw), ge[2 * j], scale);
+                const float s1 = accumulate(bf16_hi(aw), ge[2 * j + 1], scale);
+                o[j] = pack_top_halves(round_sum_word_nan_safe<SR, false>(s0, word_of(w, j)),
+                                       round_sum_word_nan_safe<SR, true>(s1, word_of(w, j)));
             }
+            st16(acc, vec, make_uint4(o[0], o[1], o[2], o[3]));
         }
         done = nvec << 3;
     }
@@ -80,7 +83,7 @@ cudaError_t launch_accum_mode(uint16_t* acc, const void* g, uint64_t n, float sc
                               uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev,
                               cudaStream_t stream) {
     auto k = k_sr_accumulate<G32, SR, MODE>;
-    const uint64_t items = MODE == 0 ? n : MODE == 1 ? ((n >> 3) / 31 + 1) * 32 + 8 : (n >> 3) + 8;
+    const uint64_t items = MODE == 0 ? n : (n >> 3) + 8;
     k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(acc, g, n, scale, elem_offset, tensor_id, seed_hi, K);
     return cudaGetLastError();
 }

@@ -121,12 +121,15 @@ __device__ __forceinline__ uint4 straddling_noise(uint64_t idx0, uint32_t slot, 
                       __funnelshift_r(y3, y4, sh));
 }
 
-// The same 128 bits when the 32 lanes of a warp hold consecutive noise groups (lane l: group A + l):
-// lane l's second group is lane l + 1's first, so the words it needs from group A + 1 come from its
-// neighbour by shuffle and nobody computes a call twice.  Lane 31 has no neighbour; the kernels that
-// use this give lanes 0..30 a vector each and let lane 31 compute the noise of the group after lane
-// 30's only.  R = idx0 & 7 (1..7) is the same for every vector of a launch: the kernels switch on it
-// once per vector, so that word selection is fixed at compile time inside each case.
+// The same 128 bits without computing any call twice.  The lanes of a warp hold 32 consecutive vectors (a ROW);
+// every lane computes the call of the group its vector ENDS in (group A + 1).  The group its vector starts in is
+// the one the previous vector ends in: lanes 1..31 take those words from the lane below by shuffle.  Lane 0 has
+// no lane below it: the call of the group its row starts in (the row's HEAD call) comes from a table in shared
+// memory that the warp refills every 32 iterations, lane j computing the head call of the row the warp will be
+// on j iterations later.  Per (vector, slot) this is 1 + 1/32 calls, against two when every thread computes both
+// groups, and the warps keep the plain grid-stride order over rows (whole 512-byte rows, consecutive warps on
+// consecutive rows).  R = idx0 & 7 (1..7) is the same for every vector of a launch: the kernels switch on it
+// once per vector, so that the word selection is fixed at compile time inside each case.
 template <int R>
 __device__ __forceinline__ uint4 straddle_select(const uint4 a, const uint4 b) {
     const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
@@ -137,48 +140,71 @@ __device__ __forceinline__ uint4 straddle_select(const uint4 a, const uint4 b) {
     return make_uint4(w[k], w[k + 1], w[k + 2], w[k + 3]);
 }
 
-// every lane of the warp must call this (full-mask shuffles)
+// own: this lane's call (the group its vector ends in); head: the row's head call (same value in every lane).
+// Every lane of the warp must call this (full-mask shuffles).
 template <int R>
-__device__ __forceinline__ uint4 straddle_from_neighbour(const uint4 a) {
-    constexpr int need = (R + 1) >> 1;   // words of the next group that the vector reaches into
-    uint4 b = make_uint4(0, 0, 0, 0);
-    b.x = __shfl_down_sync(0xFFFFFFFFu, a.x, 1);
-    if (need > 1) b.y = __shfl_down_sync(0xFFFFFFFFu, a.y, 1);
-    if (need > 2) b.z = __shfl_down_sync(0xFFFFFFFFu, a.z, 1);
-    if (need > 3) b.w = __shfl_down_sync(0xFFFFFFFFu, a.w, 1);
-    return straddle_select<R>(a, b);
+__device__ __forceinline__ uint4 chain_words(const uint4 own, const uint4 head, uint32_t lane) {
+    constexpr int k = R >> 1;   // first word of the starting group that the vector uses
+    uint4 a = head;
+    const bool first = lane == 0u;
+    if (k <= 0) { const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, own.x, 1); a.x = first ? head.x : t; }
+    if (k <= 1) { const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, own.y, 1); a.y = first ? head.y : t; }
+    if (k <= 2) { const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, own.z, 1); a.z = first ? head.z : t; }
+    { const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, own.w, 1); a.w = first ? head.w : t; }
+    return straddle_select<R>(a, own);
 }
 
-// one slot: in, the lane's own group call; out, the noise words of the lane's vector (lanes 0..30)
-__device__ __forceinline__ uint4 straddle_slot(uint32_t r, const uint4 w) {
-    switch (r) {
-        case 1: return straddle_from_neighbour<1>(w);
-        case 2: return straddle_from_neighbour<2>(w);
-        case 3: return straddle_from_neighbour<3>(w);
-        case 4: return straddle_from_neighbour<4>(w);
-        case 5: return straddle_from_neighbour<5>(w);
-        case 6: return straddle_from_neighbour<6>(w);
-        case 7: return straddle_from_neighbour<7>(w);
-        default: return w;
+// Noise of a grid-stride walk over rows whose vectors straddle two noise groups.  SLOTS: bit s set = rounding
+// slot s is drawn.  FIXED_C1: every index of the launch has the same high counter word c1 (the flat step
+// launches are cut that way); otherwise it is taken from the 64-bit call number.  `heads` is this warp's part of
+// a shared-memory table: 32 entries of 16 bytes per drawn slot.
+template <uint32_t SLOTS, bool FIXED_C1>
+struct RowChain {
+    static constexpr int kSlots = ((SLOTS >> 0) & 1) + ((SLOTS >> 1) & 1) + ((SLOTS >> 2) & 1) + ((SLOTS >> 3) & 1);
+    static constexpr int kTableEntries = 32 * (kSlots > 0 ? kSlots : 1);      // uint4 entries per warp
+    static __device__ __forceinline__ int pos(uint32_t s) { return __popc(SLOTS & ((1u << s) - 1u)); }
+
+    uint4* heads;
+    uint64_t group0;     // noise group of the launch's first element
+    uint64_t stride;     // vectors between a warp's consecutive rows
+    uint32_t r, lane, c1, c2, c3;
+
+    // Head calls of the rows this warp is on in iterations k .. k + 31; row_vec0: first vector of its row in
+    // iteration k.  Every lane must call it (when k is a multiple of 32, before `words`).
+    __device__ __forceinline__ void refill(uint64_t row_vec0, const PhiloxKeys& K) const {
+        const uint64_t number = (group0 + row_vec0 + lane * stride) << 2;
+        const uint32_t h0 = static_cast<uint32_t>(number), h1 = FIXED_C1 ? c1 : static_cast<uint32_t>(number >> 32);
+        __syncwarp();                                                       // the previous 32 entries have been read
+#pragma unroll
+        for (uint32_t s = 0; s < 4; ++s)
+            if (SLOTS & (1u << s)) heads[pos(s) * 32 + lane] = philox4x32_10(h0 | s, h1, c2, c3, K);
+        __syncwarp();
     }
-}
 
-// in: each lane's own group calls; out: the noise words of each lane's vector (lanes 0..30)
-template <uint32_t FLAGS>
-__device__ __forceinline__ void straddle_slots(uint32_t r, uint4& wx, uint4& wm, uint4& wv) {
-#define SR_STRADDLE_CASE(R)                                           \
-    case R:                                                           \
-        if (FLAGS & 1u) wx = straddle_from_neighbour<R>(wx);          \
-        if (FLAGS & 2u) wm = straddle_from_neighbour<R>(wm);          \
-        if (FLAGS & 4u) wv = straddle_from_neighbour<R>(wv);          \
+    // Noise words w[s] of this lane's vector `vec` in iteration k.  Every lane must call it.
+    __device__ __forceinline__ void words(uint64_t vec, uint32_t k, const PhiloxKeys& K, uint4 (&w)[4]) const {
+        const uint64_t number = (group0 + vec + 1) << 2;
+        const uint32_t c0 = static_cast<uint32_t>(number), c1v = FIXED_C1 ? c1 : static_cast<uint32_t>(number >> 32);
+        uint4 own[4], head[4];
+#pragma unroll
+        for (uint32_t s = 0; s < 4; ++s)
+            if (SLOTS & (1u << s)) {
+                own[s] = philox4x32_10(c0 | s, c1v, c2, c3, K);
+                head[s] = heads[pos(s) * 32 + (k & 31u)];
+            }
+#define SR_CHAIN_CASE(R)                                                            \
+    case R:                                                                         \
+        _Pragma("unroll") for (uint32_t s = 0; s < 4; ++s)                          \
+            if (SLOTS & (1u << s)) w[s] = chain_words<R>(own[s], head[s], lane);    \
         break;
-    switch (r) {
-        SR_STRADDLE_CASE(1) SR_STRADDLE_CASE(2) SR_STRADDLE_CASE(3) SR_STRADDLE_CASE(4)
-        SR_STRADDLE_CASE(5) SR_STRADDLE_CASE(6) SR_STRADDLE_CASE(7)
-        default: break;
+        switch (r) {
+            SR_CHAIN_CASE(1) SR_CHAIN_CASE(2) SR_CHAIN_CASE(3) SR_CHAIN_CASE(4)
+            SR_CHAIN_CASE(5) SR_CHAIN_CASE(6) SR_CHAIN_CASE(7)
+            default: break;
+        }
+#undef SR_CHAIN_CASE
     }
-#undef SR_STRADDLE_CASE
-}
+};
 
 // ---- reference vector: IEEE square root / division, NaN rule -------------------------------
 // GROUPED = true needs idx0 (global index of the vector's first element) to be a multiple of 8: the
@@ -328,18 +354,19 @@ __device__ __forceinline__ void step_scalar(uint16_t* p, const void* g, uint16_t
 inline bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
 
 template <typename Kernel>
-int resident_blocks(Kernel kernel, const DeviceInfo& dev, int threads = kBlockThreads) {
+int resident_blocks(Kernel kernel, const DeviceInfo& dev, int threads = kBlockThreads, size_t dynamic_smem = 0) {
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, 0) != cudaSuccess || per_sm < 1)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, dynamic_smem) != cudaSuccess || per_sm < 1)
         per_sm = 1;
     return per_sm * dev.sm_count;
 }
 
 // grid for `work_items` thread-items: no more blocks than are resident at once, no more than needed
 template <typename Kernel>
-unsigned grid_for(Kernel kernel, uint64_t work_items, const DeviceInfo& dev, int threads = kBlockThreads) {
+unsigned grid_for(Kernel kernel, uint64_t work_items, const DeviceInfo& dev, int threads = kBlockThreads,
+                  size_t dynamic_smem = 0) {
     const uint64_t needed = (work_items + threads - 1) / threads;
-    const uint64_t resident = static_cast<uint64_t>(resident_blocks(kernel, dev, threads));
+    const uint64_t resident = static_cast<uint64_t>(resident_blocks(kernel, dev, threads, dynamic_smem));
     const uint64_t g = needed < resident ? needed : resident;
     return static_cast<unsigned>(g < 1 ? 1 : g);
 }

@@ -1,6 +1,8 @@
 // Flat-buffer kernel of the fused SR-AdamW step and its launcher, for one gradient type.
 #pragma once
 
+#include <atomic>
+
 #include "adamw_body.cuh"
 
 // Direct-load shape (FP32 gradients): the next vector's loads are issued before the current vector is
@@ -41,14 +43,15 @@ k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n
 
 // The hot kernel (modes 2 and 3 of the launcher): 16-byte vectors, branch-free arithmetic, gradient
 // used as is or multiplied by gscale (VAR bit 0), epsilon outside or under the square root (VAR bit 1).
-// VAR bit 2: elem_offset is not a multiple of 8 (31 vectors per warp, noise exchanged between lanes).  Every
+// VAR bit 2: elem_offset is not a multiple of 8 (noise exchanged between lanes).  Every
 // index of the launch has the same (index >> 33) = c1.  Same persistent grid.  STAGED = true: each
 // thread keeps its next vectors in flight -- while vector k is computed out of shared memory, the
 // asynchronous copies of vectors k + T, ... are already under way (kFlatStages slots per thread and
 // array).  SHAPE 0: direct loads into registers, kBlockThreads x kMinBlocksPerSM; 1: staged, same
 // block shape, kShortStages; 2: staged, kFlatStagedThreads x kFlatStagedMinBlocks, kFlatStages.
 template <bool G32, uint32_t FLAGS, int VAR, int SHAPE>
-__global__ void __launch_bounds__(SHAPE == 2 ? kFlatStagedThreads : kBlockThreads, SHAPE == 2 ? kFlatStagedMinBlocks : kMinBlocksPerSM)
+__global__ void __launch_bounds__(SHAPE == 2 ? kFlatStagedThreads : kBlockThreads,
+                                  SHAPE == 2 ? kFlatStagedMinBlocks : (VAR & 4) ? kStraddleMinBlocks : kMinBlocksPerSM)
 k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset,
                      uint32_t c1, uint32_t tensor_id, uint32_t seed_hi, const __grid_constant__ PhiloxKeys K,
                      const __grid_constant__ StepScalars S) {
@@ -56,38 +59,46 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
     constexpr bool STAGED = SHAPE != 0;
     constexpr int kThreads = SHAPE == 2 ? kFlatStagedThreads : kBlockThreads;
     constexpr int kStages = SHAPE == 2 ? kFlatStages : kShortStages;
-    __shared__ uint4 stage[STAGED ? kStages * kArrays * kThreads : 1];
+    // The long shape's staging fills the 48 KB of static shared memory; where it also needs the table of head
+    // calls (straddling vectors), both live in dynamic shared memory that the launcher sizes.
+    constexpr bool kDynamic = SHAPE == 2 && (VAR & 4) != 0;
+    constexpr int kStageEntries = STAGED ? kStages * kArrays * kThreads : 1;
+    extern __shared__ uint4 dynamic_smem[];
+    __shared__ uint4 stage_static[kDynamic ? 1 : kStageEntries];
+    uint4* const stage = kDynamic ? dynamic_smem : stage_static;
     const float gscale = S.gscale_dev ? __ldg(S.gscale_dev) : S.gscale;
     const uint64_t tid = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
     const uint64_t nvec = n >> 3;
     if constexpr ((VAR & 4) != 0) {
-        // elem_offset is not a multiple of 8: every vector straddles two noise groups.  Lanes 0..30 of a warp
-        // take 31 consecutive vectors; all 32 lanes compute the calls of 32 consecutive groups (lane 31 only
-        // that), and each vector's second group arrives from the next lane by shuffle: three calls per vector
-        // as in the aligned case, for 1/32 of the lanes.  The loop is uniform over the warp (the shuffles need
-        // every lane); lanes without a vector skip the memory accesses and the arithmetic.
+        // elem_offset is not a multiple of 8: every vector straddles two noise groups.  Same grid-stride walk over
+        // rows of 32 vectors as below; every lane computes the calls of the group its vector ends in and receives
+        // those of the group it starts in from the lane below (RowChain): three calls per vector as in the
+        // aligned case, plus 3/32 for the head calls.  The loop is uniform over the warp (the shuffles need every
+        // lane) and covers whole rows only; the vectors of the last, partial row go element by element with the
+        // ragged tail.
+        using Chain = RowChain<FLAGS & 7u, true>;
+        __shared__ uint4 heads_static[kDynamic ? 1 : (kThreads / 32) * Chain::kTableEntries];
+        uint4* const heads = kDynamic ? dynamic_smem + kStageEntries : heads_static;
         const uint32_t lane = threadIdx.x & 31u;
-        const bool worker = lane != 31u;
-        const uint64_t wstride = (stride >> 5) * 31u;              // vectors per pass of the grid
-        const uint32_t r = static_cast<uint32_t>(elem_offset) & 7u;
-        const uint64_t group0 = elem_offset >> 3;                   // noise group of the first element
-        // call number 4 * group + slot, low word; advances by 4 * wstride per pass (the high word c1 is fixed)
-        uint32_t c0 = static_cast<uint32_t>((group0 + (tid >> 5) * 31u + lane) << 2);
-        const uint32_t c0_step = static_cast<uint32_t>(wstride << 2);
-        auto noise = [&](uint4& wx, uint4& wm, uint4& wv) {
-            if (FLAGS & 1u) wx = philox4x32_10(c0, c1, tensor_id, seed_hi, K);
-            if (FLAGS & 2u) wm = philox4x32_10(c0 + 1, c1, tensor_id, seed_hi, K);
-            if (FLAGS & 4u) wv = philox4x32_10(c0 + 2, c1, tensor_id, seed_hi, K);
-            straddle_slots<FLAGS>(r, wx, wm, wv);
-            c0 += c0_step;
+        const Chain chain{heads + (threadIdx.x >> 5) * Chain::kTableEntries, elem_offset >> 3, stride,
+                          static_cast<uint32_t>(elem_offset) & 7u, lane, c1, tensor_id, seed_hi};
+        const uint64_t row_vecs = nvec & ~static_cast<uint64_t>(31);      // vectors in whole rows
+        uint32_t k = 0;
+        auto noise = [&](uint64_t vec, uint4& wx, uint4& wm, uint4& wv) {
+            if ((k & 31u) == 0u) chain.refill(vec - lane, K);
+            uint4 w[4];
+            chain.words(vec, k, K, w);
+            ++k;
+            if (FLAGS & 1u) wx = w[0];
+            if (FLAGS & 2u) wm = w[1];
+            if (FLAGS & 4u) wv = w[2];
         };
-        uint64_t wb = (tid >> 5) * 31u;                             // first vector of this warp in this pass
         if (STAGED) {
             uint4* const mine = stage + threadIdx.x;
             auto slot = [&](int s, int a) -> uint4* { return mine + (s * kArrays + a) * kThreads; };
             auto issue = [&](uint64_t vec, int s) {
-                if (worker && vec < nvec) {
+                if (vec < row_vecs) {
                     async_copy16(slot(s, 0), reinterpret_cast<const uint4*>(p) + vec);
                     async_copy16(slot(s, 1), reinterpret_cast<const uint4*>(m) + vec);
                     async_copy16(slot(s, 2), reinterpret_cast<const uint4*>(v) + vec);
@@ -101,30 +112,27 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
                 async_copy_commit();
             };
 #pragma unroll
-            for (int s = 0; s < kStages - 1; ++s) issue(wb + s * wstride + lane, s);
+            for (int s = 0; s < kStages - 1; ++s) issue(tid + s * stride, s);
             int s = 0;
-            for (; wb < nvec; wb += wstride) {
-                const uint64_t vec = wb + lane;
+            for (uint64_t vec = tid; vec < row_vecs; vec += stride) {
                 int ahead = s + kStages - 1;
                 if (ahead >= kStages) ahead -= kStages;
-                issue(vec + (kStages - 1) * wstride, ahead);
+                issue(vec + (kStages - 1) * stride, ahead);
                 uint4 wx = make_uint4(0, 0, 0, 0), wm = wx, wv = wx;
-                noise(wx, wm, wv);
+                noise(vec, wx, wm, wv);
                 async_copy_wait<kStages - 1>();
-                if (worker && vec < nvec) {
-                    const uint4 pv = *slot(s, 0), mv = *slot(s, 1), vv = *slot(s, 2);
-                    float ge[8];
-                    unpack_grad8<G32>(*slot(s, 3), G32 ? *slot(s, kArrays - 1) : make_uint4(0, 0, 0, 0), ge);
-                    step_vec8_fast_noise<G32, FLAGS, VAR>(p, g, m, v, vec, elem_offset + (vec << 3), pv, mv, vv, ge, wx, wm, wv,
-                                                            tensor_id, seed_hi, gscale, K, S);
-                }
+                const uint4 pv = *slot(s, 0), mv = *slot(s, 1), vv = *slot(s, 2);
+                float ge[8];
+                unpack_grad8<G32>(*slot(s, 3), G32 ? *slot(s, kArrays - 1) : make_uint4(0, 0, 0, 0), ge);
+                step_vec8_fast_noise<G32, FLAGS, VAR>(p, g, m, v, vec, elem_offset + (vec << 3), pv, mv, vv, ge, wx, wm, wv,
+                                                        tensor_id, seed_hi, gscale, K, S);
                 if (++s == kStages) s = 0;
             }
             async_copy_wait<0>();
         } else {
             uint4 pv = make_uint4(0, 0, 0, 0), mv = pv, vv = pv, g0 = pv, g1 = pv;
             auto load = [&](uint64_t vec, uint4& a, uint4& b, uint4& c, uint4& d0, uint4& d1) {
-                if (worker && vec < nvec) {
+                if (vec < row_vecs) {
                     a = ld16(p, vec);
                     b = ld16(m, vec);
                     c = ld16(v, vec);
@@ -136,19 +144,16 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
                     }
                 }
             };
-            load(wb + lane, pv, mv, vv, g0, g1);
-            for (; wb < nvec; wb += wstride) {
-                const uint64_t vec = wb + lane;
+            load(tid, pv, mv, vv, g0, g1);
+            for (uint64_t vec = tid; vec < row_vecs; vec += stride) {
                 uint4 pn = pv, mn = mv, vn = vv, gn0 = g0, gn1 = g1;
-                load(vec + wstride, pn, mn, vn, gn0, gn1);
+                load(vec + stride, pn, mn, vn, gn0, gn1);
                 uint4 wx = make_uint4(0, 0, 0, 0), wm = wx, wv = wx;
-                noise(wx, wm, wv);
-                if (worker && vec < nvec) {
-                    float ge[8];
-                    unpack_grad8<G32>(g0, g1, ge);
-                    step_vec8_fast_noise<G32, FLAGS, VAR>(p, g, m, v, vec, elem_offset + (vec << 3), pv, mv, vv, ge, wx, wm, wv,
-                                                            tensor_id, seed_hi, gscale, K, S);
-                }
+                noise(vec, wx, wm, wv);
+                float ge[8];
+                unpack_grad8<G32>(g0, g1, ge);
+                step_vec8_fast_noise<G32, FLAGS, VAR>(p, g, m, v, vec, elem_offset + (vec << 3), pv, mv, vv, ge, wx, wm, wv,
+                                                        tensor_id, seed_hi, gscale, K, S);
                 pv = pn; mv = mn; vv = vn; g0 = gn0; g1 = gn1;
             }
         }
@@ -217,9 +222,10 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
             step_vec8_fast<G32, FLAGS, VAR>(p, g, m, v, vec, elem_offset + (vec << 3), c1, tensor_id, seed_hi, gscale, K, S);
 #endif
     }
-    const uint64_t done = nvec << 3;
-    if (tid < n - done)
-        step_scalar<G32, FLAGS>(p, g, m, v, done + tid, elem_offset + done + tid, tensor_id, seed_hi, gscale, K, S);
+    // ragged tail; with straddling vectors also the last, partial row (fewer than 32 * 8 + 8 elements)
+    const uint64_t done = ((VAR & 4) != 0 ? nvec & ~static_cast<uint64_t>(31) : nvec) << 3;
+    for (uint64_t i = done + tid; i < n; i += stride)
+        step_scalar<G32, FLAGS>(p, g, m, v, i, elem_offset + i, tensor_id, seed_hi, gscale, K, S);
 }
 
 // Which gradient types use the staged variant.  Measured on B200 (same GPU, back to back): BF16
@@ -227,12 +233,6 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
 // pieces per vector) 77.7% staged vs 93.2% direct at 832M elements, so they stay direct.
 #ifndef SR_STAGE_BF16
 #define SR_STAGE_BF16 1
-#endif
-// Launches whose offset is not a multiple of 8 keep the short shape at every length.  Measured on B200,
-// 6.7B elements, same GPU: 20.7 ms with 128 x 5 blocks, 21.3 ms with 256 x 2 (and 21.7 ms for the version
-// in which every thread computed both straddled groups itself).
-#ifndef SR_STRADDLE_LONG_SHAPE
-#define SR_STRADDLE_LONG_SHAPE 0
 #endif
 #ifndef SR_STAGE_F32
 #define SR_STAGE_F32 0
@@ -242,17 +242,36 @@ template <bool G32, uint32_t FLAGS, int MODE, bool EPS_IN = false, bool STRADDLE
 cudaError_t launch_flat_mode(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset,
                              uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K, const StepScalars& S,
                              const DeviceInfo& dev, cudaStream_t stream) {
-    // + 8: enough threads for the ragged tail; straddling launches give a vector to 31 of every 32 threads
-    const uint64_t items = MODE == 0 ? n : STRADDLE ? ((n >> 3) / 31 + 1) * 32 + 8 : (n >> 3) + 8;
+    // + 8: enough threads for the ragged tail
+    const uint64_t items = MODE == 0 ? n : (n >> 3) + 8;
     if (MODE == 2 || MODE == 3) {
         constexpr bool kStaged = G32 ? (SR_STAGE_F32 != 0) : (SR_STAGE_BF16 != 0);
         const uint32_t c1 = static_cast<uint32_t>(elem_offset >> 33);
-        if (kStaged && n >= kLongLaunchElems && (!STRADDLE || SR_STRADDLE_LONG_SHAPE)) {
-            auto k = k_sr_adamw_flat_fast<G32, FLAGS, (MODE == 3 ? 1 : 0) | (EPS_IN ? 2 : 0) | (STRADDLE ? 4 : 0), kStaged ? 2 : 0>;
-            constexpr int kThreads = kStaged ? kFlatStagedThreads : kBlockThreads;
-            k<<<grid_for(k, items, dev, kThreads), kThreads, 0, stream>>>(p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
-        } else {
-            auto k = k_sr_adamw_flat_fast<G32, FLAGS, (MODE == 3 ? 1 : 0) | (EPS_IN ? 2 : 0) | (STRADDLE ? 4 : 0), kStaged ? 1 : 0>;
+        constexpr int kVar = (MODE == 3 ? 1 : 0) | (EPS_IN ? 2 : 0) | (STRADDLE ? 4 : 0);
+        bool launched = false;
+        if constexpr (kStaged) {
+            if (n >= kLongLaunchElems) {
+                auto k = k_sr_adamw_flat_fast<G32, FLAGS, kVar, 2>;
+                size_t dynamic = 0;
+                if (STRADDLE) {
+                    // staging + one table of head calls per warp: above the 48 KB a kernel gets without asking
+                    dynamic = sizeof(uint4) * (kFlatStages * (G32 ? 5 : 4) * kFlatStagedThreads +
+                                               (kFlatStagedThreads / 32) * RowChain<FLAGS & 7u, true>::kTableEntries);
+                    static std::atomic<int> prepared[kMaxDevices] = {};      // per kernel instantiation and device
+                    if (!prepared[dev.index].load(std::memory_order_acquire)) {
+                        const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                                   static_cast<int>(dynamic));
+                        if (e != cudaSuccess) return e;
+                        prepared[dev.index].store(1, std::memory_order_release);
+                    }
+                }
+                k<<<grid_for(k, items, dev, kFlatStagedThreads, dynamic), kFlatStagedThreads, dynamic, stream>>>(
+                    p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
+                launched = true;
+            }
+        }
+        if (!launched) {
+            auto k = k_sr_adamw_flat_fast<G32, FLAGS, kVar, kStaged ? 1 : 0>;
             k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
         }
     } else {

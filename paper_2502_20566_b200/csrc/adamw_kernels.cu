@@ -37,33 +37,30 @@ k_sr_downcast(const float* __restrict__ src, uint16_t* __restrict__ dst, uint64_
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
     uint64_t done = 0;
     if (MODE == 1) {
-        // every vector straddles two noise groups: lanes 0..30 take a vector each, all 32 lanes compute one
-        // group's call and pass its words to the lane before them (see straddle_from_neighbour)
-        const uint64_t nvec = n >> 3;
+        // every vector straddles two noise groups: every lane computes the call of the group its vector ends in and
+        // takes the other group's words from the lane below (RowChain)
+        using Chain = RowChain<1u, false>;
+        __shared__ uint4 heads[(kBlockThreads / 32) * Chain::kTableEntries];
+        const uint64_t row_vecs = (n >> 3) & ~static_cast<uint64_t>(31);   // whole rows of 32 vectors; the rest goes element by element
         const uint32_t lane = threadIdx.x & 31u;
-        const uint64_t wstride = (stride >> 5) * 31u;
-        const uint32_t r = static_cast<uint32_t>(elem_offset) & 7u;
-        for (uint64_t wb = (tid >> 5) * 31u; wb < nvec; wb += wstride) {
-            const uint64_t vec = wb + lane;
-            const bool mine = lane != 31u && vec < nvec;
-            uint4 a = make_uint4(0, 0, 0, 0), b = a;
-            if (mine) {
-                a = ld16(src, 2 * vec);
-                b = ld16(src, 2 * vec + 1);
-            }
-            const uint64_t number = ((elem_offset >> 3) + vec) << 2;      // slot 0 of the group that holds the vector's first element
-            const uint4 w = straddle_slot(r, philox4x32_10(static_cast<uint32_t>(number), static_cast<uint32_t>(number >> 32),
-                                                           tensor_id, seed_hi, K));
-            if (mine) {
-                uint4 o;
-                o.x = cast_pair(a.x, a.y, w.x);
-                o.y = cast_pair(a.z, a.w, w.y);
-                o.z = cast_pair(b.x, b.y, w.z);
-                o.w = cast_pair(b.z, b.w, w.w);
-                st16(dst, vec, o);
-            }
+        const Chain chain{heads + (threadIdx.x >> 5) * Chain::kTableEntries, elem_offset >> 3, stride,
+                          static_cast<uint32_t>(elem_offset) & 7u, lane, 0u, tensor_id, seed_hi};
+        uint32_t k = 0;
+        for (uint64_t vec = tid; vec < row_vecs; vec += stride, ++k) {
+            const uint4 a = ld16(src, 2 * vec);
+            const uint4 b = ld16(src, 2 * vec + 1);
+            if ((k & 31u) == 0u) chain.refill(vec - lane, K);
+            uint4 w4[4];
+            chain.words(vec, k, K, w4);
+            const uint4 w = w4[0];
+            uint4 o;
+            o.x = cast_pair(a.x, a.y, w.x);
+            o.y = cast_pair(a.z, a.w, w.y);
+            o.z = cast_pair(b.x, b.y, w.z);
+            o.w = cast_pair(b.z, b.w, w.w);
+            st16(dst, vec, o);
         }
-        done = nvec << 3;
+        done = row_vecs << 3;
     } else if (MODE == 2) {
         const uint64_t nvec = n >> 3;
         for (uint64_t vec = tid; vec < nvec; vec += stride) {
@@ -90,7 +87,7 @@ template <int MODE>
 cudaError_t launch_cast_mode(const float* src, uint16_t* dst, uint64_t n, uint64_t elem_offset, uint32_t tensor_id,
                              uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev, cudaStream_t stream) {
     auto k = k_sr_downcast<MODE>;
-    const uint64_t items = MODE == 0 ? n : MODE == 1 ? ((n >> 3) / 31 + 1) * 32 + 8 : (n >> 3) + 8;
+    const uint64_t items = MODE == 0 ? n : (n >> 3) + 8;
     k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(src, dst, n, elem_offset, tensor_id, seed_hi, K);
     return cudaGetLastError();
 }

@@ -22,7 +22,6 @@ sr_status cuda_fail(cudaError_t e) {
     return SR_ERR_CUDA;
 }
 
-constexpr int kMaxDevices = 64;
 struct DeviceSlot {
     std::atomic<bool> known{false};
     DeviceInfo info{};
@@ -48,6 +47,7 @@ sr_status current_device(DeviceInfo* out) {
             if (e != cudaSuccess) return cuda_fail(e);
             slot.info.sm_count = sm;
             slot.info.cc_major = major;
+            slot.info.index = dev;
             slot.known.store(true, std::memory_order_release);
         }
     }

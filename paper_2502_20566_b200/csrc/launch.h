@@ -50,18 +50,27 @@ constexpr uint32_t kMtChunkElems = 8192;   // multiple of 8; never crosses a mul
 #ifndef SR_FLAT_STAGES
 #define SR_FLAT_STAGES 3
 #endif
+#ifndef SR_STRADDLE_MIN_BLOCKS
+#define SR_STRADDLE_MIN_BLOCKS 5
+#endif
+constexpr int kStraddleMinBlocks = SR_STRADDLE_MIN_BLOCKS;   // flat step at offsets that are not multiples of 8
 constexpr int kBlockThreads = SR_BLOCK_THREADS;
 constexpr int kMinBlocksPerSM = SR_MIN_BLOCKS_PER_SM;
 constexpr int kFlatStagedThreads = SR_FLAT_STAGED_THREADS;
 constexpr int kFlatStagedMinBlocks = SR_FLAT_STAGED_MIN_BLOCKS;
 constexpr int kFlatStages = SR_FLAT_STAGES;
 constexpr int kMtStages = 2;
-constexpr int kShortStages = 2;
+#ifndef SR_SHORT_STAGES
+#define SR_SHORT_STAGES 2
+#endif
+constexpr int kShortStages = SR_SHORT_STAGES;
 constexpr uint64_t kLongLaunchElems = static_cast<uint64_t>(1) << 29;
 
+constexpr int kMaxDevices = 64;
 struct DeviceInfo {
     int sm_count;
     int cc_major;
+    int index;      // CUDA device ordinal, < kMaxDevices
 };
 
 cudaError_t launch_downcast(const float* src, uint16_t* dst, uint64_t n, uint64_t elem_offset, uint32_t tensor_id,

@@ -200,6 +200,40 @@ def test_offsets_that_split_noise_groups(env, r):
     assert mismatches(bits(acc), want) == 0
 
 
+@pytest.mark.parametrize("n,r", [((1 << 25) + 77, 3), (200_000_013, 5)])
+def test_offsets_that_split_noise_groups_over_many_runs(env, n, r):
+    """The same at sizes where every warp walks several runs of consecutive vectors (short runs at 2^25 elements,
+    the longest ones at 2e8), so that noise words cross from row to row, from run to run and from warp to warp:
+    step with both gradient types, cast and accumulation, every element compared."""
+    oracle, binding, synth, dev = env
+    offset = (5 << 33) - 8 * 100_000 + r
+    for g_dtype, flags in ((torch.bfloat16, 7), (torch.float32, 6)):
+        p, g, m, v = synth.adamw_state(n, 70 + r, dev, g_dtype=g_dtype)
+        assert run_both(env, p, g, m, v, HP, seed=(9 << 32) | 1, step=4, tensor_id=3, elem_offset=offset, flags=flags) == (0, 0, 0)
+        del p, g, m, v
+    src = synth.downcast_mix(n, 71, dev)
+    dst = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    binding.sr_downcast_f32_bf16(src, dst, seed=11, step=1, tensor_id=2, elem_offset=offset)
+    torch.cuda.synchronize()
+    assert mismatches(bits(dst), oracle.sr_downcast(src.cpu().numpy().copy(), 11, 1, 2, offset)) == 0
+    del src, dst
+    _, g, acc, _ = synth.adamw_state(n, 72, dev)
+    want = bits(acc)
+    binding.sr_accumulate_bf16(acc, g, 0.5, seed=5, step=2, tensor_id=1, elem_offset=offset)
+    oracle.sr_accumulate(want, bits(g), 0.5, 5, 2, 1, offset, True)
+    torch.cuda.synchronize()
+    assert mismatches(bits(acc), want) == 0
+
+
+def test_offset_that_splits_noise_groups_long_launch(env):
+    """2^29 elements and more take the long launch shape (staging and the table of head calls in dynamic shared
+    memory) at offsets that are not multiples of 8 as well: every element compared, ragged end included."""
+    _, _, synth, dev = env
+    n = (1 << 29) + 8 * 37 + 5
+    p, g, m, v = synth.adamw_state(n, 81, dev)
+    assert run_both(env, p, g, m, v, HP, seed=3, step=7, tensor_id=1, elem_offset=(1 << 33) - 8 * 1000 + 3) == (0, 0, 0)
+
+
 def test_flat_step_special_values(env):
     """NaN, infinities, zeros, subnormals and huge values in every input."""
     _, _, synth, dev = env
