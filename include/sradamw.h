@@ -228,6 +228,18 @@ sr_status grad_sqnorm_static(const void* g, sr_dtype g_dtype, uint64_t n, double
 sr_status sr_clip_scale(const double* sqnorm_dev, float accum_scale, float max_norm, float* gscale_out_dev,
                         void* stream);
 
+/* Self-check of the step kernels' arithmetic.  Algorithm 1's update divides the first moment by the root of the
+ * second (its last two lines); the fused kernels evaluate that square root and that division with fixed
+ * sequences of FP32 multiply-adds on the hardware's reciprocal / reciprocal-root seeds, which equal the IEEE
+ * round-to-nearest results inside the operand range the kernels check per vector (argument of the root and
+ * |numerator| in [2^-60, 2^60], denominator in [2^-30, 2^41]).  This call draws `sets` operand sets from
+ * Philox4x32-10 keyed by `seed` -- exponents uniform over those ranges; mantissas plain, just below a power of
+ * two or just above one; and denominators formed the way the kernels form them -- evaluates both forms and
+ * counts the results that differ: mismatches_dev[0] square roots, mismatches_dev[1] divisions (device memory,
+ * two uint64_t, overwritten).  Both counts are expected to be 0; the square root has also been compared on
+ * every FP32 value of its range. */
+sr_status sr_selftest_in_range_arithmetic(uint64_t seed, uint64_t sets, uint64_t* mismatches_dev, void* stream);
+
 const char* sr_status_string(sr_status s);
 int sr_last_cuda_error(void); /* cudaError_t of the last failing runtime call on this thread, else 0 */
 uint32_t sr_abi_version(void);

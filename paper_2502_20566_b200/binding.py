@@ -28,7 +28,7 @@ EXPORTS = (
     "sr_mt_plan_create", "sr_adamw_multi_tensor",
     "sr_mt_plan_destroy", "sr_mt_plan_total_elements", "grad_sqnorm_workspace_bytes", "grad_sqnorm",
     "grad_sqnorm_static", "grad_sqnorm_static_max_elements", "grad_sqnorm_multi_tensor", "grad_sqnorm_multi_tensor_workspace_bytes",
-    "sr_clip_scale", "sr_status_string", "sr_last_cuda_error", "sr_abi_version",
+    "sr_clip_scale", "sr_selftest_in_range_arithmetic", "sr_status_string", "sr_last_cuda_error", "sr_abi_version",
 )
 
 
@@ -117,6 +117,8 @@ def lib() -> ctypes.CDLL:
         L.grad_sqnorm_static_max_elements.restype = c_uint64
         L.sr_clip_scale.argtypes = [c_void_p, c_float, c_float, c_void_p, c_void_p]
         L.sr_clip_scale.restype = c_int
+        L.sr_selftest_in_range_arithmetic.argtypes = [c_uint64, c_uint64, c_void_p, c_void_p]
+        L.sr_selftest_in_range_arithmetic.restype = c_int
         L.sr_status_string.argtypes = [c_int]
         L.sr_status_string.restype = c_char_p
         L.sr_last_cuda_error.restype = c_int
@@ -354,6 +356,17 @@ def sr_clip_scale(sqnorm: torch.Tensor, accum_scale: float, max_norm: float, gsc
     with torch.cuda.device(sqnorm.device):
         _check(lib().sr_clip_scale(sqnorm.data_ptr(), accum_scale, max_norm, gscale_out.data_ptr(), _stream(stream)),
                "sr_clip_scale")
+
+
+def sr_selftest_in_range_arithmetic(seed: int, sets: int, mismatches: torch.Tensor, stream=None) -> None:
+    """Compare the step kernels' branch-free square root and division with the IEEE instructions on `sets` seeded
+    operand sets; mismatches (two int64 on the device) receives the counts (square roots, divisions)."""
+    _want(mismatches, torch.int64, "mismatches")
+    if mismatches.numel() < 2:
+        raise ValueError("mismatches needs two elements")
+    with torch.cuda.device(mismatches.device):
+        _check(lib().sr_selftest_in_range_arithmetic(seed, sets, mismatches.data_ptr(), _stream(stream)),
+               "sr_selftest_in_range_arithmetic")
 
 
 def sr_abi_version() -> int:

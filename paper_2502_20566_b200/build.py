@@ -20,7 +20,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libsradamw.so")
 SOURCES = ["api.cu", "adamw_kernels.cu", "adamw_flat_bf16.cu", "adamw_flat_f32.cu", "adamw_mt_bf16.cu",
-           "adamw_mt_f32.cu", "master_kernels.cu", "fp8_kernels.cu", "accum_kernels.cu", "reduce_kernels.cu"]
+           "adamw_mt_f32.cu", "master_kernels.cu", "fp8_kernels.cu", "accum_kernels.cu", "reduce_kernels.cu", "selftest_kernels.cu"]
 HEADERS = ["device_math.cuh", "launch.h", "adamw_body.cuh", "adamw_flat.cuh", "adamw_mt.cuh", os.path.join("..", "..", "include", "sradamw.h")]
 
 NVCC_FLAGS = [

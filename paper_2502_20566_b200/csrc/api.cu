@@ -153,6 +153,17 @@ sr_status sr_downcast_f32_bf16(const float* src, uint16_t* dst, uint64_t n, uint
     return e == cudaSuccess ? SR_OK : cuda_fail(e);
 }
 
+sr_status sr_selftest_in_range_arithmetic(uint64_t seed, uint64_t sets, uint64_t* mismatches_dev, void* stream) {
+    if (mismatches_dev == nullptr) return SR_ERR_INVALID_ARG;
+    DeviceInfo dev;
+    sr_status st = current_device(&dev);
+    if (st != SR_OK) return st;
+    const cudaError_t e = launch_selftest_in_range(sets, static_cast<uint32_t>(seed >> 32), make_keys(seed, 0),
+                                                   reinterpret_cast<unsigned long long*>(mismatches_dev), dev,
+                                                   static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SR_OK : cuda_fail(e);
+}
+
 sr_status sr_downcast_f32_fp8(const float* src, uint8_t* dst, uint64_t n, sr_fp8_format format, uint64_t seed,
                               uint32_t step, uint32_t tensor_id, uint64_t elem_offset, void* stream) {
     if (format != SR_FP8_E4M3 && format != SR_FP8_E5M2) return SR_ERR_INVALID_ARG;

@@ -12,100 +12,78 @@ namespace {
 // FMT 0: E4M3, 1: E5M2, 2: E2M1
 constexpr int kE4M3 = 0, kE5M2 = 1, kE2M1 = 2;
 
+constexpr uint32_t kE5M2InfCode = 0x7Cu;   // the other two formats have no infinity
+
 template <int FMT>
 struct Small {
     static constexpr int M = FMT == kE5M2 ? 2 : FMT == kE4M3 ? 3 : 1;
     static constexpr int kBias = FMT == kE5M2 ? 15 : FMT == kE4M3 ? 7 : 1;
-    static constexpr uint32_t kMaxCode = FMT == kE5M2 ? 0x7Bu : FMT == kE4M3 ? 0x7Eu : 0x7u;   // 57344, 448, 6
-    static constexpr uint32_t kMaxBits = FMT == kE5M2 ? 0x47600000u : FMT == kE4M3 ? 0x43E00000u : 0x40C00000u;   // as FP32
-    static constexpr uint32_t kInfCode = 0x7Cu;                              // E5M2 only: the others have no infinity
+    // largest level as FP32: 57344 (code 0x7B), 448 (code 0x7E), 6 (code 0x7)
+    static constexpr uint32_t kMaxBits = FMT == kE5M2 ? 0x47600000u : FMT == kE4M3 ? 0x43E00000u : 0x40C00000u;
     static constexpr uint32_t kMinBiasedExp = 127 + 1 - kBias;               // FP32 exponent field of the smallest normal level
 };
 
+// Multipliers read from constant memory.  The integer (ALU) pipe and the heavy half of the FMA pipe, which takes
+// every integer multiply-add, bound these kernels about equally.  Where a subtraction or a shift-add is better
+// placed on the FMA pipe it is written as a multiply-add whose multiplier is read from memory: a runtime value to
+// the compiler, which would otherwise turn it back into an ALU instruction.  Which operation sits on which pipe
+// was settled by measurement on B200 (2^28 values; see each use).
+__constant__ uint32_t kMul[3] = {0xFFFFFFFFu, 256u, 65536u};
+__device__ __forceinline__ uint32_t mul_minus1() { return kMul[0]; }
+__device__ __forceinline__ uint32_t mul_256() { return kMul[1]; }
+__device__ __forceinline__ uint32_t mul_65536() { return kMul[2]; }
+
 // The magnitude code of one value (sign handled by the caller).  a = |x| lies in the binade
 // Eq = max(E, 1 - bias); y = a / 2^(Eq - M) = k + f; move to level k + 1 iff r < floor(f * 2^32).
-// Evaluated with exact FP32 operations, which keeps most of the work off the integer pipe that
-// bounds this kernel: y = a * 2^(M - Eq) is a scaling by a power of two (exact, subnormal a
-// included; y < 2^(M+1)); adding 2^23 with rounding toward zero leaves k in the low bits of the sum;
-// f = y - k is exact; f * 2^32 < 2^32 is exact and its truncation to an integer is the threshold.
-// The code of level k' is ((Eq + bias - 1) << M) + k' for subnormal and normal levels alike.
-// Magnitudes at or beyond the largest level (infinity and NaN included, whose y is meaningless)
-// are replaced at the end.
-template <int FMT>
-__device__ __forceinline__ uint32_t sr_fp8_magnitude(uint32_t abits, uint32_t r) {
+//   a  = min(|x|, largest level)      one float minimum: saturation and infinity land on the largest level with
+//                                     f = 0, which never moves up
+//   Eq from max(a, smallest normal level), exponent field only
+//   z  = a * 2^(32 + M - Eq)          a scaling by a power of two: exact, subnormal a included; z < 2^(33 + M)
+//   Z  = z truncated to a 64-bit integer = (k : floor(f * 2^32))
+//   code = ((Eq + bias - 1) << M) + k + (r < low word of Z)      subnormal and normal levels alike
+// NAN_ABOVE (the FP8 formats): minimum and maximum propagate a NaN, its exponent field is all ones and Z = 0, so
+// its code comes out far above every level's and the caller's min(code, 0x7F) writes the NaN pattern.  Otherwise
+// (E2M1, which has no NaN) a NaN lands on the largest level like infinity.
+template <int FMT, bool NAN_ABOVE>
+__device__ __forceinline__ uint32_t sr_small_magnitude(float x, uint32_t r) {
     using F = Small<FMT>;
-    const uint32_t e = abits >> 23;                                            // biased FP32 exponent
-    const uint32_t eqb = e < F::kMinBiasedExp ? F::kMinBiasedExp : e;          // Eq + 127
-    const float scale = __uint_as_float(((254u + F::M) << 23) - (eqb << 23));  // 2^(M - Eq)
-    const float y = __fmul_rn(__uint_as_float(abits), scale);
-    const float t = __fadd_rz(y, 8388608.0f);                                  // 2^23 + k
-    const float f = __fsub_rn(y, __fsub_rn(t, 8388608.0f));
-    const uint32_t threshold = __float2uint_rz(__fmul_rn(f, 4294967296.0f));
-    uint32_t code = (eqb << F::M) + __float_as_uint(t) - (0x4B000000u + (F::kMinBiasedExp << F::M)) + (r < threshold ? 1u : 0u);
-    code = abits >= F::kMaxBits ? F::kMaxCode : code;
-    if (FMT == kE2M1) return code;
-    if (FMT == kE5M2) code = abits == 0x7F800000u ? F::kInfCode : code;
-    return abits > 0x7F800000u ? 0x7Fu : code;                                 // NaN -> 0x7F (its sign is dropped below)
+    float a, an;
+    if (NAN_ABOVE) {
+        asm("min.NaN.f32 %0, %1, %2;" : "=f"(a) : "f"(fabsf(x)), "f"(__uint_as_float(F::kMaxBits)));
+        asm("max.NaN.f32 %0, %1, %2;" : "=f"(an) : "f"(a), "f"(__uint_as_float(F::kMinBiasedExp << 23)));
+    } else {
+        a = fminf(fabsf(x), __uint_as_float(F::kMaxBits));
+        an = fmaxf(a, __uint_as_float(F::kMinBiasedExp << 23));
+    }
+    const uint32_t eqbits = __float_as_uint(an) & 0x7F800000u;                            // (Eq + 127) << 23
+    // 2^(32 + M - Eq): exponent field 127 + 32 + M - (Eq + 127) + 127, on the FMA pipe (0.354 -> 0.330 ms for E4M3)
+    const float scale = __uint_as_float(eqbits * mul_minus1() + ((286u + F::M) << 23));
+    const unsigned long long Z = __float2ull_rz(__fmul_rn(a, scale));
+    constexpr uint32_t kBase = F::kMinBiasedExp << F::M;
+    const uint32_t zlo = static_cast<uint32_t>(Z), zhi = static_cast<uint32_t>(Z >> 32);
+    // two orders of the same additions; measured: the first is 3 % faster for E2M1 and 3 % slower for E4M3
+    if (FMT == kE2M1) return ((eqbits >> (23 - F::M)) + zhi) + (r < zlo ? 1u - kBase : 0u - kBase);
+    return (eqbits >> (23 - F::M)) + (zhi - kBase + (r < zlo ? 1u : 0u));
 }
 
-// The same for two values at once with the packed FP32 instructions of sm_100 (each lane is the scalar
-// operation, rounding mode included): half the floating-point instructions.
-__device__ __forceinline__ uint64_t add_rz2(uint64_t a, uint64_t b) {
-    uint64_t d;
-    asm("add.rz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-
-template <int FMT>
-__device__ __forceinline__ uint32_t finish_code(uint32_t abits, uint32_t eqb, float t, float fscaled, uint32_t r) {
-    using F = Small<FMT>;
-    const uint32_t threshold = __float2uint_rz(fscaled);
-    uint32_t code = (eqb << F::M) + __float_as_uint(t) - (0x4B000000u + (F::kMinBiasedExp << F::M)) + (r < threshold ? 1u : 0u);
-    code = abits >= F::kMaxBits ? F::kMaxCode : code;
-    if (FMT == kE2M1) return code;
-    if (FMT == kE5M2) code = abits == 0x7F800000u ? F::kInfCode : code;
-    return abits > 0x7F800000u ? 0x7Fu : code;
-}
-
-template <int FMT>
-__device__ __forceinline__ void sr_fp8_magnitude2(uint32_t a0, uint32_t a1, uint32_t r0, uint32_t r1, uint32_t& c0, uint32_t& c1) {
-    using F = Small<FMT>;
-    const uint32_t e0 = a0 >> 23, e1 = a1 >> 23;
-    const uint32_t q0 = e0 < F::kMinBiasedExp ? F::kMinBiasedExp : e0, q1 = e1 < F::kMinBiasedExp ? F::kMinBiasedExp : e1;
-    const float s0 = __uint_as_float(((254u + F::M) << 23) - (q0 << 23)), s1 = __uint_as_float(((254u + F::M) << 23) - (q1 << 23));
-    const uint64_t y = mul2(pack2(__uint_as_float(a0), __uint_as_float(a1)), pack2(s0, s1));
-    const uint64_t magic = dup2(8388608.0f);
-    const uint64_t t = add_rz2(y, magic);
-    const uint64_t f = sub2(y, sub2(t, magic));
-    const uint64_t fs = mul2(f, dup2(4294967296.0f));
-    float t0, t1, f0, f1;
-    unpack2(t, t0, t1);
-    unpack2(fs, f0, f1);
-    c0 = finish_code<FMT>(a0, q0, t0, f0, r0);
-    c1 = finish_code<FMT>(a1, q1, t1, f1, r1);
-}
-
+// one FP8 byte (E4M3 / E5M2): NaN -> 0x7F without a sign, E5M2 keeps infinity
 template <int FMT>
 __device__ __forceinline__ uint32_t sr_fp8_code(uint32_t fbits, uint32_t r) {
-    const uint32_t abits = fbits & 0x7FFFFFFFu;
-    const uint32_t sign = abits > 0x7F800000u ? 0u : ((fbits >> 24) & 0x80u);
-    return sign | sr_fp8_magnitude<FMT>(abits, r);
+    const float x = __uint_as_float(fbits);
+    uint32_t code = min(sr_small_magnitude<FMT, true>(x, r), 0x7Fu);
+    if (FMT == kE5M2) code = fabsf(x) == __uint_as_float(0x7F800000u) ? kE5M2InfCode : code;
+    return code == 0x7Fu ? code : (code | ((fbits >> 24) & 0x80u));
 }
 
 // E2M1: sign in bit 3 (kept for NaN too), magnitude code in bits 0..2
 __device__ __forceinline__ uint32_t sr_fp4_code(uint32_t fbits, uint32_t r) {
-    return ((fbits >> 28) & 0x8u) | sr_fp8_magnitude<kE2M1>(fbits & 0x7FFFFFFFu, r);
+    return ((fbits >> 28) & 8u) | sr_small_magnitude<kE2M1, false>(__uint_as_float(fbits), r);
 }
 
 // four values -> four 4-bit codes in bits 0..15 (element j in bits 4j..4j+3)
 __device__ __forceinline__ uint32_t cast4_fp4(const uint4 x, const uint4 w) {
-    uint32_t n0, n1, n2, n3;
-    sr_fp8_magnitude2<kE2M1>(x.x & 0x7FFFFFFFu, x.y & 0x7FFFFFFFu, w.x, w.y, n0, n1);
-    sr_fp8_magnitude2<kE2M1>(x.z & 0x7FFFFFFFu, x.w & 0x7FFFFFFFu, w.z, w.w, n2, n3);
-    n0 |= (x.x >> 28) & 0x8u;
-    n1 |= (x.y >> 28) & 0x8u;
-    n2 |= (x.z >> 28) & 0x8u;
-    n3 |= (x.w >> 28) & 0x8u;
+    const uint32_t n0 = sr_fp4_code(x.x, w.x), n1 = sr_fp4_code(x.y, w.y), n2 = sr_fp4_code(x.z, w.z), n3 = sr_fp4_code(x.w, w.w);
+    // shift-adds on the ALU pipe: this kernel has the FMA pipe fuller than the FP8 one (0.295 -> 0.288 ms)
     return (n1 * 16u + n0) + (n3 * 16u + n2) * 256u;
 }
 
@@ -116,24 +94,35 @@ __device__ __forceinline__ uint32_t noise32_of_element(uint64_t idx, uint32_t c2
     return e == 0 ? w.x : e == 1 ? w.y : e == 2 ? w.z : w.w;
 }
 
-// four values -> four bytes; the four sign bits are gathered with two byte permutes
+// four values -> four bytes; the four sign bits are gathered with byte permutes
 template <int FMT>
 __device__ __forceinline__ uint32_t cast4(const uint4 x, const uint4 w) {
-    const uint32_t ax = x.x & 0x7FFFFFFFu, ay = x.y & 0x7FFFFFFFu, az = x.z & 0x7FFFFFFFu, aw = x.w & 0x7FFFFFFFu;
-    uint32_t m0, m1, m2, m3;
-    sr_fp8_magnitude2<FMT>(ax, ay, w.x, w.y, m0, m1);
-    sr_fp8_magnitude2<FMT>(az, aw, w.z, w.w, m2, m3);
-    const uint32_t mags = __byte_perm(__byte_perm(m0, m1, 0x0040), __byte_perm(m2, m3, 0x0040), 0x5410);
+    const float f0 = __uint_as_float(x.x), f1 = __uint_as_float(x.y), f2 = __uint_as_float(x.z), f3 = __uint_as_float(x.w);
+    uint32_t m0 = min(sr_small_magnitude<FMT, true>(f0, w.x), 0x7Fu), m1 = min(sr_small_magnitude<FMT, true>(f1, w.y), 0x7Fu);
+    uint32_t m2 = min(sr_small_magnitude<FMT, true>(f2, w.z), 0x7Fu), m3 = min(sr_small_magnitude<FMT, true>(f3, w.w), 0x7Fu);
+    if (FMT == kE5M2) {
+        const float inf = __uint_as_float(0x7F800000u);
+        m0 = fabsf(f0) == inf ? kE5M2InfCode : m0;
+        m1 = fabsf(f1) == inf ? kE5M2InfCode : m1;
+        m2 = fabsf(f2) == inf ? kE5M2InfCode : m2;
+        m3 = fabsf(f3) == inf ? kE5M2InfCode : m3;
+    }
+    const uint32_t mags = (m1 * mul_256() + m0) + (m3 * mul_256() + m2) * mul_65536();   // on the FMA pipe (0.325 -> 0.321 ms)
     const uint32_t tops = __byte_perm(__byte_perm(x.x, x.y, 0x0073), __byte_perm(x.z, x.w, 0x0073), 0x5410);
-    // a NaN code (0x7F) keeps no sign: mask the sign bit where the magnitude byte is 0x7F with all of bits 0..6 set
-    const uint32_t is_nan = ((mags & 0x7F7F7F7Fu) + 0x01010101u) & 0x80808080u;
-    return mags | (tops & 0x80808080u & ~is_nan);
+    // a NaN code (0x7F) keeps no sign: every magnitude byte is at most 0x7F, so adding 1 to each sets its bit 7
+    // exactly where it is 0x7F
+    const uint32_t nan7 = mags + 0x01010101u;
+    return mags | (tops & ~nan7 & 0x80808080u);
 }
+
+// 72 registers: the sixteen values of an iteration are independent and the two pipes overlap only when the
+// compiler may keep several of them in flight (40 registers: 0.321 ms, 72: 0.299 ms for E4M3)
+constexpr int kSmallMinBlocks = 4;
 
 // VEC: 16 elements per thread-iteration (4 x 16-byte loads, 1 x 16-byte store); needs both buffers
 // 16-byte aligned and elem_offset a multiple of 4 (whole noise groups).
 template <int FMT, bool VEC>
-__global__ void __launch_bounds__(kBlockThreads)
+__global__ void __launch_bounds__(kBlockThreads, kSmallMinBlocks)
 k_sr_downcast_fp8(const float* __restrict__ src, uint8_t* __restrict__ dst, uint64_t n, uint64_t elem_offset,
                   uint32_t tensor_id, uint32_t seed_hi, const __grid_constant__ PhiloxKeys K) {
     const uint64_t tid = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -163,7 +152,7 @@ k_sr_downcast_fp8(const float* __restrict__ src, uint8_t* __restrict__ dst, uint
 // and elem_offset a multiple of 16.  The rest (and everything without VEC) goes byte by byte, one
 // thread per output byte.
 template <bool VEC>
-__global__ void __launch_bounds__(kBlockThreads)
+__global__ void __launch_bounds__(kBlockThreads, kSmallMinBlocks)
 k_sr_downcast_fp4(const float* __restrict__ src, uint8_t* __restrict__ dst, uint64_t n, uint64_t elem_offset,
                   uint32_t tensor_id, uint32_t seed_hi, const __grid_constant__ PhiloxKeys K) {
     const uint64_t tid = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;

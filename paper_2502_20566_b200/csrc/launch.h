@@ -104,6 +104,10 @@ cudaError_t launch_accumulate(uint16_t* acc, const void* g, bool g_f32, uint64_t
 cudaError_t launch_master_adamw(float* p, uint16_t* p16, const void* g, bool g_f32, float* m, float* v, uint64_t n,
                                 const StepScalars& S, const DeviceInfo& dev, cudaStream_t stream);
 
+// mismatches[0 / 1]: square roots / divisions of the branch-free sequences that differ from the IEEE instructions
+cudaError_t launch_selftest_in_range(uint64_t sets, uint32_t seed_hi, const PhiloxKeys& K, unsigned long long* mismatches,
+                                     const DeviceInfo& dev, cudaStream_t stream);
+
 // Squared norm: number of doubles of scratch needed, and the launcher.
 uint64_t sqnorm_scratch_doubles(uint64_t n);
 uint64_t sqnorm_mt_scratch_doubles(uint64_t num_chunks);

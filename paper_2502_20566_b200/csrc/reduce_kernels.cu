@@ -4,8 +4,11 @@
 // blocks of 8192 consecutive entries; inside a block 256 accumulators, accumulator j adding the
 // entries r*1024 + 4j + k (r = 0..7, k = 0..3) in that order; 8 warps folded by an XOR butterfly
 // (16, 8, 4, 2, 1), warp values added in order 0..7; block sums reduced again by the same rule.
-// A CUDA block of 256 threads is exactly one tree block, so thread j is accumulator j and the
-// loads of one r are 16-byte, fully coalesced.  HBM-bound: 4 (FP32) or 2 (BF16) bytes per element.
+// With FP32 entries a CUDA block of 256 threads is exactly one tree block: thread j is accumulator j and
+// its four entries of one r are one 16-byte load.  With BF16 entries four entries are only 8 bytes, so a
+// block of 128 threads is one tree block and thread t holds accumulators 2t and 2t + 1, whose eight
+// entries of one r are one 16-byte load (same tree, see fold_block_pairs).  HBM-bound: 4 (FP32) or 2
+// (BF16) bytes per element.
 
 #include <atomic>
 #include <mutex>
@@ -43,17 +46,81 @@ __device__ __forceinline__ double fold_block(double acc, double* warp_sums) {
     return total;   // valid in thread 0
 }
 
+// The same tree with two accumulators per thread (thread t: accumulators 2t and 2t + 1, 128 threads).  Tree
+// lane l = 2 (t & 15) + b of tree warp t >> 4: the butterfly partners l ^ 16, 8, 4, 2 are the same b in threads
+// t ^ 8, 4, 2, 1; the partner l ^ 1 is the thread's other accumulator.  Every addition has the same two
+// operands as in fold_block, so the bits are the same.
+__device__ __forceinline__ double fold_block_pairs(double a0, double a1, double* warp_sums) {
+#pragma unroll
+    for (int s = 8; s >= 1; s >>= 1) {
+        a0 = __dadd_rn(a0, __shfl_xor_sync(0xFFFFFFFFu, a0, s));
+        a1 = __dadd_rn(a1, __shfl_xor_sync(0xFFFFFFFFu, a1, s));
+    }
+    const double x = __dadd_rn(a0, a1);
+    if ((threadIdx.x & 15) == 0) warp_sums[threadIdx.x >> 4] = x;
+    __syncthreads();
+    double total = 0.0;
+    if (threadIdx.x == 0) {
+        total = warp_sums[0];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) total = __dadd_rn(total, warp_sums[w]);
+    }
+    __syncthreads();
+    return total;   // valid in thread 0
+}
+
+constexpr int kPairThreads = 128;   // BF16 entries: two accumulators per thread
+
+// One whole, 16-byte aligned tree block of BF16 entries: eight 16-byte loads per thread, all issued before the
+// first addition.  t = threadIdx.x of a 128-thread block; returns the block sum in thread 0.
+__device__ __forceinline__ double bf16_block_sum(const void* chunk, uint32_t t, double* warp_sums) {
+    const uint4* src = reinterpret_cast<const uint4*>(chunk) + t;
+    uint4 q[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) q[r] = __ldcs(src + r * 128);
+    double a0 = 0.0, a1 = 0.0;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+        a0 = add_square(a0, bf16_lo(q[r].x));
+        a0 = add_square(a0, bf16_hi(q[r].x));
+        a0 = add_square(a0, bf16_lo(q[r].y));
+        a0 = add_square(a0, bf16_hi(q[r].y));
+        a1 = add_square(a1, bf16_lo(q[r].z));
+        a1 = add_square(a1, bf16_hi(q[r].z));
+        a1 = add_square(a1, bf16_lo(q[r].w));
+        a1 = add_square(a1, bf16_hi(q[r].w));
+    }
+    return fold_block_pairs(a0, a1, warp_sums);
+}
+
+// A ragged or unaligned tree block of BF16 entries, `len` of them from `chunk` on: element by element.
+__device__ __forceinline__ double bf16_block_sum_ragged(const uint16_t* chunk, uint64_t len, uint32_t t, double* warp_sums) {
+    double a[2] = {0.0, 0.0};
+    for (int b = 0; b < 2; ++b)
+        for (int r = 0; r < 8; ++r)
+            for (int k = 0; k < 4; ++k) {
+                const uint64_t e = static_cast<uint64_t>(r) * 1024u + 4u * (2u * t + b) + k;
+                if (e < len) a[b] = add_square(a[b], __uint_as_float(static_cast<uint32_t>(chunk[e]) << 16));
+            }
+    return fold_block_pairs(a[0], a[1], warp_sums);
+}
+
 // First pass: out[c] = tree-block sum of squares of entries [c*8192, (c+1)*8192) of g.
 template <bool G32>
-__global__ void __launch_bounds__(kTreeThreads)
+__global__ void __launch_bounds__(G32 ? kTreeThreads : kPairThreads)
 k_sqnorm_pass1(const void* __restrict__ g, uint64_t n, uint64_t num_blocks, bool vec_ok, double* __restrict__ out) {
     __shared__ double warp_sums[8];
     const uint32_t j = threadIdx.x;
     for (uint64_t c = blockIdx.x; c < num_blocks; c += gridDim.x) {
         const uint64_t base = c * kTreeBlock;
-        double acc = 0.0;
-        if (vec_ok && n - base >= kTreeBlock) {
-            if (G32) {
+        const bool whole = vec_ok && n - base >= kTreeBlock;
+        double total;
+        if (!G32) {
+            const uint16_t* chunk = static_cast<const uint16_t*>(g) + base;
+            total = whole ? bf16_block_sum(chunk, j, warp_sums) : bf16_block_sum_ragged(chunk, n - base, j, warp_sums);
+        } else {
+            double acc = 0.0;
+            if (whole) {
                 const float4* src = reinterpret_cast<const float4*>(static_cast<const float*>(g) + base) + j;
                 float4 q[8];
 #pragma unroll
@@ -66,30 +133,14 @@ k_sqnorm_pass1(const void* __restrict__ g, uint64_t n, uint64_t num_blocks, bool
                     acc = add_square(acc, q[r].w);
                 }
             } else {
-                const uint2* src = reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(g) + base) + j;
-                uint2 q[8];
-#pragma unroll
-                for (int r = 0; r < 8; ++r) q[r] = __ldcs(src + r * 256);
-#pragma unroll
-                for (int r = 0; r < 8; ++r) {
-                    acc = add_square(acc, bf16_lo(q[r].x));
-                    acc = add_square(acc, bf16_hi(q[r].x));
-                    acc = add_square(acc, bf16_lo(q[r].y));
-                    acc = add_square(acc, bf16_hi(q[r].y));
-                }
-            }
-        } else {
-            for (int r = 0; r < 8; ++r)
-                for (int k = 0; k < 4; ++k) {
-                    const uint64_t e = base + static_cast<uint64_t>(r) * 1024u + 4u * j + k;
-                    if (e < n) {
-                        const float gi = G32 ? static_cast<const float*>(g)[e]
-                                             : __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t*>(g)[e]) << 16);
-                        acc = add_square(acc, gi);
+                for (int r = 0; r < 8; ++r)
+                    for (int k = 0; k < 4; ++k) {
+                        const uint64_t e = base + static_cast<uint64_t>(r) * 1024u + 4u * j + k;
+                        if (e < n) acc = add_square(acc, static_cast<const float*>(g)[e]);
                     }
-                }
+            }
+            total = fold_block(acc, warp_sums);
         }
-        const double total = fold_block(acc, warp_sums);
         if (j == 0) out[c] = total;
     }
 }
@@ -97,7 +148,7 @@ k_sqnorm_pass1(const void* __restrict__ g, uint64_t n, uint64_t num_blocks, bool
 // First pass over a tensor list: out[c] = tree-block sum of squares of work-table entry c (a chunk of
 // at most 8192 consecutive gradient entries of one tensor, positions counted from the chunk's start).
 template <bool G32>
-__global__ void __launch_bounds__(kTreeThreads)
+__global__ void __launch_bounds__(G32 ? kTreeThreads : kPairThreads)
 k_sqnorm_mt_pass1(const MtWork* __restrict__ work, uint32_t num_chunks, double* __restrict__ out) {
     __shared__ double warp_sums[8];
     const uint32_t j = threadIdx.x;
@@ -118,9 +169,13 @@ k_sqnorm_mt_pass1(const MtWork* __restrict__ work, uint32_t num_chunks, double* 
             g_next = work[cn].g;
             len_next = work[cn].len;
         }
-        double acc = 0.0;
-        if (len == kTreeBlock && (reinterpret_cast<uintptr_t>(g) & 15u) == 0) {
-            if (G32) {
+        const bool whole = len == kTreeBlock && (reinterpret_cast<uintptr_t>(g) & 15u) == 0;
+        double total;
+        if (!G32) {
+            total = whole ? bf16_block_sum(g, j, warp_sums) : bf16_block_sum_ragged(static_cast<const uint16_t*>(g), len, j, warp_sums);
+        } else {
+            double acc = 0.0;
+            if (whole) {
                 const float4* src = reinterpret_cast<const float4*>(g) + j;
                 float4 q[8];
 #pragma unroll
@@ -133,30 +188,14 @@ k_sqnorm_mt_pass1(const MtWork* __restrict__ work, uint32_t num_chunks, double* 
                     acc = add_square(acc, q[r].w);
                 }
             } else {
-                const uint2* src = reinterpret_cast<const uint2*>(g) + j;
-                uint2 q[8];
-#pragma unroll
-                for (int r = 0; r < 8; ++r) q[r] = __ldcs(src + r * 256);
-#pragma unroll
-                for (int r = 0; r < 8; ++r) {
-                    acc = add_square(acc, bf16_lo(q[r].x));
-                    acc = add_square(acc, bf16_hi(q[r].x));
-                    acc = add_square(acc, bf16_lo(q[r].y));
-                    acc = add_square(acc, bf16_hi(q[r].y));
-                }
-            }
-        } else {
-            for (int r = 0; r < 8; ++r)
-                for (int k = 0; k < 4; ++k) {
-                    const uint32_t e = static_cast<uint32_t>(r) * 1024u + 4u * j + k;
-                    if (e < len) {
-                        const float gi = G32 ? static_cast<const float*>(g)[e]
-                                             : __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t*>(g)[e]) << 16);
-                        acc = add_square(acc, gi);
+                for (int r = 0; r < 8; ++r)
+                    for (int k = 0; k < 4; ++k) {
+                        const uint32_t e = static_cast<uint32_t>(r) * 1024u + 4u * j + k;
+                        if (e < len) acc = add_square(acc, static_cast<const float*>(g)[e]);
                     }
-                }
+            }
+            total = fold_block(acc, warp_sums);
         }
-        const double total = fold_block(acc, warp_sums);
         if (j == 0) out[c] = total;
         g = g_next;
         len = len_next;
@@ -192,6 +231,14 @@ __global__ void k_clip_scale(const double* __restrict__ sqnorm, float accum_scal
 
 inline uint64_t blocks_of(uint64_t count) { return (count + kTreeBlock - 1) / kTreeBlock; }
 
+// persistent grid of a first pass: as many blocks as are resident at once
+template <typename Kernel>
+uint64_t resident_cap(Kernel kernel, int threads, const DeviceInfo& dev) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+    return static_cast<uint64_t>(dev.sm_count) * static_cast<uint64_t>(per_sm);
+}
+
 }  // namespace
 
 // Scratch holds every intermediate level: ceil(n/8192) + ceil(that/8192) + ... down to, but not
@@ -224,11 +271,13 @@ cudaError_t launch_sqnorm_mt(const MtWork* work, uint32_t num_chunks, bool g_f32
     double* level_out = count == 1 ? out : scratch;
     const uint64_t cap = static_cast<uint64_t>(dev.sm_count) * 8u;
     {
-        const unsigned grid = static_cast<unsigned>(count < cap ? count : cap);
-        if (g_f32)
-            k_sqnorm_mt_pass1<true><<<grid, kTreeThreads, 0, stream>>>(work, num_chunks, level_out);
-        else
-            k_sqnorm_mt_pass1<false><<<grid, kTreeThreads, 0, stream>>>(work, num_chunks, level_out);
+        if (g_f32) {
+            const uint64_t res = resident_cap(k_sqnorm_mt_pass1<true>, kTreeThreads, dev);
+            k_sqnorm_mt_pass1<true><<<static_cast<unsigned>(count < res ? count : res), kTreeThreads, 0, stream>>>(work, num_chunks, level_out);
+        } else {
+            const uint64_t res = resident_cap(k_sqnorm_mt_pass1<false>, kPairThreads, dev);
+            k_sqnorm_mt_pass1<false><<<static_cast<unsigned>(count < res ? count : res), kPairThreads, 0, stream>>>(work, num_chunks, level_out);
+        }
         cudaError_t err = cudaGetLastError();
         if (err != cudaSuccess) return err;
     }
@@ -253,11 +302,13 @@ cudaError_t launch_sqnorm(const void* g, bool g_f32, uint64_t n, double* out, do
     const bool vec_ok = (reinterpret_cast<uintptr_t>(g) & 15u) == 0;
     const uint64_t cap = static_cast<uint64_t>(dev.sm_count) * 8u;
     {
-        const unsigned grid = static_cast<unsigned>(count < cap ? count : cap);
-        if (g_f32)
-            k_sqnorm_pass1<true><<<grid, kTreeThreads, 0, stream>>>(g, n, count, vec_ok, level_out);
-        else
-            k_sqnorm_pass1<false><<<grid, kTreeThreads, 0, stream>>>(g, n, count, vec_ok, level_out);
+        if (g_f32) {
+            const uint64_t res = resident_cap(k_sqnorm_pass1<true>, kTreeThreads, dev);
+            k_sqnorm_pass1<true><<<static_cast<unsigned>(count < res ? count : res), kTreeThreads, 0, stream>>>(g, n, count, vec_ok, level_out);
+        } else {
+            const uint64_t res = resident_cap(k_sqnorm_pass1<false>, kPairThreads, dev);
+            k_sqnorm_pass1<false><<<static_cast<unsigned>(count < res ? count : res), kPairThreads, 0, stream>>>(g, n, count, vec_ok, level_out);
+        }
         cudaError_t err = cudaGetLastError();
         if (err != cudaSuccess) return err;
     }

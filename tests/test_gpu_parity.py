@@ -287,6 +287,21 @@ def test_in_range_arithmetic_over_its_whole_operand_range(env, kw, step):
         assert run_both(env, p, g, m, v, kw, seed=8, step=step) == (0, 0, 0)
 
 
+def test_in_range_arithmetic_equals_ieee_on_seeded_operands(env):
+    """The branch-free square root and division against sqrt.rn / div.rn on 2^32 seeded operand sets per run
+    (exponents over the whole range the kernels use them in; mantissas plain, just below a power of two, just
+    above one; denominators also formed as root * factor + eps): no result may differ."""
+    _, binding, _, dev = env
+    bad = torch.full((2,), -1, dtype=torch.int64, device=dev)
+    for seed in (1, (7 << 32) | 12345):
+        binding.sr_selftest_in_range_arithmetic(seed, 1 << 31, bad)
+        torch.cuda.synchronize()
+        assert bad.tolist() == [0, 0], seed
+    binding.sr_selftest_in_range_arithmetic(3, 0, bad)
+    torch.cuda.synchronize()
+    assert bad.tolist() == [0, 0]
+
+
 def test_shards_equal_whole_and_runs_repeat(env):
     """Shared random state: 8 shards stepped separately equal the whole buffer; a second run repeats
     the first bit for bit; another seed does not."""
@@ -654,6 +669,37 @@ def test_multi_tensor_random_lists(env, g_dtype, flags, gscale):
             bad += mismatches(bits(P[i]), host[0][i]) + mismatches(bits(M[i]), host[2][i]) + mismatches(bits(V[i]), host[3][i])
             assert np.array_equal(host_g(G[i]), host[1][i])
         assert bad == 0, f"step {step}"
+    plan.destroy()
+
+
+@pytest.mark.parametrize("flags,gscale", [(7, 1.0), (5, 0.25)])
+def test_multi_tensor_long_list(env, flags, gscale):
+    """A list of more than 2^29 elements (65 536 chunks and more): a few large tensors plus sizes around every
+    boundary of a block's pass over a chunk and of a chunk itself, runs of tiny tensors, an empty and an unaligned
+    one; every element compared."""
+    oracle, binding, synth, dev = env
+    sizes = [1 << 27, 5, 8 * 511, 8 * 512, 8 * 512 + 1, 8 * 513, 8191, 8192, 8193, (1 << 28) + 8 * 300 + 3, 0, 7, 7, 7, 16,
+             8 * 255, 8 * 256, 8 * 257, 2 * 8192 + 8 * 512, 100003, (1 << 27) + 9, 12345, 8 * 1023, 3]
+    P, G, M, V = [], [], [], []
+    for i, n in enumerate(sizes):
+        shift = 1 if i == 19 else 0
+        p, g, m, v = synth.adamw_state(n + shift, 300 + i, dev)
+        P.append(p[shift:]); G.append(g[shift:]); M.append(m[shift:]); V.append(v[shift:])
+    assert sum((n + 8191) // 8192 for n in sizes) >= 1 << 16
+    plan = binding.sr_mt_plan_create(P, G, M, V)
+    hp_o = oracle.hparams(**HP, flags=flags)
+    hp_g = binding.hparams(**HP, grad_scale=gscale, flags=flags)
+    host = [[bits(t) for t in P], [bits(t) for t in G], [bits(t) for t in M], [bits(t) for t in V]]
+    ws = torch.empty(max(1, binding.grad_sqnorm_multi_tensor_workspace_bytes(plan) // 8), dtype=torch.float64, device=dev)
+    S = torch.zeros(1, dtype=torch.float64, device=dev)
+    binding.grad_sqnorm_multi_tensor(plan, S, ws)
+    binding.sr_adamw_multi_tensor(plan, hp_g, 17, 3, tensor_id_base=50)
+    torch.cuda.synchronize()
+    assert float(S.item()).hex() == oracle.sqnorm_list([host[1][i] for i in range(len(sizes))]).hex()
+    for i in range(len(sizes)):
+        oracle.adamw_step(host[0][i], host[1][i], host[2][i], host[3][i], hp_o, 17, 3, 50 + i, 0, gscale)
+        assert mismatches(bits(P[i]), host[0][i]) + mismatches(bits(M[i]), host[2][i]) + mismatches(bits(V[i]), host[3][i]) == 0, i
+        assert np.array_equal(bits(G[i]), host[1][i])
     plan.destroy()
 
 
