@@ -37,8 +37,9 @@ NOMINAL_HBM_GBS = 7700.0        # data-sheet bandwidth of the HGX B200 (context 
 # DRAM bytes (read + write) of one launch of the headline kernel, from a profiler capture of the SAME kernel
 # build and launch shape on a smaller case: (dram bytes read + written, elements of that case).  The traffic of
 # a streaming kernel grows in proportion to the element count, so the full-size figure is bytes / elements * n.
-# None whenever the kernel has changed since the capture was taken.
-NCU_TRAFFIC_CAPTURE = None
+# None whenever the kernel has changed since the capture was taken.  Current values: k_sr_adamw_flat_fast in its long
+# launch shape (256 x 2 blocks, 3 stages) on 2^29 elements, dram__bytes_read.sum + dram__bytes_write.sum of one launch.
+NCU_TRAFFIC_CAPTURE = (7_458_763_000, 536_870_912)
 
 
 def parse_args():
@@ -414,12 +415,12 @@ def _extras_casts(torch, binding, synth, dev, peak, timed, out, want, elements):
         dst8 = torch.empty(nc, dtype=torch.uint8, device=dev).view(torch.float8_e4m3fn)
         t_8 = timed(lambda: binding.sr_downcast_f32_fp8(src, dst8, seed=7))
         out["sr_downcast_f32_fp8_e4m3"] = {"elements": nc, "ms": t_8, "params_per_s": nc / t_8 * 1e3,
-                                           "gbs": 5 * nc / t_8 / 1e6, "frac": 5 * nc / t_8 / 1e6 / peak}
+                                           "gbs": 5 * nc / t_8 / 1e6, "frac": 5 * nc / t_8 / 1e6 / peak, "bound": "alu"}
     if want("cast_fp4"):
         dst4 = torch.empty(nc // 2, dtype=torch.uint8, device=dev)
         t_4 = timed(lambda: binding.sr_downcast_f32_fp4(src, dst4, seed=7))
         out["sr_downcast_f32_fp4_e2m1"] = {"elements": nc, "ms": t_4, "params_per_s": nc / t_4 * 1e3,
-                                           "gbs": 4.5 * nc / t_4 / 1e6, "frac": 4.5 * nc / t_4 / 1e6 / peak}
+                                           "gbs": 4.5 * nc / t_4 / 1e6, "frac": 4.5 * nc / t_4 / 1e6 / peak, "bound": "alu"}
 
 
 def _extras_accumulate(torch, binding, synth, dev, peak, timed, out, elements):
