@@ -696,7 +696,8 @@ def run_sharded(args):
     os.environ.setdefault("MASTER_PORT", "29555")
     # the communicator's own account of what it uses (rings / trees / NVLS), kept out of stdout
     nccl_log = os.path.join(tempfile.gettempdir(), f"sradamw_nccl_rank{rank}.log")
-    os.environ.setdefault("NCCL_DEBUG", "INFO")
+    if os.environ.get("NCCL_DEBUG", "VERSION").upper() in ("VERSION", "WARN"):      # the box presets VERSION
+        os.environ["NCCL_DEBUG"] = "INFO"
     os.environ.setdefault("NCCL_DEBUG_FILE", nccl_log)
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
