@@ -142,7 +142,8 @@ __device__ __forceinline__ uint4 straddle_select(const uint4 a, const uint4 b) {
 
 // own: this lane's call (the group its vector ends in); head: where the row's head call lies in shared memory.
 // Lanes 1..31 take the words of the lane below; lane 0 loads the head call over them (one predicated 16-byte
-// load instead of a select per word: 832M-element step 2.11 -> 2.08 ms, accumulation 0.86 -> 0.84 ms).  Every lane of the warp must call this (full-mask shuffles).
+// load instead of a select per word: 832M-element step 2.11 -> 2.08 ms, accumulation 0.86 -> 0.84 ms).
+// Every lane of the warp must call this (full-mask shuffles).
 template <int R>
 __device__ __forceinline__ uint4 chain_words(const uint4 own, const uint4* head, uint32_t lane) {
     constexpr int k = R >> 1;   // first word of the starting group that the vector uses
