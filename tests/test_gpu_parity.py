@@ -503,15 +503,18 @@ def test_sqnorm_bit_exact(env, n, g_dtype):
     assert float(out.item()).hex() == oracle.sqnorm(host_g(g)).hex()
 
 
-def test_sqnorm_unaligned(env):
+@pytest.mark.parametrize("g_dtype", [torch.float32, torch.bfloat16])
+def test_sqnorm_unaligned(env, g_dtype):
+    """A buffer that starts one element past a 16-byte boundary: every tree block goes element by element."""
     oracle, binding, synth, dev = env
-    g = torch.empty(30000, dtype=torch.float32, device=dev)
-    synth.fill_state(g, synth.ROLE_G, 18)
+    g = torch.empty(30000, dtype=g_dtype, device=dev)
+    synth.fill_state(g, synth.ROLE_G, 18, outlier_fraction=0.01)
     g = g[1:]
     ws = torch.empty(16, dtype=torch.float64, device=dev)
     out = torch.zeros(1, dtype=torch.float64, device=dev)
     binding.grad_sqnorm(g, out, ws)
-    assert float(out.item()).hex() == oracle.sqnorm(g.cpu().numpy().copy()).hex()
+    torch.cuda.synchronize()
+    assert float(out.item()).hex() == oracle.sqnorm(host_g(g)).hex()
 
 
 def test_clip_scale_bit_exact(env):
