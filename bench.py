@@ -207,14 +207,16 @@ EXTRA_CASES = ("shard_fp32_grads", "fp32_master_recipe", "tensor_list", "tensor_
 
 
 def time_extras(torch, binding, synth, dev, peak, only=None, elements=0, reps=10, warmup=3):
-    """The other calls of the library, each timed alone (CUDA events, 3 warm-ups + 10 launches) on its
-    own workload; bytes are the algorithmic ones.  Reported beside the headline, not part of it.
+    """The other calls of the library, each timed alone (half a second of idle, then CUDA events around
+    3 warm-ups + 10 launches) on its own workload; bytes are the algorithmic ones.  Reported beside the headline, not part of it.
     `only` names one case of EXTRA_CASES (the others are skipped) and `elements` shrinks its buffers:
     the small single-kernel runs that profiler captures are taken on."""
     stream = torch.cuda.current_stream()
     want = lambda *cases: only is None or only in cases
 
     def timed(fn, reps=reps):
+        torch.cuda.synchronize()
+        time.sleep(0.5)          # every case starts from an idle GPU, like the headline's first timed region
         for _ in range(warmup):
             fn()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
