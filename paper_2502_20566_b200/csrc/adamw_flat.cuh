@@ -47,8 +47,8 @@ k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n
 // index of the launch has the same (index >> 33) = c1.  Same persistent grid.  STAGED = true: each
 // thread keeps its next vectors in flight -- while vector k is computed out of shared memory, the
 // asynchronous copies of vectors k + T, ... are already under way (kFlatStages slots per thread and
-// array).  SHAPE 0: direct loads into registers, kBlockThreads x kMinBlocksPerSM; 1: staged, same
-// block shape, kShortStages; 2: staged, kFlatStagedThreads x kFlatStagedMinBlocks, kFlatStages.
+// array).  SHAPE 0: direct loads into registers, kBlockThreads x kMinBlocksPerSM (FP32 gradients); 2: staged,
+// kFlatStagedThreads x kFlatStagedMinBlocks, kFlatStages (BF16 gradients, every launch length).
 template <bool G32, uint32_t FLAGS, int VAR, int SHAPE>
 __global__ void __launch_bounds__(SHAPE == 2 ? kFlatStagedThreads : kBlockThreads,
                                   SHAPE == 2 ? kFlatStagedMinBlocks : (VAR & 4) ? kStraddleMinBlocks : kMinBlocksPerSM)
@@ -58,14 +58,14 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
     constexpr int kArrays = G32 ? 5 : 4;   // x, m, v and one or two 16-byte pieces of g
     constexpr bool STAGED = SHAPE != 0;
     constexpr int kThreads = SHAPE == 2 ? kFlatStagedThreads : kBlockThreads;
-    constexpr int kStages = SHAPE == 2 ? kFlatStages : kShortStages;
-    // The long shape's staging fills the 48 KB of static shared memory; where it also needs the table of head
-    // calls (straddling vectors), both live in dynamic shared memory that the launcher sizes.
-    constexpr bool kDynamic = SHAPE == 2 && (VAR & 4) != 0;
+    static_assert(SHAPE == 0 || SHAPE == 2, "direct or staged");
+    constexpr int kStages = kFlatStages;
+    // The staging (and, with straddling vectors, the table of head calls) is more than the 48 KB a kernel gets
+    // without asking: it lives in dynamic shared memory that the launcher sizes.
+    constexpr bool kDynamic = STAGED;
     constexpr int kStageEntries = STAGED ? kStages * kArrays * kThreads : 1;
     extern __shared__ uint4 dynamic_smem[];
-    __shared__ uint4 stage_static[kDynamic ? 1 : kStageEntries];
-    uint4* const stage = kDynamic ? dynamic_smem : stage_static;
+    uint4* const stage = dynamic_smem;
     const float gscale = S.gscale_dev ? __ldg(S.gscale_dev) : S.gscale;
     const uint64_t tid = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
@@ -248,30 +248,22 @@ cudaError_t launch_flat_mode(uint16_t* p, const void* g, uint16_t* m, uint16_t* 
         constexpr bool kStaged = G32 ? (SR_STAGE_F32 != 0) : (SR_STAGE_BF16 != 0);
         const uint32_t c1 = static_cast<uint32_t>(elem_offset >> 33);
         constexpr int kVar = (MODE == 3 ? 1 : 0) | (EPS_IN ? 2 : 0) | (STRADDLE ? 4 : 0);
-        bool launched = false;
         if constexpr (kStaged) {
-            if (n >= kLongLaunchElems) {
-                auto k = k_sr_adamw_flat_fast<G32, FLAGS, kVar, 2>;
-                size_t dynamic = 0;
-                if (STRADDLE) {
-                    // staging + one table of head calls per warp: above the 48 KB a kernel gets without asking
-                    dynamic = sizeof(uint4) * (kFlatStages * (G32 ? 5 : 4) * kFlatStagedThreads +
-                                               (kFlatStagedThreads / 32) * RowChain<FLAGS & 7u, true>::kTableEntries);
-                    static std::atomic<int> prepared[kMaxDevices] = {};      // per kernel instantiation and device
-                    if (!prepared[dev.index].load(std::memory_order_acquire)) {
-                        const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                                   static_cast<int>(dynamic));
-                        if (e != cudaSuccess) return e;
-                        prepared[dev.index].store(1, std::memory_order_release);
-                    }
-                }
-                k<<<grid_for(k, items, dev, kFlatStagedThreads, dynamic), kFlatStagedThreads, dynamic, stream>>>(
-                    p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
-                launched = true;
+            auto k = k_sr_adamw_flat_fast<G32, FLAGS, kVar, 2>;
+            // staging, plus one table of head calls per warp where vectors straddle noise groups: more than the 48 KB a
+            // kernel gets without asking
+            const size_t dynamic = sizeof(uint4) * (kFlatStages * (G32 ? 5 : 4) * kFlatStagedThreads +
+                                                    (STRADDLE ? (kFlatStagedThreads / 32) * RowChain<FLAGS & 7u, true>::kTableEntries : 0));
+            static std::atomic<int> prepared[kMaxDevices] = {};      // per kernel instantiation and device
+            if (!prepared[dev.index].load(std::memory_order_acquire)) {
+                const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(dynamic));
+                if (e != cudaSuccess) return e;
+                prepared[dev.index].store(1, std::memory_order_release);
             }
-        }
-        if (!launched) {
-            auto k = k_sr_adamw_flat_fast<G32, FLAGS, kVar, kStaged ? 1 : 0>;
+            k<<<grid_for(k, items, dev, kFlatStagedThreads, dynamic), kFlatStagedThreads, dynamic, stream>>>(
+                p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
+        } else {
+            auto k = k_sr_adamw_flat_fast<G32, FLAGS, kVar, 0>;
             k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
         }
     } else {

@@ -27,13 +27,16 @@ constexpr uint32_t kMtChunkElems = 8192;   // multiple of 8; never crosses a mul
 // 2..6 stages on the real kernels).  Every kernel's arithmetic needs about 96 registers; tighter
 // budgets cost more in instruction scheduling than they gain in occupancy.
 //  - kernels that load straight into registers: 128 threads, >= 5 blocks/SM (640 threads/SM);
-//  - the staged flat kernel has two shapes.  Long launches (>= 2^29 elements, milliseconds and more,
-//    which run into the board's power cap): 256 threads, 2 blocks/SM, 3 vectors per thread in
-//    flight or in use (48 KB of shared memory per block) -- with the memory latency covered by the
-//    staging, fewer resident warps ran faster under the cap (90% vs 86% of the copy peak at 6.7B).
-//    Shorter launches, which finish before the cap bites: 128 x 5 with 2 stages.  Same GPU, short vs
-//    long shape: 2^26 elements 0.155 vs 0.159 ms, 2^28 0.623 vs 0.641, 355M 0.827 vs 0.817-0.842,
-//    832M 1.95-2.05 vs 1.93-1.95: the long shape takes over between 2^28 and 2^30;
+//  - the staged flat kernel (BF16 gradients): ONE block of 384 threads per SM, 3 vectors per thread in flight or
+//    in use (72 KB of dynamic shared memory).  With the memory latency covered by the staging, few resident
+//    warps run fastest, at every launch length.  6.7B elements, two GPUs, first 20 launches / 3 s sustained:
+//    384 x 1 x 3 stages 15.56-15.60 / 16.13-16.18 ms, 512 x 1 x 2 the same, 256 x 2 x 3 (the shape before)
+//    15.84-15.90 / 16.24-16.27, 384 x 1 x 4 15.72-15.76 / 16.14, 512 x 1 x 3 15.84-15.95 / 16.14-16.17,
+//    256 x 2 x 4 and x 5 as x 3, 192 x 2 x 3 16.0 / 16.55, 384 x 1 x 2 16.35 / 16.9, 320 x 1 x 3 17.2 / 17.9, 448 x 1 x 3
+//    16.7 / 16.7, 256 x 3 x 4 16.8 / 17.5 (the irregular ones: the grid's stride in memory matters as well).
+//    Against 128 x 5 x 2 stages, the shape short launches used to take, same GPU: 2^23 elements 0.0205 vs
+//    0.0225 ms, 2^26 0.150 vs 0.158, 2^28 0.594 vs 0.628, 355M 0.785 vs 0.834, 832M 1.86 vs 1.96, 2^31 4.87 vs 5.10;
+//    equal below 2^22 elements (launch latency);
 //  - the staged multi-tensor kernel keeps 128 x 5 with 2 stages.
 #ifndef SR_BLOCK_THREADS
 #define SR_BLOCK_THREADS 128
@@ -42,10 +45,10 @@ constexpr uint32_t kMtChunkElems = 8192;   // multiple of 8; never crosses a mul
 #define SR_MIN_BLOCKS_PER_SM 5
 #endif
 #ifndef SR_FLAT_STAGED_THREADS
-#define SR_FLAT_STAGED_THREADS 256
+#define SR_FLAT_STAGED_THREADS 384
 #endif
 #ifndef SR_FLAT_STAGED_MIN_BLOCKS
-#define SR_FLAT_STAGED_MIN_BLOCKS 2
+#define SR_FLAT_STAGED_MIN_BLOCKS 1
 #endif
 #ifndef SR_FLAT_STAGES
 #define SR_FLAT_STAGES 3
@@ -53,18 +56,13 @@ constexpr uint32_t kMtChunkElems = 8192;   // multiple of 8; never crosses a mul
 #ifndef SR_STRADDLE_MIN_BLOCKS
 #define SR_STRADDLE_MIN_BLOCKS 5
 #endif
-constexpr int kStraddleMinBlocks = SR_STRADDLE_MIN_BLOCKS;   // flat step at offsets that are not multiples of 8
+constexpr int kStraddleMinBlocks = SR_STRADDLE_MIN_BLOCKS;   // direct-load flat step at offsets that are not multiples of 8
 constexpr int kBlockThreads = SR_BLOCK_THREADS;
 constexpr int kMinBlocksPerSM = SR_MIN_BLOCKS_PER_SM;
 constexpr int kFlatStagedThreads = SR_FLAT_STAGED_THREADS;
 constexpr int kFlatStagedMinBlocks = SR_FLAT_STAGED_MIN_BLOCKS;
 constexpr int kFlatStages = SR_FLAT_STAGES;
 constexpr int kMtStages = 2;
-#ifndef SR_SHORT_STAGES
-#define SR_SHORT_STAGES 2
-#endif
-constexpr int kShortStages = SR_SHORT_STAGES;
-constexpr uint64_t kLongLaunchElems = static_cast<uint64_t>(1) << 29;
 
 constexpr int kMaxDevices = 64;
 struct DeviceInfo {
