@@ -47,17 +47,17 @@ k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n
 // index of the launch has the same (index >> 33) = c1.  Same persistent grid.  STAGED = true: each
 // thread keeps its next vectors in flight -- while vector k is computed out of shared memory, the
 // asynchronous copies of vectors k + T, ... are already under way (kFlatStages slots per thread and
-// array).  SHAPE 0: direct loads into registers, kBlockThreads x kMinBlocksPerSM (FP32 gradients); 2: staged,
+// array).  SHAPE 0: direct loads into registers, kFlatDirectThreads x kFlatDirectMinBlocks (FP32 gradients); 2: staged,
 // kFlatStagedThreads x kFlatStagedMinBlocks, kFlatStages (BF16 gradients, every launch length).
 template <bool G32, uint32_t FLAGS, int VAR, int SHAPE>
-__global__ void __launch_bounds__(SHAPE == 2 ? kFlatStagedThreads : kBlockThreads,
-                                  SHAPE == 2 ? kFlatStagedMinBlocks : (VAR & 4) ? kStraddleMinBlocks : kMinBlocksPerSM)
+__global__ void __launch_bounds__(SHAPE == 2 ? kFlatStagedThreads : kFlatDirectThreads,
+                                  SHAPE == 2 ? kFlatStagedMinBlocks : kFlatDirectMinBlocks)
 k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset,
                      uint32_t c1, uint32_t tensor_id, uint32_t seed_hi, const __grid_constant__ PhiloxKeys K,
                      const __grid_constant__ StepScalars S) {
     constexpr int kArrays = G32 ? 5 : 4;   // x, m, v and one or two 16-byte pieces of g
     constexpr bool STAGED = SHAPE != 0;
-    constexpr int kThreads = SHAPE == 2 ? kFlatStagedThreads : kBlockThreads;
+    constexpr int kThreads = SHAPE == 2 ? kFlatStagedThreads : kFlatDirectThreads;
     static_assert(SHAPE == 0 || SHAPE == 2, "direct or staged");
     constexpr int kStages = kFlatStages;
     // The staging (and, with straddling vectors, the table of head calls) is more than the 48 KB a kernel gets
@@ -264,7 +264,8 @@ cudaError_t launch_flat_mode(uint16_t* p, const void* g, uint16_t* m, uint16_t* 
                 p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
         } else {
             auto k = k_sr_adamw_flat_fast<G32, FLAGS, kVar, 0>;
-            k<<<grid_for(k, items, dev), kBlockThreads, 0, stream>>>(p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
+            k<<<grid_for(k, items, dev, kFlatDirectThreads), kFlatDirectThreads, 0, stream>>>(p, g, m, v, n, elem_offset, c1, tensor_id,
+                                                                                                 seed_hi, K, S);
         }
     } else {
         auto k = k_sr_adamw_flat<G32, FLAGS, (MODE < 2 || MODE == 4 ? MODE : 0)>;

@@ -53,10 +53,10 @@ constexpr uint32_t kMtChunkElems = 8192;   // multiple of 8; never crosses a mul
 #ifndef SR_FLAT_STAGES
 #define SR_FLAT_STAGES 3
 #endif
-#ifndef SR_STRADDLE_MIN_BLOCKS
-#define SR_STRADDLE_MIN_BLOCKS 5
-#endif
-constexpr int kStraddleMinBlocks = SR_STRADDLE_MIN_BLOCKS;   // direct-load flat step at offsets that are not multiples of 8
+// the direct-load flat step (FP32 gradients): 832M elements, same GPU: 256 x 2 2.20 ms, 128 x 4 2.21, 128 x 5 2.26,
+// 384 x 1 2.39, 128 x 3 2.40; staged like the BF16 kernel (five pieces per vector) 2.58-2.60
+constexpr int kFlatDirectThreads = 256;
+constexpr int kFlatDirectMinBlocks = 2;
 constexpr int kBlockThreads = SR_BLOCK_THREADS;
 constexpr int kMinBlocksPerSM = SR_MIN_BLOCKS_PER_SM;
 constexpr int kFlatStagedThreads = SR_FLAT_STAGED_THREADS;
