@@ -37,9 +37,9 @@ NOMINAL_HBM_GBS = 7700.0        # data-sheet bandwidth of the HGX B200 (context 
 # DRAM bytes (read + write) of one launch of the headline kernel, from a profiler capture of the SAME kernel
 # build and launch shape on a smaller case: (dram bytes read + written, elements of that case).  The traffic of
 # a streaming kernel grows in proportion to the element count, so the full-size figure is bytes / elements * n.
-# None whenever the kernel has changed since the capture was taken.  Current values: k_sr_adamw_flat_fast in its long
-# launch shape (256 x 2 blocks, 3 stages) on 2^29 elements, dram__bytes_read.sum + dram__bytes_write.sum of one launch.
-NCU_TRAFFIC_CAPTURE = (7_458_763_000, 536_870_912)
+# None whenever the kernel has changed since the capture was taken.  Current values: k_sr_adamw_flat_fast (BF16
+# gradients, 384 x 1 blocks, 3 stages) on 2^29 elements, dram__bytes_read.sum + dram__bytes_write.sum of one launch.
+NCU_TRAFFIC_CAPTURE = (7_459_395_000, 536_870_912)
 
 
 def parse_args():
