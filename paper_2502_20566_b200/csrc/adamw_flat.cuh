@@ -50,16 +50,19 @@ k_sr_adamw_flat(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n
 // array).  SHAPE 0: direct loads into registers, kFlatDirectThreads x kFlatDirectMinBlocks (FP32 gradients); 2: staged,
 // kFlatStagedThreads x kFlatStagedMinBlocks, kFlatStages (BF16 gradients, every launch length).
 template <bool G32, uint32_t FLAGS, int VAR, int SHAPE>
-__global__ void __launch_bounds__(SHAPE == 2 ? kFlatStagedThreads : kFlatDirectThreads,
+__global__ void __launch_bounds__(SHAPE == 2 ? (G32 ? kFlatStagedThreadsF32 : kFlatStagedThreads) : kFlatDirectThreads,
                                   SHAPE == 2 ? kFlatStagedMinBlocks : kFlatDirectMinBlocks)
 k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint64_t n, uint64_t elem_offset,
                      uint32_t c1, uint32_t tensor_id, uint32_t seed_hi, const __grid_constant__ PhiloxKeys K,
                      const __grid_constant__ StepScalars S) {
-    constexpr int kArrays = G32 ? 5 : 4;   // x, m, v and one or two 16-byte pieces of g
+    // FP32 gradients: x, m, v are staged, the gradient's two 16-byte pieces are loaded straight into a register double
+    // buffer (five staged pieces per vector measured slower than no staging at all, three staged + two direct faster)
+    constexpr bool kHybrid = G32 && (VAR & 4) == 0;
+    constexpr int kArrays = kHybrid ? 3 : G32 ? 5 : 4;   // staged 16-byte pieces per vector
     constexpr bool STAGED = SHAPE != 0;
-    constexpr int kThreads = SHAPE == 2 ? kFlatStagedThreads : kFlatDirectThreads;
+    constexpr int kThreads = SHAPE == 2 ? (G32 ? kFlatStagedThreadsF32 : kFlatStagedThreads) : kFlatDirectThreads;
     static_assert(SHAPE == 0 || SHAPE == 2, "direct or staged");
-    constexpr int kStages = kFlatStages;
+    constexpr int kStages = G32 ? kFlatStagesF32 : kFlatStages;
     // The staging (and, with straddling vectors, the table of head calls) is more than the 48 KB a kernel gets
     // without asking: it lives in dynamic shared memory that the launcher sizes.
     constexpr bool kDynamic = STAGED;
@@ -165,7 +168,8 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
                 async_copy16(slot(s, 0), reinterpret_cast<const uint4*>(p) + vec);
                 async_copy16(slot(s, 1), reinterpret_cast<const uint4*>(m) + vec);
                 async_copy16(slot(s, 2), reinterpret_cast<const uint4*>(v) + vec);
-                if (G32) {
+                if (kHybrid) {
+                } else if (G32) {
                     async_copy16(slot(s, 3), reinterpret_cast<const uint4*>(g) + 2 * vec);
                     async_copy16(slot(s, 4), reinterpret_cast<const uint4*>(g) + 2 * vec + 1);
                 } else {
@@ -177,14 +181,26 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
 #pragma unroll
         for (int s = 0; s < kStages - 1; ++s) issue(tid + s * stride, s);
         int s = 0;
+        uint4 g0 = make_uint4(0, 0, 0, 0), g1 = g0;
+        if (kHybrid && tid < nvec) {
+            g0 = ld16(g, 2 * tid);
+            g1 = ld16(g, 2 * tid + 1);
+        }
         for (uint64_t vec = tid; vec < nvec; vec += stride) {
             int ahead = s + kStages - 1;
             if (ahead >= kStages) ahead -= kStages;
             issue(vec + (kStages - 1) * stride, ahead);
+            uint4 gn0 = g0, gn1 = g1;
+            if (kHybrid && vec + stride < nvec) {
+                gn0 = ld16(g, 2 * (vec + stride));
+                gn1 = ld16(g, 2 * (vec + stride) + 1);
+            }
             async_copy_wait<kStages - 1>();   // this vector's group has landed
             const uint4 pv = *slot(s, 0), mv = *slot(s, 1), vv = *slot(s, 2);
             float ge[8];
-            unpack_grad8<G32>(*slot(s, 3), G32 ? *slot(s, kArrays - 1) : make_uint4(0, 0, 0, 0), ge);
+            if (kHybrid) unpack_grad8<true>(g0, g1, ge);
+            else unpack_grad8<G32>(*slot(s, kHybrid ? 0 : 3), G32 ? *slot(s, kArrays - 1) : make_uint4(0, 0, 0, 0), ge);
+            g0 = gn0; g1 = gn1;
             step_vec8_fast_loaded<G32, FLAGS, VAR>(p, g, m, v, vec, elem_offset + (vec << 3), pv, mv, vv, ge, c1,
                                                      tensor_id, seed_hi, gscale, K, S);
             if (++s == kStages) s = 0;
@@ -229,13 +245,14 @@ k_sr_adamw_flat_fast(uint16_t* p, const void* g, uint16_t* m, uint16_t* v, uint6
 }
 
 // Which gradient types use the staged variant.  Measured on B200 (same GPU, back to back): BF16
-// gradients 85.3% staged vs 83.8% direct of the copy peak at 6.7B; FP32 gradients (five 16-byte
-// pieces per vector) 77.7% staged vs 93.2% direct at 832M elements, so they stay direct.
+// gradients 85.3% staged vs 83.8% direct of the copy peak at 6.7B (in the block shapes of that time); FP32
+// gradients with all five 16-byte pieces of a vector staged 77.7% vs 93.2% direct at 832M elements, with x, m, v
+// staged and the gradient loaded directly 98.7%.
 #ifndef SR_STAGE_BF16
 #define SR_STAGE_BF16 1
 #endif
 #ifndef SR_STAGE_F32
-#define SR_STAGE_F32 0
+#define SR_STAGE_F32 1
 #endif
 
 template <bool G32, uint32_t FLAGS, int MODE, bool EPS_IN = false, bool STRADDLE = false>
@@ -245,22 +262,23 @@ cudaError_t launch_flat_mode(uint16_t* p, const void* g, uint16_t* m, uint16_t* 
     // + 8: enough threads for the ragged tail
     const uint64_t items = MODE == 0 ? n : (n >> 3) + 8;
     if (MODE == 2 || MODE == 3) {
-        constexpr bool kStaged = G32 ? (SR_STAGE_F32 != 0) : (SR_STAGE_BF16 != 0);
+        constexpr bool kStaged = G32 ? (SR_STAGE_F32 != 0 && !STRADDLE) : (SR_STAGE_BF16 != 0);
         const uint32_t c1 = static_cast<uint32_t>(elem_offset >> 33);
         constexpr int kVar = (MODE == 3 ? 1 : 0) | (EPS_IN ? 2 : 0) | (STRADDLE ? 4 : 0);
         if constexpr (kStaged) {
             auto k = k_sr_adamw_flat_fast<G32, FLAGS, kVar, 2>;
             // staging, plus one table of head calls per warp where vectors straddle noise groups: more than the 48 KB a
             // kernel gets without asking
-            const size_t dynamic = sizeof(uint4) * (kFlatStages * (G32 ? 5 : 4) * kFlatStagedThreads +
-                                                    (STRADDLE ? (kFlatStagedThreads / 32) * RowChain<FLAGS & 7u, true>::kTableEntries : 0));
+            constexpr int kThreads = G32 ? kFlatStagedThreadsF32 : kFlatStagedThreads;
+            const size_t dynamic = sizeof(uint4) * ((G32 ? kFlatStagesF32 * 3 : kFlatStages * 4) * kThreads +
+                                                    (STRADDLE ? (kThreads / 32) * RowChain<FLAGS & 7u, true>::kTableEntries : 0));
             static std::atomic<int> prepared[kMaxDevices] = {};      // per kernel instantiation and device
             if (!prepared[dev.index].load(std::memory_order_acquire)) {
                 const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(dynamic));
                 if (e != cudaSuccess) return e;
                 prepared[dev.index].store(1, std::memory_order_release);
             }
-            k<<<grid_for(k, items, dev, kFlatStagedThreads, dynamic), kFlatStagedThreads, dynamic, stream>>>(
+            k<<<grid_for(k, items, dev, kThreads, dynamic), kThreads, dynamic, stream>>>(
                 p, g, m, v, n, elem_offset, c1, tensor_id, seed_hi, K, S);
         } else {
             auto k = k_sr_adamw_flat_fast<G32, FLAGS, kVar, 0>;

@@ -53,10 +53,15 @@ constexpr uint32_t kMtChunkElems = 8192;   // multiple of 8; never crosses a mul
 #ifndef SR_FLAT_STAGES
 #define SR_FLAT_STAGES 3
 #endif
-// the direct-load flat step (FP32 gradients): 832M elements, same GPU: 256 x 2 2.20 ms, 128 x 4 2.21, 128 x 5 2.26,
-// 384 x 1 2.39, 128 x 3 2.40; staged like the BF16 kernel (five pieces per vector) 2.58-2.60
+// the flat step with FP32 gradients, 832M elements, same GPU.  All five 16-byte pieces of a vector loaded into a
+// register double buffer: 256 x 2 2.20 ms, 128 x 4 2.21, 128 x 5 2.26, 384 x 1 2.39, 128 x 3 2.40 (bound by load
+// latency at 128 registers); all five staged like the BF16 kernel: 2.58-2.60; x, m, v staged and the gradient in the
+// register double buffer: 512 x 1 x 2 stages 2.06 ms, 512 x 1 x 3 2.06, 256 x 2 x 3 2.07, 384 x 1 x 3 2.08.  The direct
+// shape remains for offsets that are not multiples of 8.
 constexpr int kFlatDirectThreads = 256;
 constexpr int kFlatDirectMinBlocks = 2;
+constexpr int kFlatStagedThreadsF32 = 512;
+constexpr int kFlatStagesF32 = 2;
 constexpr int kBlockThreads = SR_BLOCK_THREADS;
 constexpr int kMinBlocksPerSM = SR_MIN_BLOCKS_PER_SM;
 constexpr int kFlatStagedThreads = SR_FLAT_STAGED_THREADS;
