@@ -4,7 +4,7 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
 One step = one sr_adamw_step call over the whole buffer (6 658 404 352 BF16 elements of x, g, m, v
-resident in HBM; 14 algorithmic bytes per element).  Prints ONE JSON line: parameters updated per
+resident in HBM; 14 algorithmic bytes per element; the call enqueues 25 launches of one kernel).  Prints ONE JSON line: parameters updated per
 second over all ranks, the HBM roofline of the kernel, an end-to-end figure with host-resident
 state, and the CPU oracle timed on the same box.  With N > 1 (torchrun) every rank steps its own
 full replica, as the data-parallel replicas of Algorithm 1 do; there is no collective in the path.
@@ -559,8 +559,8 @@ def run_ours(args):
         torch.cuda.synchronize()
         ts1 = _dt.datetime.now()
         sms = [a.elapsed_time(b) for a, b in sev]
-        sustained = {"launches": reps, "seconds": sev[0][0].elapsed_time(sev[-1][1]) * 1e-3, "launch_ms_avg": sum(sms) / reps,
-                     "launch_ms_last_quarter": sum(sms[-(reps // 4):]) / (reps // 4), "window": (ts0, ts1)}
+        sustained = {"steps": reps, "seconds": sev[0][0].elapsed_time(sev[-1][1]) * 1e-3, "step_ms_avg": sum(sms) / reps,
+                     "step_ms_last_quarter": sum(sms[-(reps // 4):]) / (reps // 4), "window": (ts0, ts1)}
     if sampler is not None:
         sampler.stop()
     clocks = sampler.window(t_begin, t_end) if sampler is not None else None
@@ -613,13 +613,16 @@ def run_ours(args):
         return
 
     peak, peak_src = hbm_peak()
+    # one call = launches_per_step launches of the same kernel back to back (the library cuts a flat call into launches
+    # of 2^28 elements); the events bracket the call, so the per-launch figures below include the gaps between them
+    launches_per_step = binding.sr_adamw_step_launch_count(n, args.elem_offset)
     avg_launch_ms = sum(launch_ms) / len(launch_ms)
     achieved = BYTES_PER_ELEMENT * n / (avg_launch_ms * 1e-3) / 1e9
     gbs = lambda ms: BYTES_PER_ELEMENT * n / (ms * 1e-3) / 1e9
     if sustained is not None:
-        sustained.update(achieved=gbs(sustained["launch_ms_avg"]), frac=gbs(sustained["launch_ms_avg"]) / peak,
-                         achieved_last_quarter=gbs(sustained["launch_ms_last_quarter"]),
-                         frac_last_quarter=gbs(sustained["launch_ms_last_quarter"]) / peak, unit="GB/s")
+        sustained.update(achieved=gbs(sustained["step_ms_avg"]), frac=gbs(sustained["step_ms_avg"]) / peak,
+                         achieved_last_quarter=gbs(sustained["step_ms_last_quarter"]),
+                         frac_last_quarter=gbs(sustained["step_ms_last_quarter"]) / peak, unit="GB/s")
     if zero_cases is not None:
         for c in zero_cases.values():
             c.update(gbs=gbs(c["ms"]), frac=gbs(c["ms"]) / peak)
@@ -647,11 +650,13 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": (NCU_TRAFFIC_CAPTURE[0] / NCU_TRAFFIC_CAPTURE[1] * n if NCU_TRAFFIC_CAPTURE else None),
                      "peak_source": peak_src, "frac_nominal": achieved / NOMINAL_HBM_GBS, "nominal_gbs": NOMINAL_HBM_GBS,
-                     "kernel": "k_sr_adamw_flat_fast", "launch_ms_avg": avg_launch_ms,
-                     "launch_ms_min": min(launch_ms), "launch_ms_median": statistics.median(launch_ms),
-                     "algorithmic_bytes_per_launch": BYTES_PER_ELEMENT * n,
+                     "kernel": "k_sr_adamw_flat_fast", "launches_per_step": launches_per_step,
+                     "step_ms_avg": avg_launch_ms, "step_ms_min": min(launch_ms), "step_ms_median": statistics.median(launch_ms),
+                     "launch_ms_avg": avg_launch_ms / launches_per_step,
+                     "algorithmic_bytes_per_step": BYTES_PER_ELEMENT * n,
+                     "algorithmic_bytes_per_launch": BYTES_PER_ELEMENT * n / launches_per_step,
                      "sustained": sustained},
-        "gpu_launches": args.steps,
+        "gpu_launches": args.steps * launches_per_step,
         "clocks": clocks,
     }
     if e2e is not None:

@@ -130,6 +130,10 @@ sr_status sr_accumulate_bf16(uint16_t* acc, const void* g, sr_dtype g_dtype, uin
 sr_status sr_adamw_step(uint16_t* p, const void* g, sr_dtype g_dtype, uint16_t* m, uint16_t* v, uint64_t n,
                         const sr_adamw_hparams* hp, uint64_t seed, uint32_t step, uint32_t tensor_id,
                         uint64_t elem_offset, void* stream);
+/* Number of kernel launches one sr_adamw_step call of n elements at elem_offset enqueues: the call is cut into
+ * launches of 2^28 elements (the last one up to 1.5 times that), none crossing a multiple of 2^33 in index
+ * space.  The cuts change nothing in the result.  Host-only. */
+uint32_t sr_adamw_step_launch_count(uint64_t n, uint64_t elem_offset);
 
 /* The mixed-precision recipe the paper compares against (Section 3: FP32 master weights and FP32
  * optimizer states, BF16 copy of the weights), provided so that both recipes can be measured with
@@ -157,8 +161,10 @@ sr_status sr_adamw_step_host(uint16_t* p_host, const void* g_host, sr_dtype g_dt
                              uint32_t tensor_id, uint64_t elem_offset, void* staging, size_t staging_bytes,
                              uint64_t chunk_elems, void* stream);
 
-/* The same iteration over a list of tensors in one launch.  A plan owns device copies of the
- * pointer / size table and of the chunk table that maps thread blocks to (tensor, range).
+/* The same iteration over a list of tensors: one launch for all tensors below 2^24 elements (and for those
+ * whose buffers are not 16-byte aligned), plus one launch of the flat kernel per larger tensor, all enqueued on
+ * `stream` by the one call.  A plan owns a device copy of the chunk table that maps thread blocks to
+ * (tensor, range), and the host-side list of the large tensors.
  * The arrays passed to sr_mt_plan_create are HOST arrays of num_tensors entries holding device
  * pointers and element counts; they may be freed after the call.  Tensor i uses
  * tensor_id = tensor_id_base + i and element indices starting at 0.  One hparams set serves the list.

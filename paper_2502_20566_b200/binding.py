@@ -24,7 +24,7 @@ SR_FLAGS_DEFAULT = 7
 SR_FLAG_EPS_INSIDE = 8
 
 EXPORTS = (
-    "sr_downcast_f32_bf16", "sr_downcast_f32_fp8", "sr_downcast_f32_fp4", "sr_accumulate_bf16", "sr_adamw_step", "sr_master_adamw_step", "sr_adamw_step_host", "sr_adamw_step_host_staging_bytes",
+    "sr_downcast_f32_bf16", "sr_downcast_f32_fp8", "sr_downcast_f32_fp4", "sr_accumulate_bf16", "sr_adamw_step", "sr_adamw_step_launch_count", "sr_master_adamw_step", "sr_adamw_step_host", "sr_adamw_step_host_staging_bytes",
     "sr_mt_plan_create", "sr_adamw_multi_tensor",
     "sr_mt_plan_destroy", "sr_mt_plan_total_elements", "grad_sqnorm_workspace_bytes", "grad_sqnorm",
     "grad_sqnorm_static", "grad_sqnorm_static_max_elements", "grad_sqnorm_multi_tensor", "grad_sqnorm_multi_tensor_workspace_bytes",
@@ -117,6 +117,8 @@ def lib() -> ctypes.CDLL:
         L.grad_sqnorm_static_max_elements.restype = c_uint64
         L.sr_clip_scale.argtypes = [c_void_p, c_float, c_float, c_void_p, c_void_p]
         L.sr_clip_scale.restype = c_int
+        L.sr_adamw_step_launch_count.argtypes = [c_uint64, c_uint64]
+        L.sr_adamw_step_launch_count.restype = c_uint32
         L.sr_selftest_in_range_arithmetic.argtypes = [c_uint64, c_uint64, c_void_p, c_void_p]
         L.sr_selftest_in_range_arithmetic.restype = c_int
         L.sr_status_string.argtypes = [c_int]
@@ -356,6 +358,11 @@ def sr_clip_scale(sqnorm: torch.Tensor, accum_scale: float, max_norm: float, gsc
     with torch.cuda.device(sqnorm.device):
         _check(lib().sr_clip_scale(sqnorm.data_ptr(), accum_scale, max_norm, gscale_out.data_ptr(), _stream(stream)),
                "sr_clip_scale")
+
+
+def sr_adamw_step_launch_count(n: int, elem_offset: int = 0) -> int:
+    """Kernel launches that one sr_adamw_step call of n elements at elem_offset enqueues."""
+    return int(lib().sr_adamw_step_launch_count(n, elem_offset))
 
 
 def sr_selftest_in_range_arithmetic(seed: int, sets: int, mismatches: torch.Tensor, stream=None) -> None:

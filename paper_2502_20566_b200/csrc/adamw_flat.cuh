@@ -297,13 +297,12 @@ cudaError_t launch_flat_flags(uint16_t* p, const void* g, uint16_t* m, uint16_t*
                               uint32_t tensor_id, uint32_t seed_hi, const PhiloxKeys& K, const StepScalars& S,
                               const DeviceInfo& dev, cudaStream_t stream) {
     const size_t gsz = G32 ? 4 : 2;
-    // one launch per run of indices that share (index >> 33); a single launch unless the buffer
-    // crosses a multiple of 2^33 in global index space
+    // launches of at most 1.5 * kFlatLaunchElems elements, none of which crosses a multiple of 2^33 in global index
+    // space (every index of a launch shares index >> 33)
     uint64_t done = 0;
     while (done < n) {
         const uint64_t idx = elem_offset + done;
-        const uint64_t to_boundary = (static_cast<uint64_t>(1) << 33) - (idx & ((static_cast<uint64_t>(1) << 33) - 1));
-        const uint64_t len = n - done < to_boundary ? n - done : to_boundary;
+        const uint64_t len = next_flat_launch(idx, n - done);
         uint16_t* ps = p + done;
         const void* gs = static_cast<const char*>(g) + done * gsz;
         uint16_t* ms = m + done;

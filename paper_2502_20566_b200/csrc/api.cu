@@ -130,8 +130,25 @@ int current_device_info(DeviceInfo* out, int* device_index) {
 }
 }  // namespace sradamw
 
+// A tensor of a list that is stepped by a flat launch of its own (see sr_adamw_multi_tensor).
+struct LargeTensor {
+    uint16_t* p;
+    const void* g;
+    uint16_t* m;
+    uint16_t* v;
+    uint64_t numel;
+    uint32_t index;
+};
+// Tensors of at least this many elements whose four buffers are 16-byte aligned: from here on one flat launch per
+// tensor is faster than the tensor's share of the list kernel (B200: flat launches of 2^24 / 2^25 / 2^26 elements run
+// at 89 / 91 / 96 % of the copy peak, the list kernel at 84-88 %).
+constexpr uint64_t kMtFlatElems = static_cast<uint64_t>(1) << 24;
+
 struct sr_mt_plan {
-    MtWork* d_work = nullptr;
+    MtWork* d_work = nullptr;        // every chunk of every tensor, in list order (the list norm reads this one)
+    MtWork* d_small = nullptr;       // the chunks of the tensors that the list kernel steps (inside d_work's allocation)
+    uint32_t num_small = 0;
+    std::vector<LargeTensor> large;  // the tensors stepped by flat launches
     uint32_t num_tensors = 0;
     uint32_t num_chunks = 0;
     uint64_t total_elements = 0;
@@ -151,6 +168,12 @@ sr_status sr_downcast_f32_bf16(const float* src, uint16_t* dst, uint64_t n, uint
     const cudaError_t e = launch_downcast(src, dst, n, elem_offset, tensor_id, static_cast<uint32_t>(seed >> 32),
                                           make_keys(seed, step), dev, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? SR_OK : cuda_fail(e);
+}
+
+uint32_t sr_adamw_step_launch_count(uint64_t n, uint64_t elem_offset) {
+    uint32_t count = 0;
+    for (uint64_t done = 0; done < n; ++count) done += next_flat_launch(elem_offset + done, n - done);
+    return count;
 }
 
 sr_status sr_selftest_in_range_arithmetic(uint64_t seed, uint64_t sets, uint64_t* mismatches_dev, void* stream) {
@@ -361,7 +384,8 @@ sr_status sr_mt_plan_create(sr_mt_plan** out, uint32_t num_tensors, uint16_t* co
 
     if (num_tensors > 0x7FFFFFFFu) return SR_ERR_INVALID_ARG;
     const size_t gsz = g_dtype == SR_DT_F32 ? 4 : 2;
-    std::vector<MtWork> chunks;
+    std::vector<MtWork> chunks, small;
+    std::vector<LargeTensor> large;
     uint64_t total = 0;
     try {
     for (uint32_t i = 0; i < num_tensors; ++i) {
@@ -372,11 +396,15 @@ sr_status sr_mt_plan_create(sr_mt_plan** out, uint32_t num_tensors, uint16_t* co
         const uintptr_t bits = reinterpret_cast<uintptr_t>(p[i]) | reinterpret_cast<uintptr_t>(g[i]) |
                                reinterpret_cast<uintptr_t>(m[i]) | reinterpret_cast<uintptr_t>(v[i]);
         const uint32_t tensor_vec = i | ((bits & 15u) == 0 ? 0x80000000u : 0u);
+        const bool flat = (bits & 15u) == 0 && numel[i] >= kMtFlatElems;
+        if (flat) large.push_back(LargeTensor{p[i], g[i], m[i], v[i], numel[i], i});
         for (uint64_t c = 0; c < nchunks; ++c) {
             const uint64_t start = c * kMtChunkElems;
             const uint64_t left = numel[i] - start;
-            chunks.push_back(MtWork{p[i] + start, static_cast<const char*>(g[i]) + start * gsz, m[i] + start, v[i] + start,
-                                    start, static_cast<uint32_t>(left < kMtChunkElems ? left : kMtChunkElems), tensor_vec});
+            const MtWork w{p[i] + start, static_cast<const char*>(g[i]) + start * gsz, m[i] + start, v[i] + start,
+                           start, static_cast<uint32_t>(left < kMtChunkElems ? left : kMtChunkElems), tensor_vec};
+            chunks.push_back(w);
+            if (!flat) small.push_back(w);
         }
         total += numel[i];
     }
@@ -393,10 +421,22 @@ sr_status sr_mt_plan_create(sr_mt_plan** out, uint32_t num_tensors, uint16_t* co
     cudaGetDevice(&plan->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaSuccess;
+    plan->num_small = static_cast<uint32_t>(small.size());
+    try {
+        plan->large = std::move(large);
+    } catch (const std::bad_alloc&) {
+        delete plan;
+        return SR_ERR_WORKSPACE;
+    }
     if (!chunks.empty()) {
-        e = cudaMalloc(&plan->d_work, chunks.size() * sizeof(MtWork));
+        // one allocation: the full table, then the table of the list kernel's share
+        e = cudaMalloc(&plan->d_work, (chunks.size() + small.size()) * sizeof(MtWork));
         if (e == cudaSuccess)
             e = cudaMemcpyAsync(plan->d_work, chunks.data(), chunks.size() * sizeof(MtWork), cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess && !small.empty()) {
+            plan->d_small = plan->d_work + chunks.size();
+            e = cudaMemcpyAsync(plan->d_small, small.data(), small.size() * sizeof(MtWork), cudaMemcpyHostToDevice, s);
+        }
         // the host vectors die at return: wait for the copies (plan creation is not a hot call)
         if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     }
@@ -422,10 +462,18 @@ sr_status sr_adamw_multi_tensor(const sr_mt_plan* plan, const sr_adamw_hparams* 
     int current = -1;
     cudaGetDevice(&current);
     if (current != plan->device) return SR_ERR_INVALID_ARG;   // the work table lives on the plan's device
-    const cudaError_t e =
-        launch_adamw_mt(plan->d_work, plan->num_chunks, plan->g_f32, tensor_id_base,
-                        static_cast<uint32_t>(seed >> 32), hp->flags, make_keys(seed, step), S, dev,
-                        static_cast<cudaStream_t>(stream));
+    // large tensors: one flat launch each (index restarts at 0 in every tensor, the tensor id is base + list index:
+    // the same noise as in the list kernel); all the others: one launch of the list kernel
+    const PhiloxKeys K = make_keys(seed, step);
+    const uint32_t seed_hi = static_cast<uint32_t>(seed >> 32);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (const LargeTensor& t : plan->large) {
+        const cudaError_t e = launch_adamw_flat(t.p, t.g, plan->g_f32, t.m, t.v, t.numel, 0, tensor_id_base + t.index, seed_hi,
+                                                hp->flags, K, S, dev, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (plan->num_small == 0) return SR_OK;
+    const cudaError_t e = launch_adamw_mt(plan->d_small, plan->num_small, plan->g_f32, tensor_id_base, seed_hi, hp->flags, K, S, dev, s);
     return e == cudaSuccess ? SR_OK : cuda_fail(e);
 }
 

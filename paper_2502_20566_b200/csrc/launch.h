@@ -60,6 +60,19 @@ constexpr uint32_t kMtChunkElems = 8192;   // multiple of 8; never crosses a mul
 // shape remains for offsets that are not multiples of 8.
 constexpr int kFlatDirectThreads = 256;
 constexpr int kFlatDirectMinBlocks = 2;
+// A flat call is cut into launches of 2^28 elements (the last one up to 1.5 times that).  Mid-size launches run faster
+// per element than one huge one wherever the board is not yet on its power cap: 6.7B elements, first 20 calls /
+// sustained, cut at 2^26, 2^27, 2^28, 2^29, not at all: 14.96 / 15.60, 14.85 / 15.45, 14.80 / 15.36, 14.88 / 15.36,
+// 15.31 / 15.46 ms on a GPU that sustains 1.67 GHz, and 15.66 / 16.45 (2^28) against 15.78 / 16.43 ms (not cut) on one
+// that sustains 1.55 GHz.
+constexpr uint64_t kFlatLaunchElems = static_cast<uint64_t>(1) << 28;
+// the cut points of a flat call: lengths of its launches in order (shared by the launcher and the launch count)
+inline uint64_t next_flat_launch(uint64_t idx, uint64_t left) {
+    const uint64_t to_boundary = (static_cast<uint64_t>(1) << 33) - (idx & ((static_cast<uint64_t>(1) << 33) - 1));
+    uint64_t len = left < to_boundary ? left : to_boundary;   // every index of a launch has the same index >> 33
+    if (len > kFlatLaunchElems + kFlatLaunchElems / 2) len = kFlatLaunchElems;   // a multiple of 8: alignment and noise groups carry over
+    return len;
+}
 constexpr int kFlatStagedThreadsF32 = 512;
 constexpr int kFlatStagesF32 = 2;
 constexpr int kBlockThreads = SR_BLOCK_THREADS;
