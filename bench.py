@@ -38,8 +38,9 @@ NOMINAL_HBM_GBS = 7700.0        # data-sheet bandwidth of the HGX B200 (context 
 # build and launch shape on a smaller case: (dram bytes read + written, elements of that case).  The traffic of
 # a streaming kernel grows in proportion to the element count, so the full-size figure is bytes / elements * n.
 # None whenever the kernel has changed since the capture was taken.  Current values: k_sr_adamw_flat_fast (BF16
-# gradients, 384 x 1 blocks, 3 stages) on 2^29 elements, dram__bytes_read.sum + dram__bytes_write.sum of one launch.
-NCU_TRAFFIC_CAPTURE = (7_459_395_000, 536_870_912)
+# gradients, 384 x 1 blocks, 3 stages) on 2^28 elements (the length a flat call is cut into), dram__bytes_read.sum +
+# dram__bytes_write.sum of one launch.
+NCU_TRAFFIC_CAPTURE = (3_704_089_000, 268_435_456)
 
 
 def parse_args():
