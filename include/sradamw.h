@@ -13,6 +13,9 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls enqueue work and
  *     return; they never synchronise the device and never allocate device memory, except
  *     sr_mt_plan_create / sr_mt_plan_destroy.
+ *   - The step kernels keep their staging in more shared memory than a kernel gets by default: the first call that
+ *     needs a kernel variant on a device sets that kernel's attribute (cudaFuncSetAttribute; nothing is allocated).
+ *     Make the first call of a configuration outside any stream capture.
  *   - x, m, v are updated in place; g is only read.  Buffers of one call must not overlap each other.
  *   - n == 0 is a successful no-op.  Any base alignment is accepted; the 16-byte vector path needs
  *     all buffers of a call 16-byte aligned and otherwise an element-wise path is taken.
