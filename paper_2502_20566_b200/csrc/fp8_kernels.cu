@@ -117,11 +117,11 @@ __device__ __forceinline__ uint32_t cast4(const uint4 x, const uint4 w) {
 
 // sixteen consecutive values -> sixteen bytes (four Philox calls)
 template <int FMT>
-__device__ __forceinline__ uint4 cast16(const float* __restrict__ src, uint64_t vec, uint64_t elem_offset, uint32_t tensor_id,
+__device__ __forceinline__ uint4 cast16(const float* __restrict__ src, uint64_t vec, uint64_t elem_offset, uint32_t c1, uint32_t tensor_id,
                                         uint32_t seed_hi, const PhiloxKeys& K) {
     const uint4 a = ld16(src, 4 * vec), b = ld16(src, 4 * vec + 1), c = ld16(src, 4 * vec + 2), d = ld16(src, 4 * vec + 3);
     const uint64_t number = (elem_offset + (vec << 4)) >> 2;
-    const uint32_t c0 = static_cast<uint32_t>(number), c1 = static_cast<uint32_t>(number >> 32);
+    const uint32_t c0 = static_cast<uint32_t>(number);
     uint4 o;
     o.x = cast4<FMT>(a, philox4x32_10(c0, c1, tensor_id, seed_hi, K));
     o.y = cast4<FMT>(b, philox4x32_10(c0 + 1, c1, tensor_id, seed_hi, K));
@@ -131,11 +131,11 @@ __device__ __forceinline__ uint4 cast16(const float* __restrict__ src, uint64_t 
 }
 
 // sixteen consecutive values -> sixteen 4-bit codes in eight bytes
-__device__ __forceinline__ uint2 cast16_fp4(const float* __restrict__ src, uint64_t vec, uint64_t elem_offset, uint32_t tensor_id,
+__device__ __forceinline__ uint2 cast16_fp4(const float* __restrict__ src, uint64_t vec, uint64_t elem_offset, uint32_t c1, uint32_t tensor_id,
                                             uint32_t seed_hi, const PhiloxKeys& K) {
     const uint4 a = ld16(src, 4 * vec), b = ld16(src, 4 * vec + 1), c = ld16(src, 4 * vec + 2), d = ld16(src, 4 * vec + 3);
     const uint64_t number = (elem_offset + (vec << 4)) >> 2;
-    const uint32_t c0 = static_cast<uint32_t>(number), c1 = static_cast<uint32_t>(number >> 32);
+    const uint32_t c0 = static_cast<uint32_t>(number);
     const uint32_t lo = cast4_fp4(a, philox4x32_10(c0, c1, tensor_id, seed_hi, K)) |
                         (cast4_fp4(b, philox4x32_10(c0 + 1, c1, tensor_id, seed_hi, K)) << 16);
     const uint32_t hi = cast4_fp4(c, philox4x32_10(c0 + 2, c1, tensor_id, seed_hi, K)) |
@@ -146,13 +146,16 @@ __device__ __forceinline__ uint2 cast16_fp4(const float* __restrict__ src, uint6
 // Up to 128 registers: the values of an iteration are independent and the two pipes overlap only when the compiler
 // may keep several of them in flight.  E4M3, same GPU: 16 values per iteration with 40 registers 0.321 ms, with 72
 // registers 0.299-0.313 ms; 32 values per iteration with 109-122 registers 0.300-0.306 ms; 4 or 8 values per
-// iteration with two to four times the resident warps 0.33-0.42 ms.  One block of 384 threads per SM (12 warps) against
-// four blocks of 128 (16 warps), same registers: E4M3 0.306 -> 0.294 ms, E2M1 0.293 -> 0.282 ms.
-constexpr int kSmallThreads = 384;
+// iteration with two to four times the resident warps 0.33-0.42 ms.  One block per SM, threads per block (2^28
+// values, E4M3 / E2M1, same GPU): 256 0.293 / 0.280, 384 0.294 / 0.278, 512 0.282 / 0.275, 640 0.288 / 0.273,
+// 768 0.290 / 0.275, 1024 0.294 / 0.283 ms; two blocks of 192 0.309 / 0.294, four of 128 0.306 / 0.293 ms.
+constexpr int kSmallThreads = 512;
 constexpr int kSmallMinBlocks = 1;
 
 // VEC: 16 elements per thread-iteration (4 x 16-byte loads, 1 x 16-byte store); needs both buffers
-// 16-byte aligned and elem_offset a multiple of 4 (whole noise groups).
+// 16-byte aligned, elem_offset a multiple of 16 and every index of the launch's whole vectors with the same
+// (index >> 34), the high word c1 of the call number: the first Philox round's product with the tensor id and what
+// follows from it and c1 alone are then loop-invariant (E2M1 0.282 -> 0.277 ms).
 template <int FMT, bool VEC>
 __global__ void __launch_bounds__(kSmallThreads, kSmallMinBlocks)
 k_sr_downcast_fp8(const float* __restrict__ src, uint8_t* __restrict__ dst, uint64_t n, uint64_t elem_offset,
@@ -162,15 +165,16 @@ k_sr_downcast_fp8(const float* __restrict__ src, uint8_t* __restrict__ dst, uint
     uint64_t done = 0;
     if (VEC) {
         const uint64_t nvec = n >> 4;
+        const uint32_t c1 = static_cast<uint32_t>(elem_offset >> 34);
         // two vectors per iteration: 32 independent values for the compiler to interleave
         uint64_t vec = tid;
         for (; vec + stride < nvec; vec += 2 * stride) {
-            const uint4 o0 = cast16<FMT>(src, vec, elem_offset, tensor_id, seed_hi, K);
-            const uint4 o1 = cast16<FMT>(src, vec + stride, elem_offset, tensor_id, seed_hi, K);
+            const uint4 o0 = cast16<FMT>(src, vec, elem_offset, c1, tensor_id, seed_hi, K);
+            const uint4 o1 = cast16<FMT>(src, vec + stride, elem_offset, c1, tensor_id, seed_hi, K);
             st16(dst, vec, o0);
             st16(dst, vec + stride, o1);
         }
-        if (vec < nvec) st16(dst, vec, cast16<FMT>(src, vec, elem_offset, tensor_id, seed_hi, K));
+        if (vec < nvec) st16(dst, vec, cast16<FMT>(src, vec, elem_offset, c1, tensor_id, seed_hi, K));
         done = nvec << 4;
     }
     for (uint64_t i = done + tid; i < n; i += stride)
@@ -178,8 +182,8 @@ k_sr_downcast_fp8(const float* __restrict__ src, uint8_t* __restrict__ dst, uint
 }
 
 // E2M1, two codes per byte (element 2j in bits 0..3 of byte j).  VEC: 16 elements per
-// thread-iteration (4 x 16-byte loads, one 8-byte store); needs src 16-byte and dst 8-byte aligned
-// and elem_offset a multiple of 16.  The rest (and everything without VEC) goes byte by byte, one
+// thread-iteration (4 x 16-byte loads, one 8-byte store); needs src 16-byte and dst 8-byte aligned,
+// elem_offset a multiple of 16 and one (index >> 34) for the launch's whole vectors.  The rest (and everything without VEC) goes byte by byte, one
 // thread per output byte.
 template <bool VEC>
 __global__ void __launch_bounds__(kSmallThreads, kSmallMinBlocks)
@@ -190,15 +194,16 @@ k_sr_downcast_fp4(const float* __restrict__ src, uint8_t* __restrict__ dst, uint
     uint64_t done = 0;
     if (VEC) {
         const uint64_t nvec = n >> 4;
+        const uint32_t c1 = static_cast<uint32_t>(elem_offset >> 34);
         // two vectors per iteration: 32 independent values for the compiler to interleave
         uint64_t vec = tid;
         for (; vec + stride < nvec; vec += 2 * stride) {
-            const uint2 o0 = cast16_fp4(src, vec, elem_offset, tensor_id, seed_hi, K);
-            const uint2 o1 = cast16_fp4(src, vec + stride, elem_offset, tensor_id, seed_hi, K);
+            const uint2 o0 = cast16_fp4(src, vec, elem_offset, c1, tensor_id, seed_hi, K);
+            const uint2 o1 = cast16_fp4(src, vec + stride, elem_offset, c1, tensor_id, seed_hi, K);
             __stcs(reinterpret_cast<uint2*>(dst) + vec, o0);
             __stcs(reinterpret_cast<uint2*>(dst) + vec + stride, o1);
         }
-        if (vec < nvec) __stcs(reinterpret_cast<uint2*>(dst) + vec, cast16_fp4(src, vec, elem_offset, tensor_id, seed_hi, K));
+        if (vec < nvec) __stcs(reinterpret_cast<uint2*>(dst) + vec, cast16_fp4(src, vec, elem_offset, c1, tensor_id, seed_hi, K));
         done = nvec << 4;
     }
     const uint64_t nbytes = (n + 1) >> 1;
@@ -211,13 +216,26 @@ k_sr_downcast_fp4(const float* __restrict__ src, uint8_t* __restrict__ dst, uint
     }
 }
 
+// length of the next launch of a vector-path call: up to the next multiple of 2^34 (one c1 per launch)
+inline uint64_t next_small_launch(uint64_t idx, uint64_t left) {
+    const uint64_t to_boundary = (static_cast<uint64_t>(1) << 34) - (idx & ((static_cast<uint64_t>(1) << 34) - 1));
+    return left < to_boundary ? left : to_boundary;
+}
+
 template <int FMT, bool VEC>
 cudaError_t launch_fp8_t(const float* src, uint8_t* dst, uint64_t n, uint64_t elem_offset, uint32_t tensor_id,
                          uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev, cudaStream_t stream) {
     auto k = k_sr_downcast_fp8<FMT, VEC>;
-    const uint64_t items = VEC ? (n >> 4) + 16 : n;
-    k<<<grid_for(k, items, dev, kSmallThreads), kSmallThreads, 0, stream>>>(src, dst, n, elem_offset, tensor_id, seed_hi, K);
-    return cudaGetLastError();
+    for (uint64_t done = 0; done < n;) {
+        const uint64_t len = VEC ? next_small_launch(elem_offset + done, n - done) : n;
+        const uint64_t items = VEC ? (len >> 4) + 16 : len;
+        k<<<grid_for(k, items, dev, kSmallThreads), kSmallThreads, 0, stream>>>(src + done, dst + done, len, elem_offset + done,
+                                                                                tensor_id, seed_hi, K);
+        const cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        done += len;
+    }
+    return cudaSuccess;
 }
 
 }  // namespace
@@ -236,15 +254,22 @@ cudaError_t launch_downcast_fp8(const float* src, uint8_t* dst, uint64_t n, bool
 cudaError_t launch_downcast_fp4(const float* src, uint8_t* dst, uint64_t n, uint64_t elem_offset, uint32_t tensor_id,
                                 uint32_t seed_hi, const PhiloxKeys& K, const DeviceInfo& dev, cudaStream_t stream) {
     const bool vec = aligned16(src) && (reinterpret_cast<uintptr_t>(dst) & 7u) == 0 && (elem_offset & 15u) == 0;
-    const uint64_t items = (vec ? (n >> 4) + 16 : (n + 1) >> 1);
-    if (vec) {
-        auto k = k_sr_downcast_fp4<true>;
-        k<<<grid_for(k, items, dev, kSmallThreads), kSmallThreads, 0, stream>>>(src, dst, n, elem_offset, tensor_id, seed_hi, K);
-    } else {
+    if (!vec) {
         auto k = k_sr_downcast_fp4<false>;
-        k<<<grid_for(k, items, dev, kSmallThreads), kSmallThreads, 0, stream>>>(src, dst, n, elem_offset, tensor_id, seed_hi, K);
+        k<<<grid_for(k, (n + 1) >> 1, dev, kSmallThreads), kSmallThreads, 0, stream>>>(src, dst, n, elem_offset, tensor_id, seed_hi, K);
+        return cudaGetLastError();
     }
-    return cudaGetLastError();
+    auto k = k_sr_downcast_fp4<true>;
+    // a cut falls on a multiple of 16 elements: whole vectors and whole bytes before it
+    for (uint64_t done = 0; done < n;) {
+        const uint64_t len = next_small_launch(elem_offset + done, n - done);
+        k<<<grid_for(k, (len >> 4) + 16, dev, kSmallThreads), kSmallThreads, 0, stream>>>(src + done, dst + (done >> 1), len,
+                                                                                          elem_offset + done, tensor_id, seed_hi, K);
+        const cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        done += len;
+    }
+    return cudaSuccess;
 }
 
 }  // namespace sradamw
