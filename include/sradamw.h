@@ -97,7 +97,8 @@ sr_status sr_downcast_f32_bf16(const float* src, uint16_t* dst, uint64_t n, uint
  * 32 fractional bits).  Magnitudes at or beyond the largest finite level saturate to it (E5M2 keeps
  * +-inf), NaN gives 0x7F.  Noise: one Philox call per four consecutive indices, counter number =
  * index >> 2 (other counter and key words as above), element index & 3 takes output word index & 3.
- * src: n FP32 values; dst: n bytes. */
+ * src: n FP32 values; dst: n bytes.  A call whose indices cross a multiple of 2^34 is enqueued as one
+ * launch per stretch, in order on the stream (sr_downcast_f32_fp4 likewise). */
 typedef enum { SR_FP8_E4M3 = 0, SR_FP8_E5M2 = 1 } sr_fp8_format;
 sr_status sr_downcast_f32_fp8(const float* src, uint8_t* dst, uint64_t n, sr_fp8_format format, uint64_t seed,
                               uint32_t step, uint32_t tensor_id, uint64_t elem_offset, void* stream);
