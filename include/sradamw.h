@@ -192,8 +192,9 @@ uint64_t sr_mt_plan_total_elements(const sr_mt_plan* plan);
  * accumulators, accumulator j adding entries r*1024 + 4j + k (r = 0..7, k = 0..3) in that order;
  * 8 groups of 32 accumulators folded by an XOR butterfly (16, 8, 4, 2, 1), group values added in
  * order; the block sums are reduced again by the same rule until one value is left.
- * out_dev: one double on the device.  workspace: device memory of at least
- * grad_sqnorm_workspace_bytes(n) bytes, 8-byte aligned (may be NULL when that size is 0). */
+ * out_dev: one double on the device; while the call's kernels run it holds a count of finished blocks
+ * (n > 2^26), so nothing else may read it before they have completed.  workspace: device memory of at
+ * least grad_sqnorm_workspace_bytes(n) bytes, 8-byte aligned (may be NULL when that size is 0). */
 size_t grad_sqnorm_workspace_bytes(uint64_t n);
 sr_status grad_sqnorm(const void* g, sr_dtype g_dtype, uint64_t n, double* out_dev, void* workspace,
                       size_t workspace_bytes, void* stream);

@@ -517,6 +517,24 @@ def test_sqnorm_unaligned(env, g_dtype):
     assert float(out.item()).hex() == oracle.sqnorm(host_g(g)).hex()
 
 
+@pytest.mark.parametrize("g_dtype", [torch.float32, torch.bfloat16])
+def test_sqnorm_with_more_than_one_later_level(env, g_dtype):
+    """More than 8192 tree blocks: the pass over the block sums also folds its own results, and the output cell counts
+    its finished blocks first, whatever the cell held before the call.  Repeated, because the block that folds is the
+    one that happens to finish last."""
+    oracle, binding, synth, dev = env
+    n = 3 * 8192 * 8192 + 777
+    g = torch.empty(n, dtype=g_dtype, device=dev)
+    synth.fill_state(g, synth.ROLE_G, 19, outlier_fraction=0.01)
+    want = oracle.sqnorm(host_g(g)).hex()
+    ws = torch.empty(binding.grad_sqnorm_workspace_bytes(n) // 8, dtype=torch.float64, device=dev)
+    for before in (-1.0, float("nan"), 1e300, 0.0, 5e-324, float("inf")) * 3:
+        out = torch.full((1,), before, dtype=torch.float64, device=dev)
+        binding.grad_sqnorm(g, out, ws)
+        torch.cuda.synchronize()
+        assert float(out.item()).hex() == want
+
+
 def test_clip_scale_bit_exact(env):
     oracle, binding, _, dev = env
     out = torch.zeros(1, dtype=torch.float32, device=dev)
