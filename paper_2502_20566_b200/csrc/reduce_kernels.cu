@@ -74,6 +74,12 @@ __device__ __forceinline__ double fold_block_pairs(double a0, double a1, double*
 }
 
 constexpr int kPairThreads = 128;   // BF16 entries: two accumulators per thread
+// Resident blocks per SM asked of the compiler for the first passes (their register budgets).  355M entries, same GPU:
+// BF16 flat 0.1257 ms with 55 registers (no bound, 9 blocks), 0.1156 with 77 (6 blocks), 0.1132 with 61 (8 blocks);
+// BF16 list 0.1196 ms with 80 registers (no bound, 6 blocks), 0.1172 (7), 0.1160 (8), 0.1169 (9 blocks); FP32 list
+// 0.2322 ms with 90 registers (no bound, 2 blocks of 256 threads), 0.2090 (3 blocks), 0.2086 (4 blocks).
+constexpr int kPairMinBlocks = 8;
+constexpr int kListF32MinBlocks = 4;
 
 // One whole, 16-byte aligned tree block of BF16 entries: eight 16-byte loads per thread, all issued before the
 // first addition.  t = threadIdx.x of a 128-thread block; returns the block sum in thread 0.
@@ -146,7 +152,7 @@ __device__ __forceinline__ double bf16_block_sum_ragged(const uint16_t* chunk, u
 
 // First pass: out[c] = tree-block sum of squares of entries [c*8192, (c+1)*8192) of g.
 template <bool G32>
-__global__ void __launch_bounds__(G32 ? kTreeThreads : kPairThreads)
+__global__ void __launch_bounds__(G32 ? kTreeThreads : kPairThreads, G32 ? 1 : kPairMinBlocks)
 k_sqnorm_pass1(const void* __restrict__ g, uint64_t n, uint64_t num_blocks, bool vec_ok, double* __restrict__ out,
                unsigned long long* ticket) {
     __shared__ double warp_sums[8];
@@ -189,7 +195,7 @@ k_sqnorm_pass1(const void* __restrict__ g, uint64_t n, uint64_t num_blocks, bool
 // First pass over a tensor list: out[c] = tree-block sum of squares of work-table entry c (a chunk of
 // at most 8192 consecutive gradient entries of one tensor, positions counted from the chunk's start).
 template <bool G32>
-__global__ void __launch_bounds__(G32 ? kTreeThreads : kPairThreads)
+__global__ void __launch_bounds__(G32 ? kTreeThreads : kPairThreads, G32 ? kListF32MinBlocks : kPairMinBlocks)
 k_sqnorm_mt_pass1(const MtWork* __restrict__ work, uint32_t num_chunks, double* __restrict__ out,
                   unsigned long long* ticket) {
     __shared__ double warp_sums[8];
