@@ -22,6 +22,21 @@ __device__ __forceinline__ float accumulate(float acc, float g, float scale) {
     return __fadd_rn(acc, __fmul_rn(scale, g));
 }
 
+// one vector of eight: sums in FP32, rounded with the noise words w
+template <bool SR>
+__device__ __forceinline__ uint4 accumulate_vec(const uint4 av, const float (&ge)[8], const uint4 w, float scale) {
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint32_t aw = word_of(av, j);
+        const float s0 = accumulate(bf16_lo(aw), ge[2 * j], scale);
+        const float s1 = accumulate(bf16_hi(aw), ge[2 * j + 1], scale);
+        o[j] = pack_top_halves(round_sum_word_nan_safe<SR, false>(s0, word_of(w, j)),
+                               round_sum_word_nan_safe<SR, true>(s1, word_of(w, j)));
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 // MODE 0: element-wise; 1: 16-byte vectors straddling two noise groups (offset not a multiple of 8); 2: vectors, grouped
 #ifndef SR_ACCUM_STRADDLE_MIN_BLOCKS
 #define SR_ACCUM_STRADDLE_MIN_BLOCKS 1
@@ -44,7 +59,25 @@ k_sr_accumulate(uint16_t* acc, const void* g, uint64_t n, float scale, uint64_t 
         const Chain chain{heads + (MODE == 1 ? (threadIdx.x >> 5) * Chain::kTableEntries : 0), elem_offset >> 3, stride,
                           static_cast<uint32_t>(elem_offset) & 7u, lane, 0u, tensor_id, seed_hi};
         uint32_t k = 0;
-        for (uint64_t vec = tid; vec < nvec; vec += stride, ++k) {
+        uint64_t vec = tid;
+        if (MODE == 2) {
+            // two vectors per iteration: four 16-byte loads in flight per thread (838M elements: 0.812 -> 0.801 ms)
+            for (; vec + stride < nvec; vec += 2 * stride) {
+                const uint4 av0 = ld16(acc, vec), av1 = ld16(acc, vec + stride);
+                float ge0[8], ge1[8];
+                load_grad8<G32>(g, vec, ge0);
+                load_grad8<G32>(g, vec + stride, ge1);
+                uint4 w0 = make_uint4(0, 0, 0, 0), w1 = w0;
+                if (SR) {
+                    const uint64_t n0 = (((elem_offset >> 3) + vec) << 2) | kAccumSlot, n1 = n0 + (stride << 2);
+                    w0 = philox4x32_10(static_cast<uint32_t>(n0), static_cast<uint32_t>(n0 >> 32), tensor_id, seed_hi, K);
+                    w1 = philox4x32_10(static_cast<uint32_t>(n1), static_cast<uint32_t>(n1 >> 32), tensor_id, seed_hi, K);
+                }
+                st16(acc, vec, accumulate_vec<SR>(av0, ge0, w0, scale));
+                st16(acc, vec + stride, accumulate_vec<SR>(av1, ge1, w1, scale));
+            }
+        }
+        for (; vec < nvec; vec += stride, ++k) {
             const uint4 av = ld16(acc, vec);
             float ge[8];
             load_grad8<G32>(g, vec, ge);
@@ -58,16 +91,7 @@ k_sr_accumulate(uint16_t* acc, const void* g, uint64_t n, float scale, uint64_t 
                 const uint64_t number = (((elem_offset >> 3) + vec) << 2) | kAccumSlot;
                 w = philox4x32_10(static_cast<uint32_t>(number), static_cast<uint32_t>(number >> 32), tensor_id, seed_hi, K);
             }
-            uint32_t o[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint32_t aw = word_of(av, j);
-                const float s0 = accumulate(bf16_lo(aw), ge[2 * j], scale);
-                const float s1 = accumulate(bf16_hi(aw), ge[2 * j + 1], scale);
-                o[j] = pack_top_halves(round_sum_word_nan_safe<SR, false>(s0, word_of(w, j)),
-                                       round_sum_word_nan_safe<SR, true>(s1, word_of(w, j)));
-            }
-            st16(acc, vec, make_uint4(o[0], o[1], o[2], o[3]));
+            st16(acc, vec, accumulate_vec<SR>(av, ge, w, scale));
         }
         done = nvec << 3;
     }
