@@ -166,9 +166,13 @@ sr_status sr_adamw_step_host(uint16_t* p_host, const void* g_host, sr_dtype g_dt
                              uint64_t chunk_elems, void* stream);
 
 /* The same iteration over a list of tensors: one launch for all tensors below 2^24 elements (and for those
- * whose buffers are not 16-byte aligned), plus one launch of the flat kernel per larger tensor, all enqueued on
- * `stream` by the one call.  A plan owns a device copy of the chunk table that maps thread blocks to
- * (tensor, range), and the host-side list of the large tensors.
+ * whose buffers are not 16-byte aligned), plus one launch of the flat kernel per larger tensor, all enqueued by
+ * the one call and all ordered inside `stream`: they start after the work enqueued on `stream` before the call
+ * and whatever is enqueued on it afterwards starts after them.  With two or more large tensors every second
+ * launch runs on a stream that the plan owns, forked from and joined to `stream` by events inside the call (the
+ * tensors are disjoint, so the end of one launch overlaps the start of the next; the pattern can be captured in a
+ * CUDA graph).  One host thread at a time may step a given plan.  A plan owns a device copy of the chunk table
+ * that maps thread blocks to (tensor, range), the host-side list of the large tensors, and that stream.
  * The arrays passed to sr_mt_plan_create are HOST arrays of num_tensors entries holding device
  * pointers and element counts; they may be freed after the call.  Tensor i uses
  * tensor_id = tensor_id_base + i and element indices starting at 0.  One hparams set serves the list.

@@ -154,7 +154,20 @@ struct sr_mt_plan {
     uint64_t total_elements = 0;
     bool g_f32 = false;
     int device = 0;
+    // Two or more flat launches alternate between the caller's stream and this one, so that the last blocks of one
+    // launch run beside the first blocks of the next (the tensors are disjoint); fork / join by these events.
+    cudaStream_t side = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
 };
+
+static cudaError_t release_plan(sr_mt_plan* plan) {
+    if (plan->join) cudaEventDestroy(plan->join);
+    if (plan->fork) cudaEventDestroy(plan->fork);
+    if (plan->side) cudaStreamDestroy(plan->side);     // returns at once; the stream's work completes first
+    const cudaError_t e = cudaFree(plan->d_work);
+    delete plan;
+    return e;
+}
 
 extern "C" {
 
@@ -440,9 +453,13 @@ sr_status sr_mt_plan_create(sr_mt_plan** out, uint32_t num_tensors, uint16_t* co
         // the host vectors die at return: wait for the copies (plan creation is not a hot call)
         if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     }
+    if (e == cudaSuccess && plan->large.size() >= 2) {
+        e = cudaStreamCreateWithFlags(&plan->side, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&plan->fork, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&plan->join, cudaEventDisableTiming);
+    }
     if (e != cudaSuccess) {
-        cudaFree(plan->d_work);
-        delete plan;
+        release_plan(plan);
         return cuda_fail(e);
     }
     *out = plan;
@@ -467,22 +484,34 @@ sr_status sr_adamw_multi_tensor(const sr_mt_plan* plan, const sr_adamw_hparams* 
     const PhiloxKeys K = make_keys(seed, step);
     const uint32_t seed_hi = static_cast<uint32_t>(seed >> 32);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    for (const LargeTensor& t : plan->large) {
-        const cudaError_t e = launch_adamw_flat(t.p, t.g, plan->g_f32, t.m, t.v, t.numel, 0, tensor_id_base + t.index, seed_hi,
-                                                hp->flags, K, S, dev, s);
+    const bool two = plan->side != nullptr;
+    cudaError_t e = cudaSuccess;
+    if (two) {
+        e = cudaEventRecord(plan->fork, s);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(plan->side, plan->fork, 0);
         if (e != cudaSuccess) return cuda_fail(e);
     }
-    if (plan->num_small == 0) return SR_OK;
-    const cudaError_t e = launch_adamw_mt(plan->d_small, plan->num_small, plan->g_f32, tensor_id_base, seed_hi, hp->flags, K, S, dev, s);
+    size_t turn = 0;
+    for (const LargeTensor& t : plan->large) {
+        e = launch_adamw_flat(t.p, t.g, plan->g_f32, t.m, t.v, t.numel, 0, tensor_id_base + t.index, seed_hi, hp->flags, K, S,
+                              dev, (two && (turn++ & 1u)) ? plan->side : s);
+        if (e != cudaSuccess) break;
+    }
+    if (e == cudaSuccess && plan->num_small != 0)
+        e = launch_adamw_mt(plan->d_small, plan->num_small, plan->g_f32, tensor_id_base, seed_hi, hp->flags, K, S, dev,
+                            (two && (turn & 1u)) ? plan->side : s);
+    if (two) {   // joined on every path: the side stream never stays forked from the caller's
+        cudaError_t j = cudaEventRecord(plan->join, plan->side);
+        if (j == cudaSuccess) j = cudaStreamWaitEvent(s, plan->join, 0);
+        if (e == cudaSuccess) e = j;
+    }
     return e == cudaSuccess ? SR_OK : cuda_fail(e);
 }
 
 sr_status sr_mt_plan_destroy(sr_mt_plan* plan) {
     if (plan == nullptr) return SR_OK;
-    cudaError_t e1 = cudaFree(plan->d_work);
-    delete plan;
-    if (e1 != cudaSuccess) return cuda_fail(e1);
-    return SR_OK;
+    const cudaError_t e = release_plan(plan);
+    return e == cudaSuccess ? SR_OK : cuda_fail(e);
 }
 
 uint64_t sr_mt_plan_total_elements(const sr_mt_plan* plan) { return plan ? plan->total_elements : 0; }

@@ -724,6 +724,74 @@ def test_multi_tensor_long_list(env, flags, gscale):
     plan.destroy()
 
 
+def test_multi_tensor_large_tensors_keep_stream_order(env):
+    """Five tensors of 2^24 elements and more (their launches alternate between the caller's stream and the plan's own)
+    plus small ones, stepped three times on a stream of the caller's with no synchronisation: the gradients of every
+    step are copied in on that stream just before the call and the parameters copied out just after it."""
+    oracle, binding, synth, dev = env
+    sizes = [1 << 24, 100, (1 << 24) + 8, 3 << 23, 4097, 1 << 24, (1 << 24) + 16]
+    steps = 3
+    P, G, M, V, Gsrc = [], [], [], [], []
+    for i, n in enumerate(sizes):
+        p, g, m, v = synth.adamw_state(n, 500 + i, dev)
+        P.append(p); G.append(torch.zeros_like(g)); M.append(m); V.append(v)
+        Gsrc.append([synth.adamw_state(n, 600 + 10 * i + t, dev)[1] for t in range(steps)])
+    plan = binding.sr_mt_plan_create(P, G, M, V)
+    hp_o, hp_g = oracle.hparams(**HP), binding.hparams(**HP)
+    host = [[bits(t) for t in P], None, [bits(t) for t in M], [bits(t) for t in V]]
+    host_g = [[bits(Gsrc[i][t]) for i in range(len(sizes))] for t in range(steps)]
+    out = [[torch.empty_like(p) for p in P] for _ in range(steps)]
+    torch.cuda.synchronize()
+    s = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(s):
+        for t in range(steps):
+            for i in range(len(sizes)):
+                G[i].copy_(Gsrc[i][t], non_blocking=True)
+            binding.sr_adamw_multi_tensor(plan, hp_g, 23, 5 + t, tensor_id_base=7, stream=s)
+            for i in range(len(sizes)):
+                out[t][i].copy_(P[i], non_blocking=True)
+    s.synchronize()
+    for t in range(steps):
+        for i in range(len(sizes)):
+            oracle.adamw_step(host[0][i], host_g[t][i], host[2][i], host[3][i], hp_o, 23, 5 + t, 7 + i, 0, 1.0)
+            assert mismatches(bits(out[t][i]), host[0][i]) == 0, (t, i)
+    for i in range(len(sizes)):
+        assert mismatches(bits(M[i]), host[2][i]) + mismatches(bits(V[i]), host[3][i]) == 0, i
+    plan.destroy()
+
+
+def test_multi_tensor_with_large_tensors_in_a_cuda_graph(env):
+    """The list step whose large tensors alternate between two streams, captured once and replayed: the fork and the
+    join are events inside the call, so the capture takes the plan's stream in and releases it again."""
+    oracle, binding, synth, dev = env
+    sizes = [1 << 24, 300, (1 << 24) + 8, 1 << 24, 9000]
+    P, G, M, V = [], [], [], []
+    for i, n in enumerate(sizes):
+        p, g, m, v = synth.adamw_state(n, 700 + i, dev)
+        P.append(p); G.append(g); M.append(m); V.append(v)
+    plan = binding.sr_mt_plan_create(P, G, M, V)
+    hp_o, hp_g = oracle.hparams(**HP), binding.hparams(**HP)
+    host = [[bits(t) for t in P], [bits(t) for t in G], [bits(t) for t in M], [bits(t) for t in V]]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        binding.sr_adamw_multi_tensor(plan, hp_g, 29, 11, tensor_id_base=3)       # warm-up outside the capture
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        binding.sr_adamw_multi_tensor(plan, hp_g, 29, 11, tensor_id_base=3)
+    replays = 2
+    for _ in range(replays):
+        graph.replay()
+    torch.cuda.synchronize()
+    for i in range(len(sizes)):
+        for _ in range(1 + replays):
+            oracle.adamw_step(host[0][i], host[1][i], host[2][i], host[3][i], hp_o, 29, 11, 3 + i, 0, 1.0)
+        assert mismatches(bits(P[i]), host[0][i]) + mismatches(bits(M[i]), host[2][i]) + mismatches(bits(V[i]), host[3][i]) == 0, i
+    del graph
+    plan.destroy()
+
+
 def test_multi_tensor_gpt2_350m_ten_steps(env):
     """GPT-2 350M parameter list (292 tensors, 354 823 168 elements), 10 iterations with fresh
     gradients, zero mismatches after every iteration."""
