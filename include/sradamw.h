@@ -210,7 +210,8 @@ sr_status grad_sqnorm(const void* g, sr_dtype g_dtype, uint64_t n, double* out_d
  * array of block sums, in that order, is then reduced by the later passes of grad_sqnorm.  For a
  * list of one tensor the result equals grad_sqnorm's, bit for bit; so it does for a list whose
  * tensors all have lengths that are multiples of 8192, against grad_sqnorm of their concatenation.
- * out_dev: one double on the device.  workspace: device memory of at least
+ * out_dev: one double on the device (as in grad_sqnorm it is the call's own counter while its kernels run,
+ * for lists of more than 8192 chunks).  workspace: device memory of at least
  * grad_sqnorm_multi_tensor_workspace_bytes(plan) bytes, 8-byte aligned (may be NULL when that is 0).
  * Reads the gradient pointers the plan was created with; call under the plan's device. */
 size_t grad_sqnorm_multi_tensor_workspace_bytes(const sr_mt_plan* plan);
