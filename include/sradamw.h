@@ -169,7 +169,7 @@ sr_status sr_adamw_step_host(uint16_t* p_host, const void* g_host, sr_dtype g_dt
  * whose buffers are not 16-byte aligned), plus one launch of the flat kernel per larger tensor, all enqueued by
  * the one call and all ordered inside `stream`: they start after the work enqueued on `stream` before the call
  * and whatever is enqueued on it afterwards starts after them.  With two or more large tensors every second
- * launch runs on a stream that the plan owns, forked from and joined to `stream` by events inside the call (the
+ * flat launch runs on a stream that the plan owns, forked from and joined to `stream` by events inside the call (the
  * tensors are disjoint, so the end of one launch overlaps the start of the next; the pattern can be captured in a
  * CUDA graph).  One host thread at a time may step a given plan.  A plan owns a device copy of the chunk table
  * that maps thread blocks to (tensor, range), the host-side list of the large tensors, and that stream.

@@ -497,14 +497,15 @@ sr_status sr_adamw_multi_tensor(const sr_mt_plan* plan, const sr_adamw_hparams* 
                               dev, (two && (turn++ & 1u)) ? plan->side : s);
         if (e != cudaSuccess) break;
     }
-    if (e == cudaSuccess && plan->num_small != 0)
-        e = launch_adamw_mt(plan->d_small, plan->num_small, plan->g_f32, tensor_id_base, seed_hi, hp->flags, K, S, dev,
-                            (two && (turn & 1u)) ? plan->side : s);
     if (two) {   // joined on every path: the side stream never stays forked from the caller's
         cudaError_t j = cudaEventRecord(plan->join, plan->side);
         if (j == cudaSuccess) j = cudaStreamWaitEvent(s, plan->join, 0);
         if (e == cudaSuccess) e = j;
     }
+    // the list kernel after the join: its blocks would share SMs with a flat launch's (one flat launch beside the list
+    // kernel on the GPT-2 350M list: 0.805 -> 0.822 ms), whereas two flat launches cannot share an SM
+    if (e == cudaSuccess && plan->num_small != 0)
+        e = launch_adamw_mt(plan->d_small, plan->num_small, plan->g_f32, tensor_id_base, seed_hi, hp->flags, K, S, dev, s);
     return e == cudaSuccess ? SR_OK : cuda_fail(e);
 }
 
