@@ -144,7 +144,7 @@ def _oracle_sample(synth, torch, elements: int):
     return [synth.bits16(t).copy() for t in (p, g, m, v)]
 
 
-def time_oracle(sample_elements: int, budget_s: float = 12.0):
+def time_oracle(sample_elements: int, budget_s: float = 15.0):
     """Oracle timed as it stands (OpenMP over elements) on `sample_elements` of the workload."""
     import torch
     import oracle
@@ -155,7 +155,7 @@ def time_oracle(sample_elements: int, budget_s: float = 12.0):
     times = []
     t_all = time.perf_counter()
     rep = 0
-    while rep < 8 and (rep < 1 or time.perf_counter() - t_all < budget_s):
+    while rep < 16 and (rep < 1 or time.perf_counter() - t_all < budget_s):   # about 13 s on 16 cores
         t0 = time.perf_counter()
         oracle.adamw_step(*arrs, hp, SEED, FIRST_STEP + rep)
         times.append(time.perf_counter() - t0)
